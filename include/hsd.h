@@ -1,0 +1,209 @@
+/*
+ * hsd.h — C ABI of the B200 (sm_100a) draft-verification step of Hierarchical Speculative Decoding.
+ *
+ * One call = one step of the verification operator y_hat = SpecDecode(p_theta, z, Y~) (paper Eq. 1):
+ * the target decoder scores, in a single forward over a cached prefix, every token of one or many drafts
+ * (Eq. 8, chain-shaped candidate tree: a draft token attends to the accepted tokens and, causally, to the
+ * draft tokens before it), takes the full-vocabulary argmax per row (Eq. 10), accepts the longest prefix of
+ * the draft that matches it (Eq. 9 and 11 with one candidate per node and tau = 1; with log_tau < 0 the
+ * thresholded test of Eq. 11), and emits the accepted tokens plus the correction / bonus token (Eq. 12).
+ * KV maintenance after the step (commit of the accepted rows, rollback of the rest; counted in T_decode,
+ * Sec. 4.2) is a separate call.
+ *
+ * Conventions
+ *  - All functions return an int status: HSD_OK (0) or a negative HSD_ERR_* code.  Nothing throws.
+ *  - "dev" pointers are CUDA device pointers on the current device; "host" pointers are ordinary memory.
+ *  - The library allocates NO device memory: weights, KV pool, block table, sequence lengths, workspace,
+ *    inputs and outputs are owned by the caller and must stay alive until the stream work has finished.
+ *    An hsd_ctx owns host memory only (configuration, tensor maps, profiling events).
+ *  - Every compute call is asynchronous on the given cudaStream_t (passed as void*), performs no
+ *    synchronisation and leaves its outputs on the device.
+ *  - Pending-token convention: the most recently emitted token of a sequence has no K/V yet; it is query
+ *    row 0 of the next step.  A k-token draft is therefore k+1 query rows, and full acceptance emits k+1
+ *    tokens.
+ *  - bf16 storage, fp32 accumulation, fp32 residual stream.
+ *
+ * Memory layouts (row-major, last index fastest)
+ *  - Linear weights: bf16 [out_features, in_features]  (y = x W^T).
+ *      w_qkv     [(n_heads + 2 n_kv_heads) * head_dim, d_model]   rows: q heads, k heads, v heads
+ *      w_o       [d_model, n_heads * head_dim]
+ *      w_gate_up [2 * d_ffn, d_model]                             rows: gate, then up
+ *      w_down    [d_model, d_ffn]
+ *      embed, lm_head [vocab, d_model];  *_norm [d_model] (bf16 gains)
+ *  - Paged KV pool, block = kv_block (64) tokens:
+ *      k_pool bf16 [n_layers][n_blocks][n_kv_heads][64 tokens][head_dim]
+ *      v_pool bf16 [n_layers][n_blocks][n_kv_heads][head_dim][64 tokens]      (V is stored transposed)
+ *    block_table int32 [n_slots, max_blocks_per_seq]: physical block of logical block j of slot s.
+ *    seq_lens int32 [n_slots]: committed K/V rows per slot.
+ *  - Packed query tokens: q_tokens[cu_q[i] .. cu_q[i+1]) = [pending_i, d_i1 .. d_ik].
+ */
+#ifndef HSD_H_
+#define HSD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define HSD_API __attribute__((visibility("default")))
+#else
+#define HSD_API
+#endif
+
+#define HSD_OK 0
+#define HSD_ERR_INVALID_ARG (-1)   /* null pointer, negative size, inconsistent arguments            */
+#define HSD_ERR_SHAPE (-2)         /* model shape not supported by the kernels                        */
+#define HSD_ERR_TOO_LONG (-3)      /* a sequence has more query rows than HSD_MAX_Q_LEN               */
+#define HSD_ERR_WORKSPACE (-4)     /* workspace too small or misaligned                               */
+#define HSD_ERR_KV_CAPACITY (-5)   /* declared KV capacity cannot hold the step                       */
+#define HSD_ERR_CUDA (-6)          /* a CUDA call failed; see hsd_last_cuda_error                     */
+#define HSD_ERR_DEVICE_CHECK (-7)  /* a device-side check tripped; see hsd_device_status              */
+#define HSD_ERR_NO_DEVICE (-8)     /* no usable sm_100 device                                         */
+
+#define HSD_MAX_Q_LEN 4097         /* most query rows one sequence may have in a verify call          */
+#define HSD_KV_BLOCK 64
+
+/* hsd_model_config.flags */
+#define HSD_FLAG_SIMT_DEBUG 1      /* run the plain SIMT kernels instead of the tensor-core kernels;
+                                      a slow cross-check for debugging, never a fallback              */
+#define HSD_FLAG_SIMT_ATTENTION 2  /* debugging: only the attention runs through its plain kernel     */
+
+typedef struct hsd_ctx hsd_ctx;
+
+typedef struct {
+  int n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
+  float rope_base;   /* rotary base (10000)                                                           */
+  float rms_eps;     /* RMSNorm epsilon                                                               */
+  int kv_block;      /* must be 64                                                                    */
+  int flags;         /* HSD_FLAG_*                                                                    */
+} hsd_model_config;
+
+/* Device pointers to bf16 weights.  The per-layer members are HOST arrays of n_layers device pointers. */
+typedef struct {
+  const void *embed, *lm_head, *final_norm;
+  const void *const *attn_norm, *const *w_qkv, *const *w_o;
+  const void *const *ffn_norm, *const *w_gate_up, *const *w_down;
+} hsd_weights;
+
+/* Caller-owned paged KV cache.  All pointers are device pointers. */
+typedef struct {
+  void *k_pool, *v_pool;
+  int n_blocks;               /* physical blocks per layer                                            */
+  const int *block_table;     /* [n_slots, max_blocks_per_seq]                                        */
+  int max_blocks_per_seq;
+  int *seq_lens;              /* [n_slots], updated by hsd_prefill and hsd_kv_commit                  */
+  int n_slots;
+} hsd_kv;
+
+HSD_API const char *hsd_status_string(int status);
+
+/* Create a context for one model on the current device.  Copies the configuration and the weight POINTERS
+ * (not the weights) and builds the TMA tensor maps of the weights.  Errors: INVALID_ARG, SHAPE (requires
+ * head_dim == 64, kv_block == 64, n_heads a multiple of n_kv_heads, d_model, d_ffn, vocab multiples of 64),
+ * NO_DEVICE, CUDA.  No stream work is issued. */
+HSD_API int hsd_create(const hsd_model_config *cfg, const hsd_weights *w, hsd_ctx **out);
+HSD_API int hsd_destroy(hsd_ctx *ctx);
+
+/* Bytes of device workspace a call with at most max_total_q packed query rows and max_seqs sequences
+ * needs.  The workspace must be 1024-byte aligned.  Its first 64 bytes hold the device status words
+ * (hsd_device_status); the rest is scratch that keeps nothing between calls. */
+HSD_API size_t hsd_workspace_bytes(const hsd_ctx *ctx, int max_total_q, int max_seqs);
+
+/* Support call, outside the decode loop (Sec. 4.2 excludes prefill from T_decode): run prefix rows through
+ * the decoder, write their K/V into the pool at positions seq_lens[slot] .., advance seq_lens by the row
+ * count, and return each sequence's greedy next token (the first pending token).
+ *   cu_len    dev int32 [n_seqs+1]  row offsets of the sequences in the packed input
+ *   embeds    dev bf16 [total_rows, d_model] or NULL; row r is used where token_ids[r] < 0 (visual rows)
+ *   token_ids dev int32 [total_rows]; >= 0 selects a row of the embedding table
+ *   seq_slots dev int32 [n_seqs] or NULL (= slots 0 .. n_seqs-1)
+ *   first_token dev int32 [n_seqs] out
+ *   total_rows, max_len: host copies of cu_len[n_seqs] and max_i(cu_len[i+1]-cu_len[i]) (max_len <= 32768)
+ */
+HSD_API int hsd_prefill(hsd_ctx *ctx, const hsd_kv *kv, int n_seqs, const int *cu_len, const void *embeds,
+                const int *token_ids, const int *seq_slots, int total_rows, int max_len, int *first_token,
+                void *workspace, size_t ws_bytes, void *cuda_stream);
+
+/* Stage 1, region-level verification (Eq. 2): a varlen batch of independent sequences, each
+ * [pending, draft].  Writes the speculative K/V rows of all query rows in place at positions
+ * seq_lens[slot] .. seq_lens[slot]+k (nothing is committed; seq_lens is not changed).
+ *   cu_q, q_tokens  dev int32 [n_seqs+1], [total_q]
+ *   seq_slots       dev int32 [n_seqs] or NULL (= slots 0 .. n_seqs-1)
+ *   max_q_len, total_q  host copies of max_i(k_i+1) (<= HSD_MAX_Q_LEN) and cu_q[n_seqs]
+ *   log_tau         0 = exact greedy match (the contract); < 0 = accept d iff z[d] - z_max >= log_tau
+ *   accept_len      dev int32 [n_seqs] out: accepted draft tokens a_i
+ *   emit_tokens     dev int32 [n_seqs, max_q_len] out: d_i1..d_ia, then the correction/bonus token
+ *   n_emit          dev int32 [n_seqs] out: a_i + 1
+ *   row_argmax      dev int32 [total_q] out or NULL: u_hat per row (lowest id on ties)
+ *   row_zmax        dev fp32  [total_q] out or NULL: its logit
+ *   row_zdraft      dev fp32  [total_q] out or NULL: logit of the row's next draft token (NaN on a
+ *                   sequence's last row)
+ * Device-side checks (cu_q monotone, q_i <= max_q_len, token ids in range, block table entries in range,
+ * seq_len + q_i within max_blocks_per_seq * 64) set the status words and turn the step into a no-op. */
+HSD_API int hsd_verify_regions(hsd_ctx *ctx, const hsd_kv *kv, int n_seqs, const int *cu_q, const int *q_tokens,
+                       const int *seq_slots, int max_q_len, int total_q, float log_tau, int *accept_len,
+                       int *emit_tokens, int *n_emit, int *row_argmax, float *row_zmax, float *row_zdraft,
+                       void *workspace, size_t ws_bytes, void *cuda_stream);
+
+/* Stage 2, page-level verification (Eq. 4): one sequence, one chunk of the page draft.
+ *   pending_token   dev int32 [1]: the sequence's pending token (e.g. the last entry of the previous
+ *                   call's emit_tokens)
+ *   draft_chunk     dev int32 [chunk_len], chunk_len + 1 <= HSD_MAX_Q_LEN
+ *   outputs as above with n_seqs = 1, max_q_len = chunk_len + 1. */
+HSD_API int hsd_verify_page(hsd_ctx *ctx, const hsd_kv *kv, int seq_slot, const int *pending_token,
+                    const int *draft_chunk, int chunk_len, float log_tau, int *accept_len, int *emit_tokens,
+                    int *n_emit, int *row_argmax, float *row_zmax, float *row_zdraft, void *workspace,
+                    size_t ws_bytes, void *cuda_stream);
+
+/* KV maintenance after a step: seq_lens[slot_i] += accept_len[i] + 1 (the pending row and the accepted
+ * draft rows stay; rows after them are rolled back and will be overwritten by the next step).  The caller
+ * may pass lengths other than the ones verify produced.  blocks_in_use (dev int32 [n_seqs] or NULL)
+ * receives ceil(new_len / 64). */
+HSD_API int hsd_kv_commit(hsd_ctx *ctx, const hsd_kv *kv, int n_seqs, const int *seq_slots, const int *accept_len,
+                  int *blocks_in_use, void *cuda_stream);
+
+/* Device status words written by the last call that used `workspace` (synchronises the stream).
+ * status[0] = 0 if every device-side check passed, else a code (1 cu_q not monotone, 2 sequence too long,
+ * 3 token id out of range, 4 KV capacity, 5 block table entry out of range, 6 a bounded wait gave up);
+ * status[1] = index of the offending sequence or row. */
+HSD_API int hsd_device_status(hsd_ctx *ctx, const void *workspace, void *cuda_stream, int status[4]);
+
+/* cudaError_t of the last failed CUDA call in this context (0 if none). */
+HSD_API int hsd_last_cuda_error(const hsd_ctx *ctx);
+
+/* Kernels launched by this context so far. */
+HSD_API long long hsd_launch_count(const hsd_ctx *ctx);
+
+/* Per-kernel-class timing with CUDA events on the launching stream.  enable != 0 starts recording (resets
+ * the totals); hsd_profile_read synchronises the recorded events and fills up to `cap` entries of
+ * names[i] (static strings), total_ms[i], launches[i]; returns the number of classes or a negative status.
+ * Recording adds two event records per launch; leave it off when timing whole steps. */
+HSD_API int hsd_profile_enable(hsd_ctx *ctx, int enable);
+HSD_API int hsd_profile_read(hsd_ctx *ctx, int cap, const char **names, double *total_ms, long long *launches);
+
+/* Test-only: full logits of the query rows of the LAST verify call that used `workspace`
+ * (fp32 [total_q, vocab], row-major); total_q and n_seqs must be that call's.  Slow plain kernel. */
+HSD_API int hsd_debug_logits(hsd_ctx *ctx, const void *workspace, int total_q, int n_seqs, float *logits,
+                     void *cuda_stream);
+
+/* Test-only: device address and size of a named intermediate of the last call (with that call's total_q
+ * and n_seqs) inside `workspace`:
+ * "x" fp32 [T,d_model] residual after the last layer, "h" bf16 [T,d_model] final-normed rows,
+ * "q" bf16 [T,n_heads*head_dim], "attn" bf16 [T,n_heads*head_dim], "act" bf16 [T,d_ffn] of the last layer. */
+HSD_API int hsd_debug_buffer(hsd_ctx *ctx, const void *workspace, int total_q, int n_seqs, const char *name,
+                     void **ptr, size_t *bytes);
+
+/* Test/bench-only single operators, asynchronous on the stream.
+ * hsd_op_linear: C = A W^T with the epilogue `mode`:
+ *   0 store bf16 C[M,N]; 1 fp32 C[M,N] += result (residual add); 2 SwiGLU: W is [2N', K] (gate, up), writes
+ *   bf16 C[M,N'] = silu(gate) * up with N = 2N' passed as n_out.
+ *   A dev bf16 [M,K], W dev bf16 [n_out,K].  M >= 1; K, n_out multiples of 64. */
+HSD_API int hsd_op_linear(hsd_ctx *ctx, const void *A, const void *W, void *C, int M, int n_out, int K, int mode,
+                  void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HSD_H_ */

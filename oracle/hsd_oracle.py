@@ -208,7 +208,8 @@ class CachedSequence:
             out = self.forward_rows(x, np.arange(n), causal_allowed(n))
             self.commit(range(n))
             last = out[-1:]
-        return int(np.argmax(self.model.logits(last)[0]))
+        self.last_prefill_logits = self.model.logits(last)[0]
+        return int(np.argmax(self.last_prefill_logits))
 
 
 # ----------------------------------------------------------------------------- tree + acceptance

@@ -1,0 +1,696 @@
+// C ABI of the HSD verify-step library: context, workspace carving, the per-step kernel sequence.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "hsd_kernels.h"
+
+using namespace hsd;
+
+namespace hsd {
+int launch_attn_sm100(cudaStream_t st, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                      const RowMeta& rm, const KvView& kv, const ModelDims& md, int layer, bf16* out, int T,
+                      int max_tiles, const int* tile_count, int* status, float* split_ws, int n_sms);
+}
+
+struct ProfEvent {
+  int kc;
+  cudaEvent_t a, b;
+};
+
+struct hsd_ctx {
+  hsd_model_config cfg;
+  ModelDims md;
+  const bf16 *embed, *lm_head, *final_norm;
+  std::vector<const bf16*> attn_norm, w_qkv, w_o, ffn_norm, w_gate_up, w_down;
+  std::vector<CUtensorMap> tm_qkv, tm_o, tm_gate_up, tm_down;
+  CUtensorMap tm_lm_head;
+  int n_sms;
+  int device;
+  bool simt;
+  bool attn_simt;     // attention through the plain kernel (debug)
+  int last_cuda_error;
+  long long launches;
+  bool profiling;
+  std::vector<ProfEvent> prof_events;
+  std::vector<cudaEvent_t> event_pool;
+  double prof_ms[KC_COUNT];
+  long long prof_n[KC_COUNT];
+};
+
+namespace {
+
+struct Ws {
+  int* status;        // 16 ints; [4] = attention q-tile count
+  RowMeta rm;
+  int* sel_rows;
+  int* cu_one;        // {0, n} offsets of a single-sequence call
+  float* x;
+  bf16* h;
+  bf16* q;
+  bf16* attn;
+  bf16* act;
+  float* qkv_f32;     // SIMT debug path only
+  unsigned long long* row_best;
+  float* zdraft;
+  float* split_ws;    // attention split-KV partials
+  size_t bytes;
+};
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Split-KV partial results: per (q-tile row, q head, split) an fp32 accumulator row plus (max, sum).
+constexpr int kMaxSplits = 16;
+inline size_t split_ws_floats(const ModelDims& md, int T) {
+  return (size_t)T * md.Hq * kMaxSplits * (md.D + 2);
+}
+
+Ws carve(const hsd_ctx* c, void* base, int T, int S) {
+  const ModelDims& md = c->md;
+  Ws w;
+  size_t off = 0;
+  char* p = static_cast<char*>(base);
+  auto take = [&](size_t bytes) {
+    void* r = p ? p + off : nullptr;
+    off = align_up(off + bytes, 1024);
+    return r;
+  };
+  w.status = static_cast<int*>(take(64));
+  w.rm.row_seq = static_cast<int*>(take(sizeof(int) * T));
+  w.rm.row_pos = static_cast<int*>(take(sizeof(int) * T));
+  w.rm.row_tok = static_cast<int*>(take(sizeof(int) * T));
+  w.rm.row_kv = static_cast<int*>(take(sizeof(int) * T));
+  w.rm.row_next = static_cast<int*>(take(sizeof(int) * T));
+  w.rm.rope_cs = static_cast<float2*>(take(sizeof(float2) * (size_t)T * (md.D / 2)));
+  w.rm.seq_q0 = static_cast<int*>(take(sizeof(int) * S));
+  w.rm.seq_n = static_cast<int*>(take(sizeof(int) * S));
+  w.rm.seq_len = static_cast<int*>(take(sizeof(int) * S));
+  w.rm.seq_slot = static_cast<int*>(take(sizeof(int) * S));
+  w.rm.seq_tile0 = static_cast<int*>(take(sizeof(int) * (S + 1)));
+  w.sel_rows = static_cast<int*>(take(sizeof(int) * S));
+  w.cu_one = static_cast<int*>(take(sizeof(int) * 2));
+  w.x = static_cast<float*>(take(sizeof(float) * (size_t)T * md.d));
+  w.h = static_cast<bf16*>(take(2 * (size_t)T * md.d));
+  w.q = static_cast<bf16*>(take(2 * (size_t)T * md.Hq * md.D));
+  w.attn = static_cast<bf16*>(take(2 * (size_t)T * md.Hq * md.D));
+  w.act = static_cast<bf16*>(take(2 * (size_t)T * md.ffn));
+  w.qkv_f32 = c->simt ? static_cast<float*>(take(sizeof(float) * (size_t)T * md.qkv_out)) : nullptr;
+  w.row_best = static_cast<unsigned long long*>(take(sizeof(unsigned long long) * T));
+  w.zdraft = static_cast<float*>(take(sizeof(float) * T));
+  w.split_ws = c->simt ? nullptr : static_cast<float*>(take(sizeof(float) * split_ws_floats(md, T)));
+  w.bytes = off;
+  return w;
+}
+
+struct Scope {   // brackets one launch: counts it and, when profiling, records events around it
+  hsd_ctx* c;
+  cudaStream_t st;
+  int idx;
+  Scope(hsd_ctx* c_, cudaStream_t st_, int kc) : c(c_), st(st_), idx(-1) {
+    c->launches++;
+    if (!c->profiling) return;
+    ProfEvent e;
+    e.kc = kc;
+    cudaEvent_t ev[2];
+    for (int i = 0; i < 2; ++i) {
+      if (!c->event_pool.empty()) {
+        ev[i] = c->event_pool.back();
+        c->event_pool.pop_back();
+      } else if (cudaEventCreate(&ev[i]) != cudaSuccess) {
+        return;
+      }
+    }
+    e.a = ev[0];
+    e.b = ev[1];
+    cudaEventRecord(e.a, st);
+    c->prof_events.push_back(e);
+    idx = (int)c->prof_events.size() - 1;
+  }
+  ~Scope() {
+    if (idx >= 0) cudaEventRecord(c->prof_events[idx].b, st);
+  }
+};
+
+int fail_cuda(hsd_ctx* c) {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) c->last_cuda_error = (int)e;
+  return HSD_ERR_CUDA;
+}
+
+int check_cuda(hsd_ctx* c) {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) {
+    c->last_cuda_error = (int)e;
+    return HSD_ERR_CUDA;
+  }
+  return HSD_OK;
+}
+
+KvView kv_view(const hsd_kv* kv) {
+  KvView v;
+  v.k_pool = static_cast<bf16*>(kv->k_pool);
+  v.v_pool = static_cast<bf16*>(kv->v_pool);
+  v.n_blocks = kv->n_blocks;
+  v.block_table = kv->block_table;
+  v.max_blocks = kv->max_blocks_per_seq;
+  v.seq_lens = kv->seq_lens;
+  v.n_slots = kv->n_slots;
+  return v;
+}
+
+int check_kv(const hsd_kv* kv) {
+  if (!kv || !kv->k_pool || !kv->v_pool || !kv->block_table || !kv->seq_lens) return HSD_ERR_INVALID_ARG;
+  if (kv->n_blocks <= 0 || kv->max_blocks_per_seq <= 0 || kv->n_slots <= 0) return HSD_ERR_INVALID_ARG;
+  return HSD_OK;
+}
+
+struct StepArgs {
+  int n_seqs, total_q, max_q_len;
+  bool prefill;
+  const int* cu_q;
+  const int* tokens;
+  const int* pending;
+  const int* draft;
+  const void* embeds;
+  const int* seq_slots;
+  int slot_base;
+};
+
+// The decoder forward over one packed batch: rows -> residual stream x after the last layer.
+int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cudaStream_t st) {
+  const ModelDims& md = c->md;
+  const KvView kv = kv_view(kvp);
+  const int T = a.total_q;
+  const int tokens_per_tile = 128 / md.group;
+
+  if (cudaMemsetAsync(w.status, 0, 64, st) != cudaSuccess) return check_cuda(c);
+  {
+    Scope s(c, st, KC_SETUP);
+    SetupArgs sa;
+    sa.n_seqs = a.n_seqs;
+    sa.total_q = a.total_q;
+    sa.max_q_len = a.max_q_len;
+    sa.vocab = md.V;
+    sa.tokens_per_tile = tokens_per_tile;
+    sa.cu_q = a.cu_q;
+    sa.tokens = a.tokens;
+    sa.pending = a.pending;
+    sa.draft = a.draft;
+    sa.seq_slots = a.seq_slots;
+    sa.slot_base = a.slot_base;
+    sa.allow_embed_rows = a.prefill && a.embeds != nullptr;
+    sa.rope_base = md.rope_base;
+    sa.head_dim = md.D;
+    launch_setup_rows(st, sa, kv, w.rm, w.status, w.status + 4);
+  }
+  {
+    Scope s(c, st, KC_EMBED);
+    launch_embed(st, w.rm, c->embed, static_cast<const bf16*>(a.embeds), w.x, T, md.d, w.status);
+  }
+
+  CUtensorMap tm_h, tm_attn, tm_act, tm_q, tm_k, tm_v;
+  const int max_tiles = T / tokens_per_tile + a.n_seqs;
+  if (!c->simt) {
+    if (make_tmap_2d(&tm_h, w.h, T, md.d, 128) || make_tmap_2d(&tm_attn, w.attn, T, md.Hq * md.D, 128) ||
+        make_tmap_2d(&tm_act, w.act, T, md.ffn, 128))
+      return HSD_ERR_CUDA;
+    // q as [T][Hq][64]: one box = (128/group) tokens x group heads x 64 dims -> a 128-row MMA operand
+    if (make_tmap_3d(&tm_q, w.q, 64, md.Hq, T, 128, (uint64_t)md.Hq * 128, 64, md.group, tokens_per_tile))
+      return HSD_ERR_CUDA;
+    // K / V^T pools as 2-D [rows, 64]: one (layer, block, kv head) tile = 64 consecutive rows
+    const uint64_t pool_rows = (uint64_t)md.n_layers * kv.n_blocks * md.Hkv * 64;
+    if (make_tmap_2d(&tm_k, kv.k_pool, pool_rows, 64, 64) || make_tmap_2d(&tm_v, kv.v_pool, pool_rows, 64, 64))
+      return HSD_ERR_CUDA;
+  }
+
+  for (int l = 0; l < md.n_layers; ++l) {
+    {
+      Scope s(c, st, KC_RMSNORM);
+      launch_rmsnorm(st, w.x, c->attn_norm[l], w.h, T, md.d, md.eps, nullptr);
+    }
+    const size_t layer_elems = (size_t)kv.n_blocks * md.Hkv * 64 * 64;
+    if (c->simt) {
+      {
+        Scope s(c, st, KC_GEMM_QKV);
+        GemmOut o = {w.qkv_f32, md.qkv_out, nullptr, nullptr, nullptr};
+        launch_gemm_simt(st, w.h, c->w_qkv[l], T, md.qkv_out, md.d, GM_STORE_F32, o);
+      }
+      {
+        Scope s(c, st, KC_ROPE_KV);
+        launch_rope_kvwrite(st, w.qkv_f32, w.rm, kv, md, l, w.q, T, w.status);
+      }
+      {
+        Scope s(c, st, KC_ATTN);
+        launch_attn_simt(st, w.q, w.rm, kv, md, l, w.attn, T, w.status);
+      }
+      {
+        Scope s(c, st, KC_GEMM_O);
+        GemmOut o = {w.x, md.d, nullptr, nullptr, nullptr};
+        launch_gemm_simt(st, w.attn, c->w_o[l], T, md.d, md.Hq * md.D, GM_ADD_F32, o);
+      }
+    } else {
+      {
+        Scope s(c, st, KC_GEMM_QKV);
+        GemmSm100Args g = {};
+        g.tmA = tm_h;
+        g.tmB = c->tm_qkv[l];
+        g.M = T; g.n_out = md.qkv_out; g.K = md.d; g.mode = GS_QKV_ROPE;
+        g.qkv.row_kv = w.rm.row_kv;
+        g.qkv.rope_cs = w.rm.rope_cs;
+        g.qkv.q_out = w.q;
+        g.qkv.k_pool_layer = kv.k_pool + (size_t)l * layer_elems;
+        g.qkv.v_pool_layer = kv.v_pool + (size_t)l * layer_elems;
+        g.qkv.Hq = md.Hq; g.qkv.Hkv = md.Hkv;
+        g.status = w.status; g.n_sms = c->n_sms;
+        if (launch_gemm_sm100(st, g)) return fail_cuda(c);
+      }
+      {
+        Scope s(c, st, KC_ATTN);
+        if (c->attn_simt) {
+          launch_attn_simt(st, w.q, w.rm, kv, md, l, w.attn, T, w.status);
+        } else if (launch_attn_sm100(st, tm_q, tm_k, tm_v, w.rm, kv, md, l, w.attn, T, max_tiles, w.status + 4,
+                                     w.status, w.split_ws, c->n_sms)) {
+          return fail_cuda(c);
+        }
+      }
+      {
+        Scope s(c, st, KC_GEMM_O);
+        GemmSm100Args g = {};
+        g.tmA = tm_attn;
+        g.tmB = c->tm_o[l];
+        g.M = T; g.n_out = md.d; g.K = md.Hq * md.D; g.mode = GS_ADD_F32;
+        g.out.C = w.x; g.out.ldc = md.d;
+        g.status = w.status; g.n_sms = c->n_sms;
+        if (launch_gemm_sm100(st, g)) return HSD_ERR_CUDA;
+      }
+    }
+    {
+      Scope s(c, st, KC_RMSNORM);
+      launch_rmsnorm(st, w.x, c->ffn_norm[l], w.h, T, md.d, md.eps, nullptr);
+    }
+    if (c->simt) {
+      {
+        Scope s(c, st, KC_GEMM_GATEUP);
+        GemmOut o = {w.act, md.ffn, nullptr, nullptr, nullptr};
+        launch_gemm_simt(st, w.h, c->w_gate_up[l], T, 2 * md.ffn, md.d, GM_SWIGLU, o);
+      }
+      {
+        Scope s(c, st, KC_GEMM_DOWN);
+        GemmOut o = {w.x, md.d, nullptr, nullptr, nullptr};
+        launch_gemm_simt(st, w.act, c->w_down[l], T, md.d, md.ffn, GM_ADD_F32, o);
+      }
+    } else {
+      {
+        Scope s(c, st, KC_GEMM_GATEUP);
+        GemmSm100Args g = {};
+        g.tmA = tm_h;
+        g.tmB = c->tm_gate_up[l];
+        g.M = T; g.n_out = 2 * md.ffn; g.K = md.d; g.mode = GS_SWIGLU;
+        g.out.C = w.act; g.out.ldc = md.ffn;
+        g.status = w.status; g.n_sms = c->n_sms;
+        if (launch_gemm_sm100(st, g)) return HSD_ERR_CUDA;
+      }
+      {
+        Scope s(c, st, KC_GEMM_DOWN);
+        GemmSm100Args g = {};
+        g.tmA = tm_act;
+        g.tmB = c->tm_down[l];
+        g.M = T; g.n_out = md.d; g.K = md.ffn; g.mode = GS_ADD_F32;
+        g.out.C = w.x; g.out.ldc = md.d;
+        g.status = w.status; g.n_sms = c->n_sms;
+        if (launch_gemm_sm100(st, g)) return HSD_ERR_CUDA;
+      }
+    }
+  }
+  return check_cuda(c);
+}
+
+// Final norm + LM head + running argmax over `rows` rows of h (already selected / normalised into w.h).
+int run_lm_head(hsd_ctx* c, const Ws& w, int rows, const int* row_next, cudaStream_t st) {
+  const ModelDims& md = c->md;
+  {
+    Scope s(c, st, KC_LMHEAD);
+    launch_clear_best(st, w.row_best, w.zdraft, rows);
+  }
+  Scope s(c, st, KC_LMHEAD);
+  GemmOut o = {nullptr, 0, w.row_best, w.zdraft, row_next};
+  if (c->simt) {
+    launch_gemm_simt(st, w.h, c->lm_head, rows, md.V, md.d, GM_ARGMAX, o);
+  } else {
+    CUtensorMap tm_h;
+    if (make_tmap_2d(&tm_h, w.h, rows, md.d, 128)) return HSD_ERR_CUDA;
+    GemmSm100Args g = {};
+    g.tmA = tm_h;
+    g.tmB = c->tm_lm_head;
+    g.M = rows; g.n_out = md.V; g.K = md.d; g.mode = GS_ARGMAX;
+    g.out = o;
+    g.status = w.status; g.n_sms = c->n_sms;
+    if (launch_gemm_sm100(st, g)) return HSD_ERR_CUDA;
+  }
+  return check_cuda(c);
+}
+
+int check_ws(const hsd_ctx* c, void* workspace, size_t ws_bytes, int T, int S) {
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 1023)) return HSD_ERR_WORKSPACE;
+  if (hsd_workspace_bytes(c, T, S) > ws_bytes) return HSD_ERR_WORKSPACE;
+  return HSD_OK;
+}
+
+int verify_common(hsd_ctx* c, const hsd_kv* kv, const StepArgs& a, float log_tau, int* accept_len, int* emit_tokens,
+                  int* n_emit, int* row_argmax, float* row_zmax, float* row_zdraft, void* workspace, size_t ws_bytes,
+                  cudaStream_t st) {
+  int rc = check_ws(c, workspace, ws_bytes, a.total_q, a.n_seqs);
+  if (rc) return rc;
+  const Ws w = carve(c, workspace, a.total_q, a.n_seqs);
+  rc = run_layers(c, kv, a, w, st);
+  if (rc) return rc;
+  {
+    Scope s(c, st, KC_RMSNORM);
+    launch_rmsnorm(st, w.x, c->final_norm, w.h, a.total_q, c->md.d, c->md.eps, nullptr);
+  }
+  rc = run_lm_head(c, w, a.total_q, w.rm.row_next, st);
+  if (rc) return rc;
+  {
+    Scope s(c, st, KC_ACCEPT);
+    AcceptArgs aa;
+    aa.n_seqs = a.n_seqs;
+    aa.max_q_len = a.max_q_len;
+    aa.log_tau = log_tau;
+    aa.row_best = w.row_best;
+    aa.zdraft = w.zdraft;
+    aa.accept_len = accept_len;
+    aa.emit_tokens = emit_tokens;
+    aa.n_emit = n_emit;
+    aa.row_argmax = row_argmax;
+    aa.row_zmax = row_zmax;
+    aa.row_zdraft = row_zdraft;
+    launch_accept(st, aa, w.rm, w.status);
+  }
+  return check_cuda(c);
+}
+
+}  // namespace
+
+// =================================================================================================
+extern "C" {
+
+const char* hsd_status_string(int s) {
+  switch (s) {
+    case HSD_OK: return "ok";
+    case HSD_ERR_INVALID_ARG: return "invalid argument";
+    case HSD_ERR_SHAPE: return "unsupported model shape";
+    case HSD_ERR_TOO_LONG: return "sequence has too many query rows";
+    case HSD_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case HSD_ERR_KV_CAPACITY: return "KV capacity exceeded";
+    case HSD_ERR_CUDA: return "CUDA error";
+    case HSD_ERR_DEVICE_CHECK: return "device-side check failed";
+    case HSD_ERR_NO_DEVICE: return "no usable sm_100 device";
+    default: return "unknown status";
+  }
+}
+
+int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out) {
+  if (!cfg || !w || !out) return HSD_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (cfg->n_layers <= 0 || cfg->d_model <= 0 || cfg->n_heads <= 0 || cfg->n_kv_heads <= 0 || cfg->d_ffn <= 0 ||
+      cfg->vocab <= 0)
+    return HSD_ERR_INVALID_ARG;
+  if (cfg->head_dim != 64 || cfg->kv_block != HSD_KV_BLOCK) return HSD_ERR_SHAPE;
+  if (cfg->n_heads % cfg->n_kv_heads) return HSD_ERR_SHAPE;
+  const int group = cfg->n_heads / cfg->n_kv_heads;
+  if (128 % group) return HSD_ERR_SHAPE;
+  const int dv = cfg->d_model / 128;
+  if (cfg->d_model % 128 || !(dv == 1 || dv == 2 || dv == 4 || dv == 8 || dv == 16)) return HSD_ERR_SHAPE;
+  if (cfg->d_ffn % 64 || cfg->vocab % 64) return HSD_ERR_SHAPE;
+  if (!w->embed || !w->lm_head || !w->final_norm || !w->attn_norm || !w->w_qkv || !w->w_o || !w->ffn_norm ||
+      !w->w_gate_up || !w->w_down)
+    return HSD_ERR_INVALID_ARG;
+  for (int l = 0; l < cfg->n_layers; ++l)
+    if (!w->attn_norm[l] || !w->w_qkv[l] || !w->w_o[l] || !w->ffn_norm[l] || !w->w_gate_up[l] || !w->w_down[l])
+      return HSD_ERR_INVALID_ARG;
+
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return HSD_ERR_NO_DEVICE;
+  if (prop.major != 10) return HSD_ERR_NO_DEVICE;
+
+  hsd_ctx* c = new (std::nothrow) hsd_ctx();
+  if (!c) return HSD_ERR_INVALID_ARG;
+  c->cfg = *cfg;
+  ModelDims& md = c->md;
+  md.n_layers = cfg->n_layers; md.d = cfg->d_model; md.Hq = cfg->n_heads; md.Hkv = cfg->n_kv_heads; md.D = 64;
+  md.ffn = cfg->d_ffn; md.V = cfg->vocab; md.qkv_out = (md.Hq + 2 * md.Hkv) * 64; md.group = group;
+  md.rope_base = cfg->rope_base; md.eps = cfg->rms_eps;
+  c->embed = static_cast<const bf16*>(w->embed);
+  c->lm_head = static_cast<const bf16*>(w->lm_head);
+  c->final_norm = static_cast<const bf16*>(w->final_norm);
+  for (int l = 0; l < md.n_layers; ++l) {
+    c->attn_norm.push_back(static_cast<const bf16*>(w->attn_norm[l]));
+    c->w_qkv.push_back(static_cast<const bf16*>(w->w_qkv[l]));
+    c->w_o.push_back(static_cast<const bf16*>(w->w_o[l]));
+    c->ffn_norm.push_back(static_cast<const bf16*>(w->ffn_norm[l]));
+    c->w_gate_up.push_back(static_cast<const bf16*>(w->w_gate_up[l]));
+    c->w_down.push_back(static_cast<const bf16*>(w->w_down[l]));
+  }
+  c->n_sms = prop.multiProcessorCount;
+  c->device = dev;
+  c->simt = (cfg->flags & HSD_FLAG_SIMT_DEBUG) != 0;
+  c->attn_simt = c->simt || (cfg->flags & HSD_FLAG_SIMT_ATTENTION) != 0;
+  c->last_cuda_error = 0;
+  c->launches = 0;
+  c->profiling = false;
+  memset(c->prof_ms, 0, sizeof(c->prof_ms));
+  memset(c->prof_n, 0, sizeof(c->prof_n));
+  if (!c->simt) {
+    if (tma_init()) { delete c; return HSD_ERR_CUDA; }
+    c->tm_qkv.resize(md.n_layers); c->tm_o.resize(md.n_layers);
+    c->tm_gate_up.resize(md.n_layers); c->tm_down.resize(md.n_layers);
+    int bad = 0;
+    for (int l = 0; l < md.n_layers; ++l) {
+      bad |= make_tmap_2d(&c->tm_qkv[l], c->w_qkv[l], md.qkv_out, md.d, 64);
+      bad |= make_tmap_2d(&c->tm_o[l], c->w_o[l], md.d, md.Hq * 64, 64);
+      bad |= make_tmap_2d(&c->tm_gate_up[l], c->w_gate_up[l], 2 * md.ffn, md.d, 64);
+      bad |= make_tmap_2d(&c->tm_down[l], c->w_down[l], md.d, md.ffn, 64);
+    }
+    bad |= make_tmap_2d(&c->tm_lm_head, c->lm_head, md.V, md.d, 64);
+    if (bad) { delete c; return HSD_ERR_CUDA; }
+  }
+  *out = c;
+  return HSD_OK;
+}
+
+int hsd_destroy(hsd_ctx* c) {
+  if (!c) return HSD_ERR_INVALID_ARG;
+  for (auto& e : c->prof_events) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
+  for (auto& e : c->event_pool) cudaEventDestroy(e);
+  delete c;
+  return HSD_OK;
+}
+
+size_t hsd_workspace_bytes(const hsd_ctx* c, int max_total_q, int max_seqs) {
+  if (!c || max_total_q <= 0 || max_seqs <= 0) return 0;
+  return carve(c, nullptr, max_total_q, max_seqs).bytes;
+}
+
+int hsd_prefill(hsd_ctx* c, const hsd_kv* kv, int n_seqs, const int* cu_len, const void* embeds, const int* token_ids,
+                const int* seq_slots, int total_rows, int max_len, int* first_token, void* workspace, size_t ws_bytes,
+                void* cuda_stream) {
+  if (!c || !cu_len || !token_ids || !first_token) return HSD_ERR_INVALID_ARG;
+  if (n_seqs <= 0 || total_rows <= 0 || max_len <= 0 || max_len > total_rows) return HSD_ERR_INVALID_ARG;
+  if (max_len > 32768) return HSD_ERR_TOO_LONG;
+  int rc = check_kv(kv);
+  if (rc) return rc;
+  if ((long long)max_len > (long long)kv->max_blocks_per_seq * HSD_KV_BLOCK) return HSD_ERR_KV_CAPACITY;
+  rc = check_ws(c, workspace, ws_bytes, total_rows, n_seqs);
+  if (rc) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const Ws w = carve(c, workspace, total_rows, n_seqs);
+  StepArgs a = {};
+  a.n_seqs = n_seqs; a.total_q = total_rows; a.max_q_len = max_len; a.prefill = true;
+  a.cu_q = cu_len; a.tokens = token_ids; a.embeds = embeds; a.seq_slots = seq_slots; a.slot_base = 0;
+  rc = run_layers(c, kv, a, w, st);
+  if (rc) return rc;
+  {
+    Scope s(c, st, KC_RMSNORM);
+    launch_select_last_rows(st, w.rm, n_seqs, w.sel_rows);
+  }
+  {
+    Scope s(c, st, KC_RMSNORM);
+    launch_rmsnorm(st, w.x, c->final_norm, w.h, n_seqs, c->md.d, c->md.eps, w.sel_rows);
+  }
+  rc = run_lm_head(c, w, n_seqs, nullptr, st);
+  if (rc) return rc;
+  {
+    Scope s(c, st, KC_ACCEPT);
+    launch_first_token(st, w.row_best, n_seqs, first_token, w.rm, kv_view(kv), w.status);
+  }
+  return check_cuda(c);
+}
+
+int hsd_verify_regions(hsd_ctx* c, const hsd_kv* kv, int n_seqs, const int* cu_q, const int* q_tokens,
+                       const int* seq_slots, int max_q_len, int total_q, float log_tau, int* accept_len,
+                       int* emit_tokens, int* n_emit, int* row_argmax, float* row_zmax, float* row_zdraft,
+                       void* workspace, size_t ws_bytes, void* cuda_stream) {
+  if (!c || !cu_q || !q_tokens || !accept_len || !emit_tokens || !n_emit) return HSD_ERR_INVALID_ARG;
+  if (n_seqs <= 0 || total_q <= 0 || max_q_len <= 0 || max_q_len > total_q) return HSD_ERR_INVALID_ARG;
+  if (!(log_tau <= 0.f)) return HSD_ERR_INVALID_ARG;
+  if (max_q_len > HSD_MAX_Q_LEN) return HSD_ERR_TOO_LONG;
+  int rc = check_kv(kv);
+  if (rc) return rc;
+  if ((long long)max_q_len > (long long)kv->max_blocks_per_seq * HSD_KV_BLOCK) return HSD_ERR_KV_CAPACITY;
+  StepArgs a = {};
+  a.n_seqs = n_seqs; a.total_q = total_q; a.max_q_len = max_q_len; a.prefill = false;
+  a.cu_q = cu_q; a.tokens = q_tokens; a.seq_slots = seq_slots; a.slot_base = 0;
+  return verify_common(c, kv, a, log_tau, accept_len, emit_tokens, n_emit, row_argmax, row_zmax, row_zdraft, workspace,
+                       ws_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+}  // extern "C"
+
+namespace {
+// cu_q = {0, n} of a single-sequence call.
+__global__ void page_cu_q_kernel(int* cu, int n) {
+  cu[0] = 0;
+  cu[1] = n;
+}
+}  // namespace
+
+extern "C" {
+
+int hsd_verify_page(hsd_ctx* c, const hsd_kv* kv, int seq_slot, const int* pending_token, const int* draft_chunk,
+                    int chunk_len, float log_tau, int* accept_len, int* emit_tokens, int* n_emit, int* row_argmax,
+                    float* row_zmax, float* row_zdraft, void* workspace, size_t ws_bytes, void* cuda_stream) {
+  if (!c || !pending_token || !accept_len || !emit_tokens || !n_emit) return HSD_ERR_INVALID_ARG;
+  if (chunk_len < 0 || (chunk_len > 0 && !draft_chunk)) return HSD_ERR_INVALID_ARG;
+  if (!(log_tau <= 0.f)) return HSD_ERR_INVALID_ARG;
+  if (chunk_len + 1 > HSD_MAX_Q_LEN) return HSD_ERR_TOO_LONG;
+  int rc = check_kv(kv);
+  if (rc) return rc;
+  if (seq_slot < 0 || seq_slot >= kv->n_slots) return HSD_ERR_INVALID_ARG;
+  if ((long long)chunk_len + 1 > (long long)kv->max_blocks_per_seq * HSD_KV_BLOCK) return HSD_ERR_KV_CAPACITY;
+  rc = check_ws(c, workspace, ws_bytes, chunk_len + 1, 1);
+  if (rc) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const Ws w = carve(c, workspace, chunk_len + 1, 1);
+  int* cu = w.cu_one;
+  {
+    Scope s(c, st, KC_SETUP);
+    page_cu_q_kernel<<<1, 1, 0, st>>>(cu, chunk_len + 1);
+  }
+  StepArgs a = {};
+  a.n_seqs = 1; a.total_q = chunk_len + 1; a.max_q_len = chunk_len + 1; a.prefill = false;
+  a.cu_q = cu; a.tokens = nullptr; a.pending = pending_token; a.draft = draft_chunk;
+  a.seq_slots = nullptr; a.slot_base = seq_slot;
+  return verify_common(c, kv, a, log_tau, accept_len, emit_tokens, n_emit, row_argmax, row_zmax, row_zdraft, workspace,
+                       ws_bytes, st);
+}
+
+int hsd_kv_commit(hsd_ctx* c, const hsd_kv* kv, int n_seqs, const int* seq_slots, const int* accept_len,
+                  int* blocks_in_use, void* cuda_stream) {
+  if (!c || !accept_len || n_seqs <= 0) return HSD_ERR_INVALID_ARG;
+  int rc = check_kv(kv);
+  if (rc) return rc;
+  if (!seq_slots && n_seqs > kv->n_slots) return HSD_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  Scope s(c, st, KC_COMMIT);
+  launch_commit(st, kv_view(kv), n_seqs, seq_slots, accept_len, blocks_in_use);
+  return check_cuda(c);
+}
+
+int hsd_device_status(hsd_ctx* c, const void* workspace, void* cuda_stream, int status[4]) {
+  if (!c || !workspace || !status) return HSD_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(status, workspace, 4 * sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return fail_cuda(c);
+  return status[0] ? HSD_ERR_DEVICE_CHECK : HSD_OK;
+}
+
+int hsd_last_cuda_error(const hsd_ctx* c) { return c ? c->last_cuda_error : 0; }
+long long hsd_launch_count(const hsd_ctx* c) { return c ? c->launches : 0; }
+
+int hsd_profile_enable(hsd_ctx* c, int enable) {
+  if (!c) return HSD_ERR_INVALID_ARG;
+  for (auto& e : c->prof_events) { c->event_pool.push_back(e.a); c->event_pool.push_back(e.b); }
+  c->prof_events.clear();
+  memset(c->prof_ms, 0, sizeof(c->prof_ms));
+  memset(c->prof_n, 0, sizeof(c->prof_n));
+  c->profiling = enable != 0;
+  return HSD_OK;
+}
+
+int hsd_profile_read(hsd_ctx* c, int cap, const char** names, double* total_ms, long long* launches) {
+  if (!c || cap < 0) return HSD_ERR_INVALID_ARG;
+  for (auto& e : c->prof_events) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(e.b) != cudaSuccess || cudaEventElapsedTime(&ms, e.a, e.b) != cudaSuccess)
+      return fail_cuda(c);
+    c->prof_ms[e.kc] += ms;
+    c->prof_n[e.kc] += 1;
+    c->event_pool.push_back(e.a);
+    c->event_pool.push_back(e.b);
+  }
+  c->prof_events.clear();
+  int n = 0;
+  for (int k = 0; k < KC_COUNT; ++k) {
+    if (!c->prof_n[k]) continue;
+    if (n < cap) {
+      if (names) names[n] = kernel_class_name(k);
+      if (total_ms) total_ms[n] = c->prof_ms[k];
+      if (launches) launches[n] = c->prof_n[k];
+    }
+    ++n;
+  }
+  return n;
+}
+
+int hsd_debug_logits(hsd_ctx* c, const void* workspace, int total_q, int n_seqs, float* logits, void* cuda_stream) {
+  if (!c || !workspace || !logits || total_q <= 0 || n_seqs <= 0) return HSD_ERR_INVALID_ARG;
+  const Ws w = carve(c, const_cast<void*>(workspace), total_q, n_seqs);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  Scope s(c, st, KC_DEBUG);
+  GemmOut o = {logits, c->md.V, nullptr, nullptr, nullptr};
+  launch_gemm_simt(st, w.h, c->lm_head, total_q, c->md.V, c->md.d, GM_STORE_F32, o);
+  return check_cuda(c);
+}
+
+int hsd_debug_buffer(hsd_ctx* c, const void* workspace, int total_q, int n_seqs, const char* name, void** ptr,
+                     size_t* bytes) {
+  if (!c || !workspace || !name || !ptr || !bytes || total_q <= 0 || n_seqs <= 0) return HSD_ERR_INVALID_ARG;
+  const Ws w = carve(c, const_cast<void*>(workspace), total_q, n_seqs);
+  const ModelDims& md = c->md;
+  const size_t T = (size_t)total_q;
+  if (!strcmp(name, "x")) { *ptr = w.x; *bytes = 4 * T * md.d; }
+  else if (!strcmp(name, "h")) { *ptr = w.h; *bytes = 2 * T * md.d; }
+  else if (!strcmp(name, "q")) { *ptr = w.q; *bytes = 2 * T * md.Hq * md.D; }
+  else if (!strcmp(name, "attn")) { *ptr = w.attn; *bytes = 2 * T * md.Hq * md.D; }
+  else if (!strcmp(name, "act")) { *ptr = w.act; *bytes = 2 * T * md.ffn; }
+  else return HSD_ERR_INVALID_ARG;
+  return HSD_OK;
+}
+
+int hsd_op_linear(hsd_ctx* c, const void* A, const void* W, void* C, int M, int n_out, int K, int mode,
+                  void* cuda_stream) {
+  if (!c || !A || !W || !C || M <= 0 || n_out <= 0 || K <= 0) return HSD_ERR_INVALID_ARG;
+  if (K % 64 || n_out % 64 || mode < 0 || mode > 2 || (mode == 2 && n_out % 128)) return HSD_ERR_SHAPE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int ldc = mode == 2 ? n_out / 2 : n_out;
+  Scope s(c, st, KC_DEBUG);
+  if (c->simt) {
+    GemmOut o = {C, ldc, nullptr, nullptr, nullptr};
+    launch_gemm_simt(st, static_cast<const bf16*>(A), static_cast<const bf16*>(W), M, n_out, K, mode, o);
+    return check_cuda(c);
+  }
+  GemmSm100Args g = {};
+  if (make_tmap_2d(&g.tmA, A, M, K, 128) || make_tmap_2d(&g.tmB, W, n_out, K, 64)) return HSD_ERR_CUDA;
+  g.M = M; g.n_out = n_out; g.K = K; g.mode = mode;
+  g.out.C = C; g.out.ldc = ldc;
+  g.status = nullptr; g.n_sms = c->n_sms;
+  if (launch_gemm_sm100(st, g)) return fail_cuda(c);
+  return check_cuda(c);
+}
+
+}  // extern "C"

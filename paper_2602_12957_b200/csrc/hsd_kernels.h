@@ -1,0 +1,119 @@
+// Host-side launchers of the library's kernels (one translation unit per kernel family).
+#pragma once
+
+#include "hsd_common.cuh"
+
+namespace hsd {
+
+typedef __nv_bfloat16 bf16;
+
+struct ModelDims {
+  int n_layers, d, Hq, Hkv, D, ffn, V, qkv_out, group;
+  float rope_base, eps;
+};
+
+// The paged KV cache as the kernels see it.
+struct KvView {
+  bf16* k_pool;
+  bf16* v_pool;
+  int n_blocks;
+  const int* block_table;
+  int max_blocks;
+  int* seq_lens;
+  int n_slots;
+};
+
+// Launch bookkeeping: counts launches and, when profiling is on, brackets each with CUDA events.
+struct Launcher;
+enum KernelClass {
+  KC_SETUP = 0, KC_EMBED, KC_RMSNORM, KC_GEMM_QKV, KC_ROPE_KV, KC_ATTN, KC_ATTN_COMBINE, KC_GEMM_O, KC_GEMM_GATEUP,
+  KC_GEMM_DOWN, KC_LMHEAD, KC_ACCEPT, KC_COMMIT, KC_DEBUG, KC_COUNT
+};
+const char* kernel_class_name(int kc);
+
+// ---- small kernels (hsd_small.cu) ---------------------------------------------------------------
+struct SetupArgs {
+  int n_seqs, total_q, max_q_len, vocab, tokens_per_tile;
+  const int* cu_q;          // dev [S+1]
+  const int* tokens;        // dev [T] or nullptr (page mode)
+  const int* pending;       // dev [1] page mode: token of row 0
+  const int* draft;         // dev [T-1] page mode: tokens of rows 1..
+  const int* seq_slots;     // dev [S] or nullptr
+  int slot_base;            // slot of sequence 0 when seq_slots == nullptr
+  int allow_embed_rows;     // prefill: token id < 0 means "use the embeds row"
+  float rope_base;
+  int head_dim;
+};
+void launch_setup_rows(cudaStream_t st, const SetupArgs& a, const KvView& kv, const RowMeta& rm, int* status,
+                       int* tile_count);
+void launch_embed(cudaStream_t st, const RowMeta& rm, const bf16* table, const bf16* embeds, float* x, int T, int d,
+                  const int* status);
+// h[r] = bf16(rmsnorm(x[src]) * gain), src = sel_rows ? sel_rows[r] : r
+void launch_rmsnorm(cudaStream_t st, const float* x, const bf16* gain, bf16* h, int rows, int d, float eps,
+                    const int* sel_rows);
+// last row of every sequence (prefill's LM-head rows)
+void launch_select_last_rows(cudaStream_t st, const RowMeta& rm, int n_seqs, int* sel_rows);
+void launch_rope_kvwrite(cudaStream_t st, const float* qkv, const RowMeta& rm, const KvView& kv, const ModelDims& md,
+                         int layer, bf16* q, int T, const int* status);
+void launch_attn_simt(cudaStream_t st, const bf16* q, const RowMeta& rm, const KvView& kv, const ModelDims& md,
+                      int layer, bf16* out, int T, const int* status);
+struct AcceptArgs {
+  int n_seqs, max_q_len;
+  float log_tau;
+  const unsigned long long* row_best;
+  const float* zdraft;
+  int* accept_len;
+  int* emit_tokens;
+  int* n_emit;
+  int* row_argmax;     // optional outputs
+  float* row_zmax;
+  float* row_zdraft;
+};
+void launch_accept(cudaStream_t st, const AcceptArgs& a, const RowMeta& rm, const int* status);
+void launch_first_token(cudaStream_t st, const unsigned long long* row_best, int n_seqs, int* first_token,
+                        const RowMeta& rm, const KvView& kv, const int* status);
+void launch_commit(cudaStream_t st, const KvView& kv, int n_seqs, const int* seq_slots, const int* accept_len,
+                   int* blocks_in_use);
+void launch_clear_best(cudaStream_t st, unsigned long long* row_best, float* zdraft, int rows);
+
+// ---- plain SIMT GEMM (hsd_gemm_simt.cu): the debug cross-check and hsd_debug_logits --------------
+enum GemmMode { GM_STORE_BF16 = 0, GM_ADD_F32 = 1, GM_SWIGLU = 2, GM_STORE_F32 = 3, GM_ARGMAX = 4 };
+struct GemmOut {
+  void* C;                         // bf16 / fp32 output (modes 0-3), leading dimension ldc
+  int ldc;
+  unsigned long long* row_best;    // mode 4
+  float* zdraft;                   // mode 4
+  const int* row_next;             // mode 4 (nullptr = no draft-token capture)
+};
+void launch_gemm_simt(cudaStream_t st, const bf16* A, const bf16* W, int M, int n_out, int K, int mode,
+                      const GemmOut& out);
+
+// ---- tcgen05 GEMM (hsd_gemm_sm100.cu) ------------------------------------------------------------
+struct TmaFns;   // driver entry points
+// Encode a 2-D bf16 row-major [rows, cols] tensor map with a {64, box_rows} box and 128-byte swizzle.
+int make_tmap_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+int make_tmap_3d(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t stride1_bytes,
+                 uint64_t stride2_bytes, uint32_t b0, uint32_t b1, uint32_t b2);
+int tma_init();   // resolves cuTensorMapEncodeTiled; 0 on success
+
+struct QkvEpilogue {      // fused RoPE + paged KV write (QKV projection)
+  const int* row_kv;
+  const float2* rope_cs;
+  bf16* q_out;            // [T, Hq*64]
+  bf16* k_pool_layer;     // layer base of the K pool
+  bf16* v_pool_layer;
+  int Hq, Hkv;
+};
+struct GemmSm100Args {
+  CUtensorMap tmA, tmB;
+  int M, n_out, K, mode;
+  GemmOut out;
+  QkvEpilogue qkv;
+  int* status;
+  int n_sms;
+};
+enum GemmSm100Mode { GS_STORE_BF16 = 0, GS_ADD_F32 = 1, GS_SWIGLU = 2, GS_ARGMAX = 4, GS_QKV_ROPE = 5 };
+int launch_gemm_sm100(cudaStream_t st, const GemmSm100Args& a);
+int gemm_sm100_box_rows(int mode, int n_out, int M, int n_sms);   // B-operand TMA box height for this problem
+
+}  // namespace hsd

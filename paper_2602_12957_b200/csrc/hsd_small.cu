@@ -1,0 +1,390 @@
+// Memory- and latency-bound kernels of the verify step: row metadata + checks, embedding gather,
+// RMSNorm, RoPE + paged KV write, the plain SIMT attention (debug cross-check), accept/emit, KV commit.
+#include "hsd_kernels.h"
+
+namespace hsd {
+
+const char* kernel_class_name(int kc) {
+  static const char* names[KC_COUNT] = {"setup_rows", "embed",     "rmsnorm",     "gemm_qkv",  "rope_kv_write",
+                                        "attention",  "attn_combine", "gemm_o",   "gemm_gate_up", "gemm_down",
+                                        "lm_head_argmax", "accept_emit", "kv_commit", "debug"};
+  return (kc >= 0 && kc < KC_COUNT) ? names[kc] : "?";
+}
+
+// ------------------------------------------------------------------------------------------------
+// Row metadata.  One CTA per sequence.  Validates what the host cannot see (device-resident lengths and
+// tables); any violation sets the status words, and every kernel that follows an indirection returns early.
+constexpr int kSetupRows = 64;   // rows of one sequence handled by one CTA
+__global__ void setup_rows_kernel(SetupArgs a, KvView kv, RowMeta rm, int* status, int* tile_count) {
+  const int i = blockIdx.x;
+  const int tid = threadIdx.x;
+  __shared__ int s_red[32];
+  __shared__ int s_bad;
+  if (tid == 0) s_bad = 0;
+  __syncthreads();
+
+  // every CTA scans cu_q once: monotone + total, and the exclusive scan of q-tiles before sequence i
+  int my_tiles = 0, bad = 0;
+  for (int s = tid; s < a.n_seqs; s += blockDim.x) {
+    const int n = a.cu_q[s + 1] - a.cu_q[s];
+    if (n < 0) bad = 1;
+    if (n > a.max_q_len) bad = 2;
+    if (s < i && n > 0) my_tiles += (n + a.tokens_per_tile - 1) / a.tokens_per_tile;
+  }
+  if (tid == 0 && (a.cu_q[0] != 0 || a.cu_q[a.n_seqs] != a.total_q)) bad = 1;
+  for (int o = 16; o; o >>= 1) my_tiles += __shfl_xor_sync(0xffffffffu, my_tiles, o);
+  if ((tid & 31) == 0) s_red[tid >> 5] = my_tiles;
+  if (bad) atomicMax(&s_bad, bad);
+  __syncthreads();
+  int tile0 = 0;
+  for (int w = 0; w < (blockDim.x >> 5); ++w) tile0 += s_red[w];
+  if (s_bad) {
+    if (tid == 0 && blockIdx.y == 0) dev_fail(status, s_bad == 2 ? DEV_TOO_LONG : DEV_CU_Q, i);
+    return;
+  }
+
+  const int q0 = a.cu_q[i];
+  const int n = a.cu_q[i + 1] - q0;
+  const int slot = a.seq_slots ? a.seq_slots[i] : a.slot_base + i;
+  if (slot < 0 || slot >= kv.n_slots) {
+    if (tid == 0) dev_fail(status, DEV_KV_CAPACITY, i);
+    return;
+  }
+  const int L = kv.seq_lens[slot];
+  if (L < 0 || (long long)L + n > (long long)kv.max_blocks * HSD_KV_BLOCK) {
+    if (tid == 0) dev_fail(status, DEV_KV_CAPACITY, i);
+    return;
+  }
+  if (tid == 0 && blockIdx.y == 0) {
+    rm.seq_q0[i] = q0;
+    rm.seq_n[i] = n;
+    rm.seq_len[i] = L;
+    rm.seq_slot[i] = slot;
+    rm.seq_tile0[i] = tile0;
+    if (i == a.n_seqs - 1) {
+      const int t = tile0 + (n + a.tokens_per_tile - 1) / a.tokens_per_tile;
+      rm.seq_tile0[a.n_seqs] = t;
+      *tile_count = t;
+    }
+  }
+  const int j_lo = blockIdx.y * kSetupRows;
+  const int j_hi = min(n, j_lo + kSetupRows);
+  const int half = a.head_dim / 2;
+  for (int j = j_lo + tid; j < j_hi; j += blockDim.x) {
+    const int r = q0 + j;
+    int tok, nxt = -1;
+    if (a.tokens) {
+      tok = a.tokens[r];
+      if (j + 1 < n) nxt = a.tokens[r + 1];
+    } else {
+      tok = (j == 0) ? a.pending[0] : a.draft[j - 1];
+      if (j + 1 < n) nxt = a.draft[j];
+    }
+    if (tok >= a.vocab || (tok < 0 && !a.allow_embed_rows)) {
+      dev_fail(status, DEV_TOKEN_RANGE, r);
+      tok = 0;
+    }
+    if (tok < 0) tok = -1;
+    const int pos = L + j;
+    int phys = kv.block_table[(size_t)slot * kv.max_blocks + pos / HSD_KV_BLOCK];
+    if (phys < 0 || phys >= kv.n_blocks) {
+      dev_fail(status, DEV_BLOCK_RANGE, r);
+      phys = 0;
+    }
+    rm.row_seq[r] = i;
+    rm.row_pos[r] = pos;
+    rm.row_tok[r] = tok;
+    rm.row_kv[r] = phys * HSD_KV_BLOCK + pos % HSD_KV_BLOCK;
+    rm.row_next[r] = a.allow_embed_rows ? -1 : nxt;
+  }
+  // rotary table: (cos, sin) of pos * base^(-2i/D), angle formed in double so long contexts keep accuracy
+  for (int e = j_lo * half + tid; e < j_hi * half; e += blockDim.x) {
+    const int j = e / half, f = e % half;
+    const double inv = exp2(-(double)(2 * f) / (double)a.head_dim * log2((double)a.rope_base));
+    double sn, cs;
+    sincos((double)(L + j) * inv, &sn, &cs);
+    rm.rope_cs[(size_t)(q0 + j) * half + f] = make_float2((float)cs, (float)sn);
+  }
+}
+
+void launch_setup_rows(cudaStream_t st, const SetupArgs& a, const KvView& kv, const RowMeta& rm, int* status,
+                       int* tile_count) {
+  dim3 grid(a.n_seqs, (a.max_q_len + kSetupRows - 1) / kSetupRows);
+  setup_rows_kernel<<<grid, 256, 0, st>>>(a, kv, rm, status, tile_count);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Embedding gather: x[r] = fp32(table[tok]) or fp32(embeds[r]).  One warp per row, 16-byte loads.
+__global__ void embed_kernel(RowMeta rm, const bf16* __restrict__ table, const bf16* __restrict__ embeds,
+                             float* __restrict__ x, int T, int d, const int* status) {
+  if (*status) return;
+  const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (r >= T) return;
+  const int lane = threadIdx.x & 31;
+  const int tok = rm.row_tok[r];
+  const bf16* src = tok >= 0 ? table + (size_t)tok * d : embeds + (size_t)r * d;
+  float* dst = x + (size_t)r * d;
+  for (int c = lane * 8; c < d; c += 256) {
+    uint4 v = *reinterpret_cast<const uint4*>(src + c);
+    float4 lo = make_float4(bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y));
+    float4 hi = make_float4(bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w));
+    *reinterpret_cast<float4*>(dst + c) = lo;
+    *reinterpret_cast<float4*>(dst + c + 4) = hi;
+  }
+}
+void launch_embed(cudaStream_t st, const RowMeta& rm, const bf16* table, const bf16* embeds, float* x, int T, int d,
+                  const int* status) {
+  embed_kernel<<<(T + 7) / 8, 256, 0, st>>>(rm, table, embeds, x, T, d, status);
+}
+
+// ------------------------------------------------------------------------------------------------
+// RMSNorm: h = bf16(x * rsqrt(mean(x^2) + eps) * gain).  One warp per row; the row stays in registers
+// between the reduction and the scaling (d <= 2048), so x is read once.
+template <int VEC>   // VEC float4 per lane: d = 128 * VEC
+__global__ void rmsnorm_kernel(const float* __restrict__ x, const bf16* __restrict__ gain, bf16* __restrict__ h,
+                               int rows, int d, float eps, const int* __restrict__ sel_rows) {
+  const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (r >= rows) return;
+  const int lane = threadIdx.x & 31;
+  const int src = sel_rows ? sel_rows[r] : r;
+  const float4* xp = reinterpret_cast<const float4*>(x + (size_t)src * d);
+  float4 v[VEC];
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < VEC; ++i) {
+    v[i] = xp[lane + 32 * i];
+    ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
+  }
+  for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  const float rs = rsqrtf(ss / (float)d + eps);
+  const uint2* gp = reinterpret_cast<const uint2*>(gain);
+  uint2* hp = reinterpret_cast<uint2*>(h + (size_t)r * d);
+#pragma unroll
+  for (int i = 0; i < VEC; ++i) {
+    uint2 g = gp[lane + 32 * i];
+    uint2 o;
+    o.x = pack_bf16(v[i].x * rs * bf16_lo(g.x), v[i].y * rs * bf16_hi(g.x));
+    o.y = pack_bf16(v[i].z * rs * bf16_lo(g.y), v[i].w * rs * bf16_hi(g.y));
+    hp[lane + 32 * i] = o;
+  }
+}
+void launch_rmsnorm(cudaStream_t st, const float* x, const bf16* gain, bf16* h, int rows, int d, float eps,
+                    const int* sel_rows) {
+  if (rows <= 0) return;
+  dim3 grid((rows + 7) / 8), block(256);
+  switch (d / 128) {
+    case 1: rmsnorm_kernel<1><<<grid, block, 0, st>>>(x, gain, h, rows, d, eps, sel_rows); break;
+    case 2: rmsnorm_kernel<2><<<grid, block, 0, st>>>(x, gain, h, rows, d, eps, sel_rows); break;
+    case 4: rmsnorm_kernel<4><<<grid, block, 0, st>>>(x, gain, h, rows, d, eps, sel_rows); break;
+    case 8: rmsnorm_kernel<8><<<grid, block, 0, st>>>(x, gain, h, rows, d, eps, sel_rows); break;
+    case 16: rmsnorm_kernel<16><<<grid, block, 0, st>>>(x, gain, h, rows, d, eps, sel_rows); break;
+    default: break;   // hsd_create rejects other widths
+  }
+}
+
+__global__ void select_last_rows_kernel(RowMeta rm, int n_seqs, int* sel_rows) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n_seqs) sel_rows[i] = rm.seq_q0[i] + max(rm.seq_n[i], 1) - 1;
+}
+void launch_select_last_rows(cudaStream_t st, const RowMeta& rm, int n_seqs, int* sel_rows) {
+  select_last_rows_kernel<<<(n_seqs + 127) / 128, 128, 0, st>>>(rm, n_seqs, sel_rows);
+}
+
+__global__ void clear_best_kernel(unsigned long long* row_best, float* zdraft, int rows) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < rows) {
+    row_best[i] = 0ull;
+    zdraft[i] = __int_as_float(0x7fc00000);
+  }
+}
+void launch_clear_best(cudaStream_t st, unsigned long long* row_best, float* zdraft, int rows) {
+  clear_best_kernel<<<(rows + 255) / 256, 256, 0, st>>>(row_best, zdraft, rows);
+}
+
+// ------------------------------------------------------------------------------------------------
+// RoPE + paged KV write from an fp32 qkv row (SIMT path; the tensor-core path fuses this into the
+// QKV projection's epilogue).  One warp per (row, head); lane i holds dims i and i + 32.
+__global__ void rope_kvwrite_kernel(const float* __restrict__ qkv, RowMeta rm, KvView kv, ModelDims md, int layer,
+                                    bf16* __restrict__ q, int T, const int* status) {
+  if (*status) return;
+  const int heads = md.Hq + 2 * md.Hkv;
+  const int w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (w >= T * heads) return;
+  const int r = w / heads, hd = w % heads, lane = threadIdx.x & 31;
+  const float* src = qkv + (size_t)r * md.qkv_out + hd * 64;
+  float a = src[lane], b = src[lane + 32];
+  const int phys = rm.row_kv[r];
+  const size_t blk_base = ((size_t)layer * kv.n_blocks + phys / 64) * md.Hkv;
+  const int off = phys % 64;
+  if (hd < md.Hq + md.Hkv) {
+    const float2 cs = rm.rope_cs[(size_t)r * 32 + lane];
+    const float ra = a * cs.x - b * cs.y, rb = b * cs.x + a * cs.y;
+    if (hd < md.Hq) {
+      bf16* dst = q + (size_t)r * md.Hq * 64 + hd * 64;
+      dst[lane] = __float2bfloat16(ra);
+      dst[lane + 32] = __float2bfloat16(rb);
+    } else {
+      bf16* dst = kv.k_pool + ((blk_base + (hd - md.Hq)) * 64 + off) * 64;
+      dst[lane] = __float2bfloat16(ra);
+      dst[lane + 32] = __float2bfloat16(rb);
+    }
+  } else {
+    bf16* dst = kv.v_pool + (blk_base + (hd - md.Hq - md.Hkv)) * 4096;
+    dst[(size_t)lane * 64 + off] = __float2bfloat16(a);
+    dst[(size_t)(lane + 32) * 64 + off] = __float2bfloat16(b);
+  }
+}
+void launch_rope_kvwrite(cudaStream_t st, const float* qkv, const RowMeta& rm, const KvView& kv, const ModelDims& md,
+                         int layer, bf16* q, int T, const int* status) {
+  const long long warps = (long long)T * (md.Hq + 2 * md.Hkv);
+  rope_kvwrite_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(qkv, rm, kv, md, layer, q, T, status);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Plain SIMT attention (debug cross-check): one warp per (row, q head), online softmax over 32-key chunks.
+__global__ void attn_simt_kernel(const bf16* __restrict__ q, RowMeta rm, KvView kv, ModelDims md, int layer,
+                                 bf16* __restrict__ out, int T, const int* status) {
+  if (*status) return;
+  const int w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (w >= T * md.Hq) return;
+  const int r = w / md.Hq, hq = w % md.Hq, lane = threadIdx.x & 31;
+  const int kvh = hq / md.group;
+  const int seq = rm.row_seq[r];
+  const int slot = rm.seq_slot[seq];
+  const int n_keys = rm.row_pos[r] + 1;            // keys at positions 0 .. pos (causal, own row included)
+  __shared__ float s_q[8][64];
+  float* qs = s_q[threadIdx.x >> 5];
+  const bf16* qp = q + (size_t)r * md.Hq * 64 + hq * 64;
+  qs[lane] = __bfloat162float(qp[lane]) * 0.125f;   // 1/sqrt(64)
+  qs[lane + 32] = __bfloat162float(qp[lane + 32]) * 0.125f;
+  __syncwarp();
+  float m = -INFINITY, l = 0.f, o0 = 0.f, o1 = 0.f;
+  const int* bt = kv.block_table + (size_t)slot * kv.max_blocks;
+  for (int k0 = 0; k0 < n_keys; k0 += 32) {
+    const int key = k0 + lane;
+    const int phys = bt[k0 / 64];                   // a 32-key chunk never straddles a 64-token block
+    const size_t tile = ((size_t)layer * kv.n_blocks + phys) * md.Hkv + kvh;
+    float s = -INFINITY;
+    if (key < n_keys) {
+      const uint4* kp = reinterpret_cast<const uint4*>(kv.k_pool + (tile * 64 + key % 64) * 64);
+      float acc = 0.f;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        uint4 v = kp[c];
+        const float* qq = qs + c * 8;
+        acc += qq[0] * bf16_lo(v.x) + qq[1] * bf16_hi(v.x) + qq[2] * bf16_lo(v.y) + qq[3] * bf16_hi(v.y) +
+               qq[4] * bf16_lo(v.z) + qq[5] * bf16_hi(v.z) + qq[6] * bf16_lo(v.w) + qq[7] * bf16_hi(v.w);
+      }
+      s = acc;
+    }
+    float cm = s;
+    for (int o = 16; o; o >>= 1) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, o));
+    const float m_new = fmaxf(m, cm);
+    const float p = (key < n_keys) ? __expf(s - m_new) : 0.f;
+    float ps = p;
+    for (int o = 16; o; o >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, o);
+    const float scale = __expf(m - m_new);
+    l = l * scale + ps;
+    o0 *= scale;
+    o1 *= scale;
+    m = m_new;
+    // V^T tile [dim][tok]: lane owns dims lane and lane + 32
+    const bf16* vt = kv.v_pool + tile * 4096;
+    const int tok0 = k0 % 64;
+    const int cnt = min(32, n_keys - k0);
+    for (int t = 0; t < cnt; ++t) {
+      const float pt = __shfl_sync(0xffffffffu, p, t);
+      o0 += pt * __bfloat162float(vt[(size_t)lane * 64 + tok0 + t]);
+      o1 += pt * __bfloat162float(vt[(size_t)(lane + 32) * 64 + tok0 + t]);
+    }
+  }
+  bf16* op = out + (size_t)r * md.Hq * 64 + hq * 64;
+  op[lane] = __float2bfloat16(o0 / l);
+  op[lane + 32] = __float2bfloat16(o1 / l);
+}
+void launch_attn_simt(cudaStream_t st, const bf16* q, const RowMeta& rm, const KvView& kv, const ModelDims& md,
+                      int layer, bf16* out, int T, const int* status) {
+  const long long warps = (long long)T * md.Hq;
+  attn_simt_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(q, rm, kv, md, layer, out, T, status);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Draft compare + longest-prefix accept + emit.  One warp per sequence.
+// Row j (0-based) of a sequence holds the distribution after [.., pending, d_1..d_j]; its next draft token is
+// d_{j+1}.  a = first j < k whose test fails (or k).  Exact mode: argmax == d_{j+1}.  Threshold mode:
+// z[d_{j+1}] - z_max >= log_tau.
+__global__ void accept_kernel(AcceptArgs a, RowMeta rm, const int* status) {
+  if (*status) return;
+  const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (i >= a.n_seqs) return;
+  const int lane = threadIdx.x & 31;
+  const int q0 = rm.seq_q0[i], n = rm.seq_n[i];
+  if (n <= 0) {
+    if (lane == 0) { a.accept_len[i] = 0; a.n_emit[i] = 0; }
+    return;
+  }
+  const int k = n - 1;
+  int acc = k;
+  for (int j0 = 0; j0 < k && acc == k; j0 += 32) {
+    const int j = j0 + lane;
+    bool ok = true;
+    if (j < k) {
+      const unsigned long long best = a.row_best[q0 + j];
+      const int nxt = rm.row_next[q0 + j];
+      if (a.log_tau == 0.f) ok = (key_col(best) == nxt);
+      else ok = (a.zdraft[q0 + j] - key_value(best) >= a.log_tau);
+    }
+    const unsigned fail = __ballot_sync(0xffffffffu, !ok);
+    if (fail) acc = j0 + __ffs(fail) - 1;
+  }
+  int* emit = a.emit_tokens + (size_t)i * a.max_q_len;
+  for (int j = lane; j < acc; j += 32) emit[j] = rm.row_next[q0 + j];
+  if (lane == 0) {
+    emit[acc] = key_col(a.row_best[q0 + acc]);
+    a.accept_len[i] = acc;
+    a.n_emit[i] = acc + 1;
+  }
+  for (int j = lane; j < n; j += 32) {
+    const unsigned long long best = a.row_best[q0 + j];
+    if (a.row_argmax) a.row_argmax[q0 + j] = key_col(best);
+    if (a.row_zmax) a.row_zmax[q0 + j] = key_value(best);
+    if (a.row_zdraft) a.row_zdraft[q0 + j] = a.zdraft[q0 + j];
+  }
+}
+void launch_accept(cudaStream_t st, const AcceptArgs& a, const RowMeta& rm, const int* status) {
+  accept_kernel<<<(a.n_seqs + 3) / 4, 128, 0, st>>>(a, rm, status);
+}
+
+// Prefill epilogue: first pending token per sequence, and seq_lens += rows.
+__global__ void first_token_kernel(const unsigned long long* row_best, int n_seqs, int* first_token, RowMeta rm,
+                                   KvView kv, const int* status) {
+  if (*status) return;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_seqs) return;
+  first_token[i] = key_col(row_best[i]);
+  kv.seq_lens[rm.seq_slot[i]] = rm.seq_len[i] + rm.seq_n[i];
+}
+void launch_first_token(cudaStream_t st, const unsigned long long* row_best, int n_seqs, int* first_token,
+                        const RowMeta& rm, const KvView& kv, const int* status) {
+  first_token_kernel<<<(n_seqs + 127) / 128, 128, 0, st>>>(row_best, n_seqs, first_token, rm, kv, status);
+}
+
+// ------------------------------------------------------------------------------------------------
+// KV commit / rollback: the pending row and the accepted rows stay, the rest is dead and gets overwritten.
+__global__ void commit_kernel(KvView kv, int n_seqs, const int* seq_slots, const int* accept_len, int* blocks_in_use) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_seqs) return;
+  const int slot = seq_slots ? seq_slots[i] : i;
+  if (slot < 0 || slot >= kv.n_slots) return;
+  const int a = accept_len[i];
+  int L = kv.seq_lens[slot];
+  if (a >= 0) L = min(L + a + 1, kv.max_blocks * HSD_KV_BLOCK);
+  kv.seq_lens[slot] = L;
+  if (blocks_in_use) blocks_in_use[i] = (L + HSD_KV_BLOCK - 1) / HSD_KV_BLOCK;
+}
+void launch_commit(cudaStream_t st, const KvView& kv, int n_seqs, const int* seq_slots, const int* accept_len,
+                   int* blocks_in_use) {
+  commit_kernel<<<(n_seqs + 127) / 128, 128, 0, st>>>(kv, n_seqs, seq_slots, accept_len, blocks_in_use);
+}
+
+}  // namespace hsd

@@ -1,0 +1,68 @@
+"""GPU parity of the GEMM operator (all epilogues that store a matrix) against a float64 product of the
+same bf16 inputs."""
+import numpy as np
+import pytest
+
+from paper_2602_12957_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def models():
+    import torch
+    from paper_2602_12957_b200 import runtime as R
+    cfg = I.TINY
+    w = I.make_weights(cfg, 1)
+    return {0: R.DeviceModel(cfg, w, 0), 1: R.DeviceModel(cfg, w, 1)}
+
+
+def _run(model, M, N, K, mode, seed):
+    import torch
+    from paper_2602_12957_b200 import binding as B
+    rng = np.random.default_rng(seed)
+    A = I.bf16_round(rng.standard_normal((M, K), dtype=np.float32))
+    W = I.bf16_round(rng.standard_normal((N, K), dtype=np.float32) * 0.05)
+    dev = model.device
+    tA = torch.from_numpy(A).to(dev, torch.bfloat16)
+    tW = torch.from_numpy(W).to(dev, torch.bfloat16)
+    ref = A.astype(np.float64) @ W.astype(np.float64).T
+    st = torch.cuda.current_stream().cuda_stream
+    if mode == 0:
+        C = torch.full((M, N), 7.0, dtype=torch.bfloat16, device=dev)
+        B.check(B.hsd_op_linear(model.ctx, tA, tW, C, M, N, K, 0, st))
+        got = C.float().cpu().numpy().astype(np.float64)
+    elif mode == 1:
+        base = rng.standard_normal((M, N), dtype=np.float32)
+        C = torch.from_numpy(base.copy()).to(dev)
+        B.check(B.hsd_op_linear(model.ctx, tA, tW, C, M, N, K, 1, st))
+        got = C.cpu().numpy().astype(np.float64)
+        ref = ref + base
+    else:
+        C = torch.full((M, N // 2), 7.0, dtype=torch.bfloat16, device=dev)
+        B.check(B.hsd_op_linear(model.ctx, tA, tW, C, M, N, K, 2, st))
+        got = C.float().cpu().numpy().astype(np.float64)
+        g, u = ref[:, :N // 2], ref[:, N // 2:]
+        ref = g / (1.0 + np.exp(-g)) * u
+    torch.cuda.synchronize()
+    return got, ref
+
+
+SHAPES = [(1040, 2048, 1024), (70, 256, 256), (128, 64, 64), (1, 1024, 4096), (513, 8192, 1024), (300, 1024, 4096)]
+
+
+@pytest.mark.parametrize("flags", [1, 0], ids=["simt", "tensor"])
+@pytest.mark.parametrize("mode", [0, 1, 2])
+@pytest.mark.parametrize("shape", SHAPES)
+def test_linear_matches_float64_product(models, flags, mode, shape):
+    M, N, K = shape
+    if mode == 2 and N % 128:
+        pytest.skip("SwiGLU needs an even split into 64-column halves")
+    got, ref = _run(models[flags], M, N, K, mode, seed=M + N + K + mode)
+    scale = np.abs(ref).max()
+    if mode == 1:
+        tol = 1e-4 * scale            # fp32 output: only accumulation order differs
+    else:
+        tol = 2.0 ** -8 * scale + 1e-3   # one bf16 rounding of the stored result
+    err = np.abs(got - ref).max()
+    assert err <= tol, f"shape {shape} mode {mode}: max err {err:.3e} > {tol:.3e}"
