@@ -12,8 +12,8 @@ using namespace hsd;
 
 namespace hsd {
 int launch_attn_sm100(cudaStream_t st, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
-                      const RowMeta& rm, const KvView& kv, const ModelDims& md, int layer, bf16* out, int T,
-                      int max_tiles, const int* tile_count, int* status, float* split_ws, int n_sms);
+                      const RowMeta& rm, const KvView& kv, const ModelDims& md, int layer, bf16* out, int n_seqs,
+                      int max_tiles, const int* tile_count, int* status, float* split_ws);
 }
 
 struct ProfEvent {
@@ -271,8 +271,8 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         Scope s(c, st, KC_ATTN);
         if (c->attn_simt) {
           launch_attn_simt(st, w.q, w.rm, kv, md, l, w.attn, T, w.status);
-        } else if (launch_attn_sm100(st, tm_q, tm_k, tm_v, w.rm, kv, md, l, w.attn, T, max_tiles, w.status + 4,
-                                     w.status, w.split_ws, c->n_sms)) {
+        } else if (launch_attn_sm100(st, tm_q, tm_k, tm_v, w.rm, kv, md, l, w.attn, a.n_seqs, max_tiles, w.status + 4,
+                                     w.status, w.split_ws)) {
           return fail_cuda(c);
         }
       }

@@ -112,13 +112,23 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait.  Every spin in these kernels has an iteration limit: when it runs out (or another thread
 // of the CTA has already given up) the wait records DEV_WAIT_TIMEOUT in the status words, raises the
 // CTA-wide abort flag and returns false; callers then fall through to the common teardown.
-constexpr uint32_t kWaitSpins = 1u << 22;
+constexpr uint32_t kWaitSpins = 1u << 24;
+constexpr unsigned long long kWaitNs = 2000000000ull;   // 2 s of wall clock
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
                                           int where) {
+  unsigned long long t0 = 0;
   for (uint32_t i = 0; i < kWaitSpins; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 63u) == 63u) {
       if (*abort_flag) return false;
+      const unsigned long long now = global_ns();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > kWaitNs) break;
       __nanosleep(64);
     }
   }

@@ -29,3 +29,14 @@ def test_tiny_config_matches_oracle(flags):
     assert stats["exact_rows"] + stats["near_tie_rows"] == 4 * 17
     assert stats["max_dz"] < H.LOGIT_TOL
     print("tiny", flags, stats)
+
+
+@pytest.mark.parametrize("flags", [2, 0], ids=["simt_attention", "tensor"])
+def test_small_decoder_regions_match_oracle(flags):
+    """Same layer shape as the 24-layer decoder (GQA 16/8, d 1024, FFN 4096), 2 layers, vocab 8192: several
+    q-tiles per sequence, ragged tails, prefixes that end inside a KV block."""
+    wl = I.region_workload(seed=77, n_regions=5, prefix_lo=70, prefix_hi=330, draft_mean=60, draft_lo=8, draft_hi=200,
+                           cfg=I.small_decoder(2, 8192), name="small_regions")
+    stats, orc, per, _ = run_region_parity(wl, flags)
+    print("small", flags, stats, [(len(o.draft), o.res.accept_len) for o in orc.values()])
+    assert stats["max_dz"] < H.LOGIT_TOL
