@@ -1,0 +1,399 @@
+#!/usr/bin/env python
+"""Benchmark of the HSD draft-verification step on B200.
+
+    python bench.py --gpus N --steps K --warmup W            # this library (one process per GPU)
+    python bench.py --impl reference --steps K --warmup W    # the CPU oracle, as it stands, on host cores
+
+One step = one pass of the whole hot path over one batch: pack/embed, 24 x (norm, QKV+RoPE+KV write, paged
+causal attention, O, norm, gate/up+SwiGLU, down), final norm, LM head + argmax + draft logit, accept/emit,
+KV commit.  Workload (default): the region-level stage — 16 regions per GPU, prefixes 256-1024 visual rows,
+lognormal draft lengths (mean 64, clipped 8-256), planted agreement with mean acceptance 0.8, paged KV with
+64-token blocks and shuffled physical blocks.  Inputs are synthetic and seeded; weights are random-init.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2602_12957_b200 import inputs as I          # noqa: E402
+from paper_2602_12957_b200 import roofline as RF       # noqa: E402
+
+METRIC = "draft tokens verified per second (verify step: forward over paged prefix + accept + KV commit)"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM traffic per launch of the dominant kernel classes, from the ncu captures summarised under profiles/
+# (dram__bytes_read.sum + dram__bytes_write.sum); None where no capture exists yet.
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"])}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+# ------------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,utilization.gpu,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.tmp.flush()
+        rows = []
+        for line in open(self.tmp.name):
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                rows.append((float(parts[0]), float(parts[1]), float(parts[2]), float(parts[3]), parts[4:8]))
+            except ValueError:
+                continue
+        os.unlink(self.tmp.name)
+        load = [r for r in rows if r[3] >= 50.0] or rows
+        reasons = set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in load:
+            for n, v in zip(names, r[4]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median([r[0] for r in load])) if load else None,
+                "sm_max_mhz": load[0][1] if load else None,
+                "power_w_max": max([r[2] for r in load]) if load else None,
+                "reasons": sorted(reasons), "samples": len(load)}
+
+
+# ------------------------------------------------------------------------------------------------ workload
+def build_gpu_state(args, rank):
+    import torch
+    from paper_2602_12957_b200 import runtime as R
+    cfg = I.DECODER
+    wl = I.region_workload(seed=I.BASE_SEED + 1 + 1000 * rank, cfg=cfg)
+    weights = I.make_weights(cfg, I.BASE_SEED + 1)
+    model = R.DeviceModel(cfg, weights, 0, f"cuda:{torch.cuda.current_device()}")
+    del weights
+    seqs = wl.seqs
+    S = len(seqs)
+    kv = R.KvCache(model, [s.prefix_len + s.draft_len + 2 for s in seqs], seed=wl.seed)
+    ks = [s.draft_len for s in seqs]
+    total_q = sum(ks) + S
+    total_prefix = sum(s.prefix_len for s in seqs)
+    eng = R.Engine(model, kv, max(total_prefix, total_q), S)
+    first = eng.prefill([s.prefix_embeds for s in seqs], [s.prefix_ids for s in seqs])
+    eng.check_device("prefill")
+    prefix_lens = kv.seq_lens.clone()
+
+    # greedy continuation by plain one-token steps (empty drafts), to plant the agreement lengths
+    need = 0 if args.random_drafts else max(min(s.agree_len + 1, s.draft_len) for s in seqs)
+    cu1 = eng._i32(np.arange(S + 1))
+    out1 = eng.alloc_outputs(S, 1, S)
+    pending = first.clone()
+    hist = []
+    for _ in range(need):
+        eng.verify_regions(pending, cu1, 1, S, out=out1)
+        eng.commit(out1["accept_len"])
+        pending = out1["emit_tokens"][:, 0].clone()
+        hist.append(pending)
+    eng.check_device("greedy continuation")
+    greedy = torch.stack(hist, 1).cpu().numpy() if hist else np.zeros((S, 0), np.int32)
+    kv.seq_lens.copy_(prefix_lens)
+    if args.random_drafts:      # profiling runs: kernel time does not depend on token values
+        drafts = [s.rand_tokens[:s.draft_len] for s in seqs]
+    else:
+        drafts = [I.plant_draft(greedy[i], s.draft_len, s.agree_len, s.rand_tokens, cfg.vocab, False)
+                  for i, s in enumerate(seqs)]
+    toks, cu = I.pack_queries(first.cpu().numpy(), drafts)
+    return dict(cfg=cfg, wl=wl, model=model, kv=kv, eng=eng, toks=toks, cu=cu, total_q=total_q, max_q=max(ks) + 1,
+                prefix_lens=prefix_lens, ks=ks, S=S, drafts=drafts)
+
+
+def kernel_work_table(cfg, work: RF.StepWork, T: int):
+    """Algorithmic (flops, bytes) per launch of each kernel class."""
+    d, f, V = cfg.d_model, cfg.d_ffn, cfg.vocab
+    L = cfg.n_layers
+    t = {}
+    t["gemm_qkv"] = RF.gemm_work(T, cfg.qkv_out, d)
+    t["gemm_o"] = RF.gemm_work(T, d, cfg.n_heads * cfg.head_dim, 8.0)          # fp32 read-modify-write
+    t["gemm_gate_up"] = (2.0 * T * 2 * f * d, 2.0 * (T * d + 2 * f * d) + 2.0 * T * f)
+    t["gemm_down"] = RF.gemm_work(T, d, f, 8.0)
+    t["lm_head_argmax"] = (2.0 * T * V * d, 2.0 * (T * d + V * d) + 12.0 * T)
+    t["attention"] = (work.attn_flops / L, work.kv_read_bytes / L + 4.0 * T * cfg.n_heads * cfg.head_dim)
+    t["rmsnorm"] = (0.0, 6.0 * T * d)
+    return t
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2602_12957_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    st = build_gpu_state(args, rank)
+    eng, kv, cfg = st["eng"], st["kv"], st["cfg"]
+    dev = eng.dev
+    S, T, max_q = st["S"], st["total_q"], st["max_q"]
+    d_toks, d_cu = eng._i32(st["toks"]), eng._i32(st["cu"])
+    out = eng.alloc_outputs(S, max_q, T)
+    stream = torch.cuda.Stream(device=dev)
+
+    def step():
+        eng.verify_regions(d_toks, d_cu, max_q, T, out=out)
+        eng.commit(out["accept_len"])
+        kv.seq_lens.copy_(st["prefix_lens"])          # rewind so every timed step sees the same state
+
+    launches0 = B.hsd_launch_count(eng.model.ctx)
+    with torch.cuda.stream(stream):
+        for _ in range(max(3, args.warmup)):
+            step()
+        stream.synchronize()
+        eng.check_device("warmup")
+        launches_per_step = (B.hsd_launch_count(eng.model.ctx) - launches0) // max(3, args.warmup)
+        graph = None
+        if not args.no_graph:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                step()
+            for _ in range(3):
+                graph.replay()
+            stream.synchronize()
+    run = (lambda: graph.replay()) if graph is not None else step
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    uuid = str(torch.cuda.get_device_properties(dev).uuid)
+    uuid = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+    sampler = ClockSampler(uuid)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        barrier()
+        e0.record(stream)
+        for _ in range(args.steps):
+            run()
+        e1.record(stream)
+        barrier()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    clocks["sampled"] = "timed region"
+    if clocks["samples"] < 3:        # a short timed region leaves nvidia-smi nothing to sample: replay longer
+        sampler = ClockSampler(uuid)
+        with torch.cuda.stream(stream):
+            t_end = time.time() + 1.5
+            while time.time() < t_end:
+                for _ in range(20):
+                    run()
+                stream.synchronize()
+        clocks = sampler.stop()
+        clocks["sampled"] = "1.5 s replay of the same step after the timed region"
+    if world > 1:
+        tt = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total = float(tt.item())
+    ms_step = ms_total / args.steps
+    draft_tokens = sum(st["ks"])
+    value = draft_tokens * world / (ms_step * 1e-3)
+
+    # ---- end to end through the C-ABI with host buffers (pinned): H2D inputs, verify + commit, D2H results
+    h_toks = torch.from_numpy(st["toks"]).pin_memory()
+    h_cu = torch.from_numpy(st["cu"]).pin_memory()
+    h_acc = torch.empty(S, dtype=torch.int32).pin_memory()
+    h_nem = torch.empty(S, dtype=torch.int32).pin_memory()
+    h_emit = torch.empty(S, max_q, dtype=torch.int32).pin_memory()
+    e2e_steps = max(3, min(args.steps, 200))
+    with torch.cuda.stream(stream):
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            d_toks.copy_(h_toks, non_blocking=True)
+            d_cu.copy_(h_cu, non_blocking=True)
+            run()
+            h_acc.copy_(out["accept_len"], non_blocking=True)
+            h_nem.copy_(out["n_emit"], non_blocking=True)
+            h_emit.copy_(out["emit_tokens"], non_blocking=True)
+            stream.synchronize()
+        t1 = time.perf_counter()
+        barrier()
+    e2e_ms = (t1 - t0) * 1e3 / e2e_steps
+    if world > 1:
+        tt = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tt.item())
+    e2e = {"value": draft_tokens * world / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+           "h2d_bytes_per_step": int(h_toks.numel() * 4 + h_cu.numel() * 4),
+           "d2h_bytes_per_step": int((h_acc.numel() + h_nem.numel() + h_emit.numel()) * 4)}
+    accept_mean = float(np.mean([a / k for a, k in zip(h_acc.numpy().tolist(), st["ks"])]))
+
+    # ---- per-kernel durations (CUDA events around every launch, eager) for the roofline of the top kernel
+    peaks, peak_src = load_peaks()
+    prof_steps = max(3, min(args.steps, 30))
+    with torch.cuda.stream(stream):
+        B.hsd_profile_enable(eng.model.ctx, 1)
+        for _ in range(prof_steps):
+            step()
+        stream.synchronize()
+        _, prof = B.hsd_profile_read(eng.model.ctx)
+        B.hsd_profile_enable(eng.model.ctx, 0)
+    ctx_lens = [s.prefix_len for s in st["wl"].seqs]
+    work = RF.step_work(cfg, ctx_lens, [k + 1 for k in st["ks"]])
+    table = kernel_work_table(cfg, work, T)
+    tot_ms = sum(v[0] for v in prof.values()) or 1.0
+    kernels = {k: {"ms_per_step": v[0] / prof_steps, "launches_per_step": v[1] / prof_steps,
+                   "share": v[0] / tot_ms} for k, v in prof.items()}
+    top = max((k for k in prof if k in table), key=lambda k: prof[k][0])
+    flops, nbytes = table[top]
+    dur = prof[top][0] * 1e-3 / prof[top][1]
+    bw = peaks["hbm_gbs"] * 1e9
+    pk = peaks["bf16_tflops_sustained"] * 1e12
+    if flops / pk >= nbytes / bw:
+        roof = {"kernel": top, "bound": "tensor", "achieved": flops / dur / 1e12, "peak": peaks["bf16_tflops_sustained"],
+                "unit": "TFLOP/s", "peak_burst": peaks["bf16_tflops"]}
+    else:
+        roof = {"kernel": top, "bound": "hbm", "achieved": nbytes / dur / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get(top)
+    roof["peak_source"] = f"{peak_src} (sustained bf16 figure: kernel timed inside a long step)"
+    roof["us_per_launch"] = dur * 1e6
+    t_roof = RF.roofline_time(work.bytes, work.flops, bw, pk)
+    step_roof = {"roofline_us": t_roof * 1e6, "frac": t_roof / (ms_step * 1e-3), "bytes": work.bytes, "flops": work.flops,
+                 "bound": "tensor" if work.flops / pk > work.bytes / bw else "hbm"}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline_sample(st["wl"], budget_s=20.0)
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": "region-level stage: 24-layer decoder d1024 16q/8kv x64 ffn4096 vocab32768, "
+                                       "16 regions per GPU, prefix 256-1024, lognormal drafts mean 64 (8-256), "
+                                       "acceptance 0.8, paged KV block 64",
+                           "regions_per_gpu": S, "query_rows_per_gpu": T, "draft_tokens_per_gpu": draft_tokens,
+                           "context_tokens_per_gpu": int(sum(ctx_lens)), "mean_acceptance_rate": accept_mean,
+                           "planted_acceptance_rate": float(np.mean([s.agree_len / s.draft_len for s in st["wl"].seqs])),
+                           "l2_policy": "inputs larger than L2: 822 MB of weights are streamed every step",
+                           "launch": "CUDA graph replay" if graph is not None else "eager",
+                           "sharding": "regions sharded across ranks, no data-path collective"},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches_per_step * args.steps),
+                "gpu_launches_per_step": int(launches_per_step), "roofline": roof, "step_roofline": step_roof,
+                "kernels": kernels, "cpu_baseline": cpu}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------------ oracle arm
+def cpu_baseline_sample(wl, budget_s=20.0, steps=1, warmup=0):
+    """Times the oracle (float32, as it stands) on the two shortest regions of the workload: prefix K/V is
+    built first (untimed), then one verify step per region is timed."""
+    from oracle import hsd_oracle as O
+    weights = I.make_weights(wl.cfg, I.BASE_SEED + 1)
+    model = O.Decoder(wl.cfg, weights, np.float32)
+    order = sorted(range(len(wl.seqs)), key=lambda i: wl.seqs[i].prefix_len + wl.seqs[i].draft_len)[:2]
+    caches, pend, drafts = [], [], []
+    for i in order:
+        s = wl.seqs[i]
+        c = O.CachedSequence(model)
+        p = c.prefill(s.prefix_embeds, s.prefix_ids)
+        caches.append(c)
+        pend.append(p)
+        drafts.append(s.rand_tokens[:s.draft_len])        # timing does not depend on the token values
+    times = []
+    for it in range(warmup + steps):
+        t0 = time.perf_counter()
+        O.verify_regions(model, caches, pend, drafts)
+        dt = time.perf_counter() - t0
+        if it >= warmup:
+            times.append(dt)
+        if sum(times) > budget_s:
+            break
+    k = int(sum(len(d) for d in drafts))
+    t = float(np.mean(times))
+    return {"value": k / t, "unit": UNIT, "cores": host_cores(), "kind": "oracle",
+            "sample": f"regions {order} of the workload ({k} draft tokens, contexts "
+                      f"{[wl.seqs[i].prefix_len for i in order]}), float32 numpy oracle, prefix K/V prebuilt, "
+                      f"{len(times)} timed step(s)", "ms_per_step": t * 1e3}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = I.region_workload(seed=I.BASE_SEED + 1, cfg=I.DECODER)
+    r = cpu_baseline_sample(wl, budget_s=120.0, steps=max(1, args.steps), warmup=max(0, min(args.warmup, 1)))
+    line = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT,
+            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "region-level stage (bounded sample: the two shortest regions per step)"},
+            "cpu_baseline": {k: r[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--random-drafts", action="store_true",
+                    help="skip the greedy-continuation pass that plants agreement (for profiler captures)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
