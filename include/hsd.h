@@ -203,6 +203,17 @@ HSD_API int hsd_debug_buffer(hsd_ctx *ctx, const void *workspace, int total_q, i
 HSD_API int hsd_op_linear(hsd_ctx *ctx, const void *A, const void *W, void *C, int M, int n_out, int K, int mode,
                   void *cuda_stream);
 
+/* hsd_op_lm_head_argmax: the fused LM head on its own (Eq. 10 per row): for `rows` already-normalised hidden rows
+ * h (dev bf16 [rows, d_model]) compute z = h W_lm^T tile by tile and keep only, per row, the argmax (lowest id on
+ * ties), its logit, and the logit of next_tokens[row] (dev int32 [rows] or NULL; entries < 0 give NaN).  Logits
+ * are never written to memory.
+ *   scratch   dev, 8-byte aligned, at least rows * 8 bytes (the per-row running best), contents irrelevant
+ *   argmax    dev int32 [rows] out;  zmax dev fp32 [rows] out;  zdraft dev fp32 [rows] out (required with
+ *             next_tokens, else may be NULL)
+ * Errors: INVALID_ARG, WORKSPACE (scratch too small / misaligned), CUDA. */
+HSD_API int hsd_op_lm_head_argmax(hsd_ctx *ctx, const void *h, int rows, const int *next_tokens, void *scratch,
+                          size_t scratch_bytes, int *argmax, float *zmax, float *zdraft, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -25,6 +25,7 @@ EXPORTS = [
     "hsd_status_string", "hsd_create", "hsd_destroy", "hsd_workspace_bytes", "hsd_prefill", "hsd_verify_regions",
     "hsd_verify_page", "hsd_kv_commit", "hsd_device_status", "hsd_last_cuda_error", "hsd_launch_count",
     "hsd_profile_enable", "hsd_profile_read", "hsd_debug_logits", "hsd_debug_buffer", "hsd_op_linear",
+    "hsd_op_lm_head_argmax",
 ]
 
 
@@ -79,6 +80,7 @@ def _load():
     lib.hsd_debug_logits.argtypes = [vp, vp, i, i, vp, vp]
     lib.hsd_debug_buffer.argtypes = [vp, vp, i, i, C.c_char_p, C.POINTER(vp), C.POINTER(sz)]
     lib.hsd_op_linear.argtypes = [vp, vp, vp, vp, i, i, i, i, vp]
+    lib.hsd_op_lm_head_argmax.argtypes = [vp, vp, i, vp, vp, sz, vp, vp, vp, vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if name not in ("hsd_status_string", "hsd_workspace_bytes", "hsd_launch_count"):
@@ -223,3 +225,8 @@ def hsd_debug_buffer(ctx, workspace, total_q, n_seqs, name: str):
 
 def hsd_op_linear(ctx, A, W, Cout, M, n_out, K, mode, stream) -> int:
     return _lib.hsd_op_linear(ctx, _p(A), _p(W), _p(Cout), M, n_out, K, mode, _p(stream))
+
+
+def hsd_op_lm_head_argmax(ctx, h, rows, next_tokens, scratch, scratch_bytes, argmax, zmax, zdraft, stream) -> int:
+    return _lib.hsd_op_lm_head_argmax(ctx, _p(h), rows, _p(next_tokens), _p(scratch), scratch_bytes, _p(argmax),
+                                      _p(zmax), _p(zdraft), _p(stream))

@@ -672,6 +672,46 @@ int hsd_debug_buffer(hsd_ctx* c, const void* workspace, int total_q, int n_seqs,
   return HSD_OK;
 }
 
+// Shared body of the LM-head operator: rows of h -> per-row argmax / max logit / next-token logit, with
+// `best` (8 bytes per row) as the only scratch.
+static int lm_head_argmax_impl(hsd_ctx* c, const void* h, int rows, const int* next_tokens, unsigned long long* best,
+                               int* argmax, float* zmax, float* zdraft, cudaStream_t st) {
+  const ModelDims& md = c->md;
+  {
+    Scope s(c, st, KC_LMHEAD);
+    launch_clear_best(st, best, next_tokens ? zdraft : nullptr, rows);
+  }
+  {
+    Scope s(c, st, KC_LMHEAD);
+    GemmOut o = {nullptr, 0, best, zdraft, next_tokens};
+    if (c->simt) {
+      launch_gemm_simt(st, static_cast<const bf16*>(h), c->lm_head, rows, md.V, md.d, GM_ARGMAX, o);
+    } else {
+      GemmSm100Args g = {};
+      if (make_tmap_2d(&g.tmA, h, rows, md.d, 128)) return HSD_ERR_CUDA;
+      g.tmB = c->tm_lm_head;
+      g.M = rows; g.n_out = md.V; g.K = md.d; g.mode = GS_ARGMAX;
+      g.out = o;
+      g.status = nullptr; g.n_sms = c->n_sms;
+      if (launch_gemm_sm100(st, g)) return fail_cuda(c);
+    }
+  }
+  {
+    Scope s(c, st, KC_LMHEAD);
+    launch_unpack_best(st, best, rows, argmax, zmax);
+  }
+  return check_cuda(c);
+}
+
+int hsd_op_lm_head_argmax(hsd_ctx* c, const void* h, int rows, const int* next_tokens, void* scratch,
+                          size_t scratch_bytes, int* argmax, float* zmax, float* zdraft, void* cuda_stream) {
+  if (!c || !h || !scratch || !argmax || !zmax || rows <= 0) return HSD_ERR_INVALID_ARG;
+  if (next_tokens && !zdraft) return HSD_ERR_INVALID_ARG;
+  if (scratch_bytes < (size_t)rows * 8 || (reinterpret_cast<uintptr_t>(scratch) & 7)) return HSD_ERR_WORKSPACE;
+  return lm_head_argmax_impl(c, h, rows, next_tokens, static_cast<unsigned long long*>(scratch), argmax, zmax, zdraft,
+                             static_cast<cudaStream_t>(cuda_stream));
+}
+
 int hsd_op_linear(hsd_ctx* c, const void* A, const void* W, void* C, int M, int n_out, int K, int mode,
                   void* cuda_stream) {
   if (!c || !A || !W || !C || M <= 0 || n_out <= 0 || K <= 0) return HSD_ERR_INVALID_ARG;

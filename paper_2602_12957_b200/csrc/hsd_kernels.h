@@ -75,6 +75,7 @@ void launch_first_token(cudaStream_t st, const unsigned long long* row_best, int
 void launch_commit(cudaStream_t st, const KvView& kv, int n_seqs, const int* seq_slots, const int* accept_len,
                    int* blocks_in_use);
 void launch_clear_best(cudaStream_t st, unsigned long long* row_best, float* zdraft, int rows);
+void launch_unpack_best(cudaStream_t st, const unsigned long long* row_best, int rows, int* argmax, float* zmax);
 
 // ---- plain SIMT GEMM (hsd_gemm_simt.cu): the debug cross-check and hsd_debug_logits --------------
 enum GemmMode { GM_STORE_BF16 = 0, GM_ADD_F32 = 1, GM_SWIGLU = 2, GM_STORE_F32 = 3, GM_ARGMAX = 4 };

@@ -194,11 +194,23 @@ __global__ void clear_best_kernel(unsigned long long* row_best, float* zdraft, i
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < rows) {
     row_best[i] = 0ull;
-    zdraft[i] = __int_as_float(0x7fc00000);
+    if (zdraft) zdraft[i] = __int_as_float(0x7fc00000);
   }
 }
 void launch_clear_best(cudaStream_t st, unsigned long long* row_best, float* zdraft, int rows) {
   clear_best_kernel<<<(rows + 255) / 256, 256, 0, st>>>(row_best, zdraft, rows);
+}
+
+__global__ void unpack_best_kernel(const unsigned long long* row_best, int rows, int* argmax, float* zmax) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < rows) {
+    const unsigned long long b = row_best[i];
+    if (argmax) argmax[i] = key_col(b);
+    if (zmax) zmax[i] = key_value(b);
+  }
+}
+void launch_unpack_best(cudaStream_t st, const unsigned long long* row_best, int rows, int* argmax, float* zmax) {
+  unpack_best_kernel<<<(rows + 255) / 256, 256, 0, st>>>(row_best, rows, argmax, zmax);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -66,3 +66,38 @@ def test_linear_matches_float64_product(models, flags, mode, shape):
         tol = 2.0 ** -8 * scale + 1e-3   # one bf16 rounding of the stored result
     err = np.abs(got - ref).max()
     assert err <= tol, f"shape {shape} mode {mode}: max err {err:.3e} > {tol:.3e}"
+
+
+@pytest.mark.parametrize("flags", [1, 0], ids=["simt", "tensor"])
+@pytest.mark.parametrize("rows", [1, 68, 300])
+def test_lm_head_argmax_matches_float64(models, flags, rows):
+    """Fused LM head: per-row argmax, its logit and the next token's logit against a float64 product."""
+    import torch
+    from paper_2602_12957_b200 import binding as B
+    model = models[flags]
+    cfg = model.cfg
+    rng = np.random.default_rng(rows)
+    h = I.bf16_round(rng.standard_normal((rows, cfg.d_model), dtype=np.float32))
+    nxt = rng.integers(0, cfg.vocab, rows).astype(np.int32)
+    nxt[0] = -1
+    W = model.lm_head.float().cpu().numpy().astype(np.float64)
+    z = h.astype(np.float64) @ W.T
+    dev = model.device
+    th = torch.from_numpy(h).to(dev, torch.bfloat16)
+    tn = torch.from_numpy(nxt).to(dev)
+    scratch = torch.empty(rows, dtype=torch.int64, device=dev)
+    am = torch.empty(rows, dtype=torch.int32, device=dev)
+    zm = torch.empty(rows, dtype=torch.float32, device=dev)
+    zd = torch.empty(rows, dtype=torch.float32, device=dev)
+    B.check(B.hsd_op_lm_head_argmax(model.ctx, th, rows, tn, scratch, rows * 8, am, zm, zd,
+                                    torch.cuda.current_stream().cuda_stream))
+    torch.cuda.synchronize()
+    am, zm, zd = am.cpu().numpy(), zm.cpu().numpy(), zd.cpu().numpy()
+    srt = np.sort(z, axis=1)
+    gap = srt[:, -1] - srt[:, -2]
+    assert np.abs(zm - srt[:, -1]).max() < 2e-3
+    clear = gap > 5e-3
+    assert np.array_equal(am[clear], z.argmax(1)[clear]) and clear.sum() > 0.5 * rows
+    assert np.all(z[np.arange(rows), am] >= srt[:, -1] - 5e-3)
+    assert np.isnan(zd[0])
+    assert np.abs(zd[1:] - z[np.arange(1, rows), nxt[1:]]).max() < 2e-3 if rows > 1 else True
