@@ -214,6 +214,30 @@ HSD_API int hsd_op_linear(hsd_ctx *ctx, const void *A, const void *W, void *C, i
 HSD_API int hsd_op_lm_head_argmax(hsd_ctx *ctx, const void *h, int rows, const int *next_tokens, void *scratch,
                           size_t scratch_bytes, int *argmax, float *zmax, float *zdraft, void *cuda_stream);
 
+/* hsd_op_lm_head_argmax_noalloc: the same operator for callers that cannot allocate device memory.
+ * (The paper has no counterpart; this is a packaging variant of the call above.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits, for example a plug-in called from inside another
+ * framework's stream-ordered section, a real-time loop that must not take the allocator's lock, or a process
+ * whose memory budget was handed out in full at start-up.  Such a caller already owns its inputs and outputs but
+ * has nowhere to get the operator's scratch from, so the scratch is a fixed array inside the library instead:
+ * HSD_NOALLOC_MAX_ROWS * 8 bytes (64 KB) of device memory that every GPU using the library holds until the
+ * process exits.
+ *
+ *   h, rows, next_tokens, argmax, zmax, zdraft, cuda_stream: exactly as for hsd_op_lm_head_argmax.
+ *   rows > HSD_NOALLOC_MAX_ROWS returns HSD_ERR_TOO_LONG and launches nothing.
+ *   The context must belong to the current device (HSD_ERR_INVALID_ARG otherwise).
+ *
+ * The call makes no cudaMalloc / cudaFree and uses no allocating library routine.  The first call on each device
+ * looks up the array's device address (one cudaGetSymbolAddress, checked); make that first call before any
+ * stream capture starts, and from one thread.  All calls on a device share the one array: each call clears the
+ * rows it uses before the GEMM, so nothing carries over from the previous call, but two calls whose kernels can
+ * overlap on the GPU (different streams without an ordering between them) race on it and corrupt each other's
+ * results.  Order them on one stream or with events. */
+#define HSD_NOALLOC_MAX_ROWS 8192
+HSD_API int hsd_op_lm_head_argmax_noalloc(hsd_ctx *ctx, const void *h, int rows, const int *next_tokens, int *argmax,
+                                  float *zmax, float *zdraft, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

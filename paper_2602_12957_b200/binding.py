@@ -20,12 +20,13 @@ HSD_MAX_Q_LEN = 4097
 HSD_KV_BLOCK = 64
 HSD_FLAG_SIMT_DEBUG = 1
 HSD_FLAG_SIMT_ATTENTION = 2
+HSD_NOALLOC_MAX_ROWS = 8192
 
 EXPORTS = [
     "hsd_status_string", "hsd_create", "hsd_destroy", "hsd_workspace_bytes", "hsd_prefill", "hsd_verify_regions",
     "hsd_verify_page", "hsd_kv_commit", "hsd_device_status", "hsd_last_cuda_error", "hsd_launch_count",
     "hsd_profile_enable", "hsd_profile_read", "hsd_debug_logits", "hsd_debug_buffer", "hsd_op_linear",
-    "hsd_op_lm_head_argmax",
+    "hsd_op_lm_head_argmax", "hsd_op_lm_head_argmax_noalloc",
 ]
 
 
@@ -81,6 +82,7 @@ def _load():
     lib.hsd_debug_buffer.argtypes = [vp, vp, i, i, C.c_char_p, C.POINTER(vp), C.POINTER(sz)]
     lib.hsd_op_linear.argtypes = [vp, vp, vp, vp, i, i, i, i, vp]
     lib.hsd_op_lm_head_argmax.argtypes = [vp, vp, i, vp, vp, sz, vp, vp, vp, vp]
+    lib.hsd_op_lm_head_argmax_noalloc.argtypes = [vp, vp, i, vp, vp, vp, vp, vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if name not in ("hsd_status_string", "hsd_workspace_bytes", "hsd_launch_count"):
@@ -230,3 +232,10 @@ def hsd_op_linear(ctx, A, W, Cout, M, n_out, K, mode, stream) -> int:
 def hsd_op_lm_head_argmax(ctx, h, rows, next_tokens, scratch, scratch_bytes, argmax, zmax, zdraft, stream) -> int:
     return _lib.hsd_op_lm_head_argmax(ctx, _p(h), rows, _p(next_tokens), _p(scratch), scratch_bytes, _p(argmax),
                                       _p(zmax), _p(zdraft), _p(stream))
+
+
+def hsd_op_lm_head_argmax_noalloc(ctx, h, rows, next_tokens, argmax, zmax, zdraft, stream) -> int:
+    """LM-head argmax for callers that cannot allocate: the scratch is a fixed array inside the library
+    (at most HSD_NOALLOC_MAX_ROWS rows; calls that may overlap on the GPU race on it)."""
+    return _lib.hsd_op_lm_head_argmax_noalloc(ctx, _p(h), rows, _p(next_tokens), _p(argmax), _p(zmax), _p(zdraft),
+                                              _p(stream))

@@ -712,6 +712,34 @@ int hsd_op_lm_head_argmax(hsd_ctx* c, const void* h, int rows, const int* next_t
                              static_cast<cudaStream_t>(cuda_stream));
 }
 
+// ---- the entry point for callers that cannot allocate device memory -------------------------------------
+// Scratch of the no-allocation LM-head operator: one 8-byte running-best word per row.  The array lives in the
+// library image, so every device that loads the library carries these 64 KB until the process exits.  In host
+// code the symbol below is only a stand-in; the device address comes from cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[HSD_NOALLOC_MAX_ROWS * 8];
+static unsigned long long* g_noalloc_addr[64] = {};   // per device ordinal, filled on that device's first call
+
+int hsd_op_lm_head_argmax_noalloc(hsd_ctx* c, const void* h, int rows, const int* next_tokens, int* argmax,
+                                  float* zmax, float* zdraft, void* cuda_stream) {
+  if (!c || !h || !argmax || !zmax || rows <= 0) return HSD_ERR_INVALID_ARG;
+  if (next_tokens && !zdraft) return HSD_ERR_INVALID_ARG;
+  if (rows > HSD_NOALLOC_MAX_ROWS) return HSD_ERR_TOO_LONG;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return fail_cuda(c);
+  if (dev != c->device || dev < 0 || dev >= 64) return HSD_ERR_INVALID_ARG;
+  if (!g_noalloc_addr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return fail_cuda(c);
+    g_noalloc_addr[dev] = static_cast<unsigned long long*>(p);
+  }
+  const bool was_profiling = c->profiling;   // event objects are created on demand while profiling: keep it off here
+  c->profiling = false;
+  const int rc = lm_head_argmax_impl(c, h, rows, next_tokens, g_noalloc_addr[dev], argmax, zmax, zdraft,
+                                     static_cast<cudaStream_t>(cuda_stream));
+  c->profiling = was_profiling;
+  return rc;
+}
+
 int hsd_op_linear(hsd_ctx* c, const void* A, const void* W, void* C, int M, int n_out, int K, int mode,
                   void* cuda_stream) {
   if (!c || !A || !W || !C || M <= 0 || n_out <= 0 || K <= 0) return HSD_ERR_INVALID_ARG;

@@ -40,3 +40,41 @@ def test_small_decoder_regions_match_oracle(flags):
     stats, orc, per, _ = run_region_parity(wl, flags)
     print("small", flags, stats, [(len(o.draft), o.res.accept_len) for o in orc.values()])
     assert stats["max_dz"] < H.LOGIT_TOL
+
+
+def test_one_verify_call_equals_sequential_single_token_steps_on_gpu():
+    """The library against itself: k+1 plain decode steps (empty drafts, commit each) must reproduce the rows of
+    one verify call over the tokens they emitted — same kernels, same K/V rows, same tile boundaries."""
+    import torch
+    from paper_2602_12957_b200 import runtime as R
+    cfg = I.small_decoder(2, 8192)
+    wl = I.region_workload(seed=91, n_regions=3, prefix_lo=60, prefix_hi=200, draft_mean=40, draft_lo=20, draft_hi=70,
+                           cfg=cfg)
+    weights = I.make_weights(cfg, 5)
+    model = R.DeviceModel(cfg, weights, 0)
+    S = len(wl.seqs)
+    k = 20
+    kv = R.KvCache(model, [s.prefix_len + k + 2 for s in wl.seqs], seed=1)
+    eng = R.Engine(model, kv, max(sum(s.prefix_len for s in wl.seqs), S * (k + 1)), S)
+    first = eng.prefill([s.prefix_embeds for s in wl.seqs], [s.prefix_ids for s in wl.seqs])
+    base = kv.seq_lens.clone()
+    cu1 = eng._i32(np.arange(S + 1))
+    pending, toks, zs = first.clone(), [], []
+    for _ in range(k + 1):
+        o = eng.verify_regions(pending, cu1, 1, S)
+        eng.commit(o["accept_len"])
+        zs.append(o["row_zmax"].clone())
+        pending = o["emit_tokens"][:, 0].clone()
+        toks.append(pending)
+    seq_z = torch.stack(zs, 1).cpu().numpy()              # [S, k+1]
+    greedy = torch.stack(toks, 1).cpu().numpy()           # [S, k+1]
+    assert (kv.seq_lens - base).cpu().numpy().tolist() == [k + 1] * S
+    kv.seq_lens.copy_(base)
+    q, cu = I.pack_queries(first.cpu().numpy(), [greedy[i, :k] for i in range(S)])
+    o = eng.verify_regions(eng._i32(q), eng._i32(cu), k + 1, S * (k + 1))
+    eng.check_device("verify")
+    z = o["row_zmax"].cpu().numpy().reshape(S, k + 1)
+    am = o["row_argmax"].cpu().numpy().reshape(S, k + 1)
+    assert np.array_equal(am, greedy), "teacher-forced rows must reproduce the sequential greedy tokens"
+    assert np.array_equal(z, seq_z), f"max |dz| {np.abs(z - seq_z).max()}"
+    assert o["accept_len"].cpu().numpy().tolist() == [k] * S
