@@ -70,6 +70,11 @@ extern "C" {
 #define HSD_FLAG_SIMT_DEBUG 1      /* run the plain SIMT kernels instead of the tensor-core kernels;
                                       a slow cross-check for debugging, never a fallback              */
 #define HSD_FLAG_SIMT_ATTENTION 2  /* debugging: only the attention runs through its plain kernel     */
+#define HSD_FLAG_DETERMINISTIC 4   /* no split-K in the residual-add projections: their K slices add into
+                                      the fp32 residual in arrival order, so results can differ in the last
+                                      bit from run to run; with this flag every run is bit-identical      */
+#define HSD_FLAG_NO_PDL 8          /* debugging: plain stream-ordered launches (no programmatic dependent
+                                      launch overlap between consecutive kernels)                       */
 
 typedef struct hsd_ctx hsd_ctx;
 
@@ -202,6 +207,11 @@ HSD_API int hsd_debug_buffer(hsd_ctx *ctx, const void *workspace, int total_q, i
  *   A dev bf16 [M,K], W dev bf16 [n_out,K].  M >= 1; K, n_out multiples of 64. */
 HSD_API int hsd_op_linear(hsd_ctx *ctx, const void *A, const void *W, void *C, int M, int n_out, int K, int mode,
                   void *cuda_stream);
+
+/* Test-only: make hsd_op_linear use output tiles of `tile_n` columns (64, 128 or 256) and, for mode 1, `k_slices`
+ * slices of K per tile, instead of what the library would choose for the problem; 0 = choose.  A combination the
+ * problem does not allow makes hsd_op_linear return HSD_ERR_CUDA.  Lets the parity tests reach every tile shape. */
+HSD_API int hsd_debug_set_gemm_tile(hsd_ctx *ctx, int tile_n, int k_slices);
 
 /* hsd_op_lm_head_argmax: the fused LM head on its own (Eq. 10 per row): for `rows` already-normalised hidden rows
  * h (dev bf16 [rows, d_model]) compute z = h W_lm^T tile by tile and keep only, per row, the argmax (lowest id on

@@ -20,13 +20,15 @@ HSD_MAX_Q_LEN = 4097
 HSD_KV_BLOCK = 64
 HSD_FLAG_SIMT_DEBUG = 1
 HSD_FLAG_SIMT_ATTENTION = 2
+HSD_FLAG_DETERMINISTIC = 4
+HSD_FLAG_NO_PDL = 8
 HSD_NOALLOC_MAX_ROWS = 8192
 
 EXPORTS = [
     "hsd_status_string", "hsd_create", "hsd_destroy", "hsd_workspace_bytes", "hsd_prefill", "hsd_verify_regions",
     "hsd_verify_page", "hsd_kv_commit", "hsd_device_status", "hsd_last_cuda_error", "hsd_launch_count",
     "hsd_profile_enable", "hsd_profile_read", "hsd_debug_logits", "hsd_debug_buffer", "hsd_op_linear",
-    "hsd_op_lm_head_argmax", "hsd_op_lm_head_argmax_noalloc",
+    "hsd_op_lm_head_argmax", "hsd_op_lm_head_argmax_noalloc", "hsd_debug_set_gemm_tile",
 ]
 
 
@@ -80,6 +82,7 @@ def _load():
     lib.hsd_profile_read.argtypes = [vp, i, C.POINTER(C.c_char_p), C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
     lib.hsd_debug_logits.argtypes = [vp, vp, i, i, vp, vp]
     lib.hsd_debug_buffer.argtypes = [vp, vp, i, i, C.c_char_p, C.POINTER(vp), C.POINTER(sz)]
+    lib.hsd_debug_set_gemm_tile.argtypes = [vp, i, i]
     lib.hsd_op_linear.argtypes = [vp, vp, vp, vp, i, i, i, i, vp]
     lib.hsd_op_lm_head_argmax.argtypes = [vp, vp, i, vp, vp, sz, vp, vp, vp, vp]
     lib.hsd_op_lm_head_argmax_noalloc.argtypes = [vp, vp, i, vp, vp, vp, vp, vp]
@@ -223,6 +226,10 @@ def hsd_debug_buffer(ctx, workspace, total_q, n_seqs, name: str):
     ptr, sz = C.c_void_p(), C.c_size_t()
     st = _lib.hsd_debug_buffer(ctx, _p(workspace), total_q, n_seqs, name.encode(), C.byref(ptr), C.byref(sz))
     return st, ptr.value, sz.value
+
+
+def hsd_debug_set_gemm_tile(ctx, tile_n: int, k_slices: int) -> int:
+    return _lib.hsd_debug_set_gemm_tile(ctx, tile_n, k_slices)
 
 
 def hsd_op_linear(ctx, A, W, Cout, M, n_out, K, mode, stream) -> int:

@@ -13,7 +13,7 @@ using namespace hsd;
 namespace hsd {
 int launch_attn_sm100(cudaStream_t st, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                       const RowMeta& rm, const KvView& kv, const ModelDims& md, int layer, bf16* out, int n_seqs,
-                      int max_tiles, const int* tile_count, int* status, float* split_ws);
+                      int max_tiles, const int* tile_count, int* status, float* split_ws, bool pdl);
 }
 
 struct ProfEvent {
@@ -26,8 +26,11 @@ struct hsd_ctx {
   ModelDims md;
   const bf16 *embed, *lm_head, *final_norm;
   std::vector<const bf16*> attn_norm, w_qkv, w_o, ffn_norm, w_gate_up, w_down;
-  std::vector<CUtensorMap> tm_qkv, tm_o, tm_gate_up, tm_down;
-  CUtensorMap tm_lm_head;
+  std::vector<WeightMaps> tm_qkv, tm_o, tm_gate_up, tm_down;
+  WeightMaps tm_lm_head;
+  int max_splits;     // K slices the residual-add projections may use (1 with HSD_FLAG_DETERMINISTIC)
+  bool pdl;           // kernels are launched with programmatic stream serialization
+  int force_bn, force_splits;   // hsd_debug_set_gemm_tile
   int n_sms;
   int device;
   bool simt;
@@ -204,18 +207,22 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
     sa.allow_embed_rows = a.prefill && a.embeds != nullptr;
     sa.rope_base = md.rope_base;
     sa.head_dim = md.D;
-    launch_setup_rows(st, sa, kv, w.rm, w.status, w.status + 4);
+    launch_setup_rows(st, sa, kv, w.rm, w.status, w.status + 4, c->pdl);
   }
   {
     Scope s(c, st, KC_EMBED);
-    launch_embed(st, w.rm, c->embed, static_cast<const bf16*>(a.embeds), w.x, T, md.d, w.status);
+    launch_embed(st, w.rm, c->embed, static_cast<const bf16*>(a.embeds), w.x, T, md.d, w.status, c->pdl);
   }
 
-  CUtensorMap tm_h, tm_attn, tm_act, tm_q, tm_k, tm_v;
+  CUtensorMap tm_h, tm_attn, tm_act, tm_q, tm_k, tm_v, tm_x_add, tm_q_st, tm_act_st;
   const int max_tiles = T / tokens_per_tile + a.n_seqs;
   if (!c->simt) {
     if (make_tmap_2d(&tm_h, w.h, T, md.d, 128) || make_tmap_2d(&tm_attn, w.attn, T, md.Hq * md.D, 128) ||
         make_tmap_2d(&tm_act, w.act, T, md.ffn, 128))
+      return HSD_ERR_CUDA;
+    // epilogue targets: residual stream (fp32 reduce-add), q and the SwiGLU activation (bf16 stores)
+    if (make_tmap_2d_f32(&tm_x_add, w.x, T, md.d, 32) || make_tmap_2d(&tm_q_st, w.q, T, md.Hq * md.D, 32) ||
+        make_tmap_2d(&tm_act_st, w.act, T, md.ffn, 32))
       return HSD_ERR_CUDA;
     // q as [T][Hq][64]: one box = (128/group) tokens x group heads x 64 dims -> a 128-row MMA operand
     if (make_tmap_3d(&tm_q, w.q, 64, md.Hq, T, 128, (uint64_t)md.Hq * 128, 64, md.group, tokens_per_tile))
@@ -229,7 +236,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
   for (int l = 0; l < md.n_layers; ++l) {
     {
       Scope s(c, st, KC_RMSNORM);
-      launch_rmsnorm(st, w.x, c->attn_norm[l], w.h, T, md.d, md.eps, nullptr);
+      launch_rmsnorm(st, w.x, c->attn_norm[l], w.h, T, md.d, md.eps, nullptr, c->pdl);
     }
     const size_t layer_elems = (size_t)kv.n_blocks * md.Hkv * 64 * 64;
     if (c->simt) {
@@ -256,7 +263,8 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         Scope s(c, st, KC_GEMM_QKV);
         GemmSm100Args g = {};
         g.tmA = tm_h;
-        g.tmB = c->tm_qkv[l];
+        g.tmB = &c->tm_qkv[l];
+        g.tmC = tm_q_st;
         g.M = T; g.n_out = md.qkv_out; g.K = md.d; g.mode = GS_QKV_ROPE;
         g.qkv.row_kv = w.rm.row_kv;
         g.qkv.rope_cs = w.rm.rope_cs;
@@ -264,7 +272,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         g.qkv.k_pool_layer = kv.k_pool + (size_t)l * layer_elems;
         g.qkv.v_pool_layer = kv.v_pool + (size_t)l * layer_elems;
         g.qkv.Hq = md.Hq; g.qkv.Hkv = md.Hkv;
-        g.status = w.status; g.n_sms = c->n_sms;
+        g.status = w.status; g.n_sms = c->n_sms; g.max_splits = 1; g.pdl = c->pdl;
         if (launch_gemm_sm100(st, g)) return fail_cuda(c);
       }
       {
@@ -272,7 +280,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         if (c->attn_simt) {
           launch_attn_simt(st, w.q, w.rm, kv, md, l, w.attn, T, w.status);
         } else if (launch_attn_sm100(st, tm_q, tm_k, tm_v, w.rm, kv, md, l, w.attn, a.n_seqs, max_tiles, w.status + 4,
-                                     w.status, w.split_ws)) {
+                                     w.status, w.split_ws, c->pdl)) {
           return fail_cuda(c);
         }
       }
@@ -280,16 +288,16 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         Scope s(c, st, KC_GEMM_O);
         GemmSm100Args g = {};
         g.tmA = tm_attn;
-        g.tmB = c->tm_o[l];
+        g.tmB = &c->tm_o[l];
+        g.tmC = tm_x_add;
         g.M = T; g.n_out = md.d; g.K = md.Hq * md.D; g.mode = GS_ADD_F32;
-        g.out.C = w.x; g.out.ldc = md.d;
-        g.status = w.status; g.n_sms = c->n_sms;
-        if (launch_gemm_sm100(st, g)) return HSD_ERR_CUDA;
+        g.status = w.status; g.n_sms = c->n_sms; g.max_splits = c->max_splits; g.pdl = c->pdl;
+        if (launch_gemm_sm100(st, g)) return fail_cuda(c);
       }
     }
     {
       Scope s(c, st, KC_RMSNORM);
-      launch_rmsnorm(st, w.x, c->ffn_norm[l], w.h, T, md.d, md.eps, nullptr);
+      launch_rmsnorm(st, w.x, c->ffn_norm[l], w.h, T, md.d, md.eps, nullptr, c->pdl);
     }
     if (c->simt) {
       {
@@ -307,21 +315,21 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         Scope s(c, st, KC_GEMM_GATEUP);
         GemmSm100Args g = {};
         g.tmA = tm_h;
-        g.tmB = c->tm_gate_up[l];
+        g.tmB = &c->tm_gate_up[l];
+        g.tmC = tm_act_st;
         g.M = T; g.n_out = 2 * md.ffn; g.K = md.d; g.mode = GS_SWIGLU;
-        g.out.C = w.act; g.out.ldc = md.ffn;
-        g.status = w.status; g.n_sms = c->n_sms;
-        if (launch_gemm_sm100(st, g)) return HSD_ERR_CUDA;
+        g.status = w.status; g.n_sms = c->n_sms; g.max_splits = 1; g.pdl = c->pdl;
+        if (launch_gemm_sm100(st, g)) return fail_cuda(c);
       }
       {
         Scope s(c, st, KC_GEMM_DOWN);
         GemmSm100Args g = {};
         g.tmA = tm_act;
-        g.tmB = c->tm_down[l];
+        g.tmB = &c->tm_down[l];
+        g.tmC = tm_x_add;
         g.M = T; g.n_out = md.d; g.K = md.ffn; g.mode = GS_ADD_F32;
-        g.out.C = w.x; g.out.ldc = md.d;
-        g.status = w.status; g.n_sms = c->n_sms;
-        if (launch_gemm_sm100(st, g)) return HSD_ERR_CUDA;
+        g.status = w.status; g.n_sms = c->n_sms; g.max_splits = c->max_splits; g.pdl = c->pdl;
+        if (launch_gemm_sm100(st, g)) return fail_cuda(c);
       }
     }
   }
@@ -333,7 +341,7 @@ int run_lm_head(hsd_ctx* c, const Ws& w, int rows, const int* row_next, cudaStre
   const ModelDims& md = c->md;
   {
     Scope s(c, st, KC_LMHEAD);
-    launch_clear_best(st, w.row_best, w.zdraft, rows);
+    launch_clear_best(st, w.row_best, w.zdraft, rows, c->pdl);
   }
   Scope s(c, st, KC_LMHEAD);
   GemmOut o = {nullptr, 0, w.row_best, w.zdraft, row_next};
@@ -344,11 +352,11 @@ int run_lm_head(hsd_ctx* c, const Ws& w, int rows, const int* row_next, cudaStre
     if (make_tmap_2d(&tm_h, w.h, rows, md.d, 128)) return HSD_ERR_CUDA;
     GemmSm100Args g = {};
     g.tmA = tm_h;
-    g.tmB = c->tm_lm_head;
+    g.tmB = &c->tm_lm_head;
     g.M = rows; g.n_out = md.V; g.K = md.d; g.mode = GS_ARGMAX;
     g.out = o;
-    g.status = w.status; g.n_sms = c->n_sms;
-    if (launch_gemm_sm100(st, g)) return HSD_ERR_CUDA;
+    g.status = w.status; g.n_sms = c->n_sms; g.max_splits = 1; g.pdl = c->pdl;
+    if (launch_gemm_sm100(st, g)) return fail_cuda(c);
   }
   return check_cuda(c);
 }
@@ -369,7 +377,7 @@ int verify_common(hsd_ctx* c, const hsd_kv* kv, const StepArgs& a, float log_tau
   if (rc) return rc;
   {
     Scope s(c, st, KC_RMSNORM);
-    launch_rmsnorm(st, w.x, c->final_norm, w.h, a.total_q, c->md.d, c->md.eps, nullptr);
+    launch_rmsnorm(st, w.x, c->final_norm, w.h, a.total_q, c->md.d, c->md.eps, nullptr, c->pdl);
   }
   rc = run_lm_head(c, w, a.total_q, w.rm.row_next, st);
   if (rc) return rc;
@@ -387,7 +395,7 @@ int verify_common(hsd_ctx* c, const hsd_kv* kv, const StepArgs& a, float log_tau
     aa.row_argmax = row_argmax;
     aa.row_zmax = row_zmax;
     aa.row_zdraft = row_zdraft;
-    launch_accept(st, aa, w.rm, w.status);
+    launch_accept(st, aa, w.rm, w.status, c->pdl);
   }
   return check_cuda(c);
 }
@@ -459,6 +467,9 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
   c->device = dev;
   c->simt = (cfg->flags & HSD_FLAG_SIMT_DEBUG) != 0;
   c->attn_simt = c->simt || (cfg->flags & HSD_FLAG_SIMT_ATTENTION) != 0;
+  c->max_splits = (cfg->flags & HSD_FLAG_DETERMINISTIC) ? 1 : 8;
+  c->pdl = (cfg->flags & HSD_FLAG_NO_PDL) == 0;
+  c->force_bn = c->force_splits = 0;
   c->last_cuda_error = 0;
   c->launches = 0;
   c->profiling = false;
@@ -470,12 +481,12 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
     c->tm_gate_up.resize(md.n_layers); c->tm_down.resize(md.n_layers);
     int bad = 0;
     for (int l = 0; l < md.n_layers; ++l) {
-      bad |= make_tmap_2d(&c->tm_qkv[l], c->w_qkv[l], md.qkv_out, md.d, 64);
-      bad |= make_tmap_2d(&c->tm_o[l], c->w_o[l], md.d, md.Hq * 64, 64);
-      bad |= make_tmap_2d(&c->tm_gate_up[l], c->w_gate_up[l], 2 * md.ffn, md.d, 64);
-      bad |= make_tmap_2d(&c->tm_down[l], c->w_down[l], md.d, md.ffn, 64);
+      bad |= make_weight_tmaps(&c->tm_qkv[l], c->w_qkv[l], md.qkv_out, md.d);
+      bad |= make_weight_tmaps(&c->tm_o[l], c->w_o[l], md.d, md.Hq * 64);
+      bad |= make_weight_tmaps(&c->tm_gate_up[l], c->w_gate_up[l], 2 * md.ffn, md.d);
+      bad |= make_weight_tmaps(&c->tm_down[l], c->w_down[l], md.d, md.ffn);
     }
-    bad |= make_tmap_2d(&c->tm_lm_head, c->lm_head, md.V, md.d, 64);
+    bad |= make_weight_tmaps(&c->tm_lm_head, c->lm_head, md.V, md.d);
     if (bad) { delete c; return HSD_ERR_CUDA; }
   }
   *out = c;
@@ -515,17 +526,17 @@ int hsd_prefill(hsd_ctx* c, const hsd_kv* kv, int n_seqs, const int* cu_len, con
   if (rc) return rc;
   {
     Scope s(c, st, KC_RMSNORM);
-    launch_select_last_rows(st, w.rm, n_seqs, w.sel_rows);
+    launch_select_last_rows(st, w.rm, n_seqs, w.sel_rows, c->pdl);
   }
   {
     Scope s(c, st, KC_RMSNORM);
-    launch_rmsnorm(st, w.x, c->final_norm, w.h, n_seqs, c->md.d, c->md.eps, w.sel_rows);
+    launch_rmsnorm(st, w.x, c->final_norm, w.h, n_seqs, c->md.d, c->md.eps, w.sel_rows, c->pdl);
   }
   rc = run_lm_head(c, w, n_seqs, nullptr, st);
   if (rc) return rc;
   {
     Scope s(c, st, KC_ACCEPT);
-    launch_first_token(st, w.row_best, n_seqs, first_token, w.rm, kv_view(kv), w.status);
+    launch_first_token(st, w.row_best, n_seqs, first_token, w.rm, kv_view(kv), w.status, c->pdl);
   }
   return check_cuda(c);
 }
@@ -596,7 +607,7 @@ int hsd_kv_commit(hsd_ctx* c, const hsd_kv* kv, int n_seqs, const int* seq_slots
   if (!seq_slots && n_seqs > kv->n_slots) return HSD_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   Scope s(c, st, KC_COMMIT);
-  launch_commit(st, kv_view(kv), n_seqs, seq_slots, accept_len, blocks_in_use);
+  launch_commit(st, kv_view(kv), n_seqs, seq_slots, accept_len, blocks_in_use, c->pdl);
   return check_cuda(c);
 }
 
@@ -679,7 +690,7 @@ static int lm_head_argmax_impl(hsd_ctx* c, const void* h, int rows, const int* n
   const ModelDims& md = c->md;
   {
     Scope s(c, st, KC_LMHEAD);
-    launch_clear_best(st, best, next_tokens ? zdraft : nullptr, rows);
+    launch_clear_best(st, best, next_tokens ? zdraft : nullptr, rows, false);
   }
   {
     Scope s(c, st, KC_LMHEAD);
@@ -689,16 +700,16 @@ static int lm_head_argmax_impl(hsd_ctx* c, const void* h, int rows, const int* n
     } else {
       GemmSm100Args g = {};
       if (make_tmap_2d(&g.tmA, h, rows, md.d, 128)) return HSD_ERR_CUDA;
-      g.tmB = c->tm_lm_head;
+      g.tmB = &c->tm_lm_head;
       g.M = rows; g.n_out = md.V; g.K = md.d; g.mode = GS_ARGMAX;
       g.out = o;
-      g.status = nullptr; g.n_sms = c->n_sms;
+      g.status = nullptr; g.n_sms = c->n_sms; g.max_splits = 1; g.pdl = false;
       if (launch_gemm_sm100(st, g)) return fail_cuda(c);
     }
   }
   {
     Scope s(c, st, KC_LMHEAD);
-    launch_unpack_best(st, best, rows, argmax, zmax);
+    launch_unpack_best(st, best, rows, argmax, zmax, false);
   }
   return check_cuda(c);
 }
@@ -740,6 +751,13 @@ int hsd_op_lm_head_argmax_noalloc(hsd_ctx* c, const void* h, int rows, const int
   return rc;
 }
 
+int hsd_debug_set_gemm_tile(hsd_ctx* c, int tile_n, int k_slices) {
+  if (!c || tile_n < 0 || k_slices < 0) return HSD_ERR_INVALID_ARG;
+  c->force_bn = tile_n;
+  c->force_splits = k_slices;
+  return HSD_OK;
+}
+
 int hsd_op_linear(hsd_ctx* c, const void* A, const void* W, void* C, int M, int n_out, int K, int mode,
                   void* cuda_stream) {
   if (!c || !A || !W || !C || M <= 0 || n_out <= 0 || K <= 0) return HSD_ERR_INVALID_ARG;
@@ -753,10 +771,13 @@ int hsd_op_linear(hsd_ctx* c, const void* A, const void* W, void* C, int M, int 
     return check_cuda(c);
   }
   GemmSm100Args g = {};
-  if (make_tmap_2d(&g.tmA, A, M, K, 128) || make_tmap_2d(&g.tmB, W, n_out, K, 64)) return HSD_ERR_CUDA;
+  WeightMaps wm;
+  if (make_tmap_2d(&g.tmA, A, M, K, 128) || make_weight_tmaps(&wm, W, n_out, K)) return HSD_ERR_CUDA;
+  if (mode == 1 ? make_tmap_2d_f32(&g.tmC, C, M, ldc, 32) : make_tmap_2d(&g.tmC, C, M, ldc, 32)) return HSD_ERR_CUDA;
+  g.tmB = &wm;
   g.M = M; g.n_out = n_out; g.K = K; g.mode = mode;
-  g.out.C = C; g.out.ldc = ldc;
-  g.status = nullptr; g.n_sms = c->n_sms;
+  g.status = nullptr; g.n_sms = c->n_sms; g.max_splits = c->max_splits; g.pdl = false;
+  g.force_bn = c->force_bn; g.force_splits = c->force_splits;
   if (launch_gemm_sm100(st, g)) return fail_cuda(c);
   return check_cuda(c);
 }

@@ -49,6 +49,8 @@ __device__ __forceinline__ float ex2(float x) {
 __global__ void __launch_bounds__(kAttnThreads, 2)
 attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, AttnParams p) {
+  pdl_wait();               // q, the K/V rows of this step and the row metadata come from earlier kernels
+  pdl_launch_dependents();
   if (*p.status) return;
   const int tile_idx = blockIdx.x / p.Hkv;
   const int kvh = blockIdx.x % p.Hkv;
@@ -295,7 +297,7 @@ done:
 
 int launch_attn_sm100(cudaStream_t st, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                         const RowMeta& rm, const KvView& kv, const ModelDims& md, int layer, bf16* out, int n_seqs,
-                        int max_tiles, const int* tile_count, int* status, float* split_ws) {
+                        int max_tiles, const int* tile_count, int* status, float* split_ws, bool pdl) {
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(attn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_SMEM) != cudaSuccess)
@@ -316,8 +318,8 @@ int launch_attn_sm100(cudaStream_t st, const CUtensorMap& tmQ, const CUtensorMap
   p.tile_count = tile_count;
   p.status = status;
   p.n_seqs = n_seqs;
-  attn_sm100_kernel<<<max_tiles * md.Hkv, kAttnThreads, ATTN_SMEM, st>>>(tmQ, tmK, tmV, p);
-  return cudaGetLastError() == cudaSuccess ? 0 : -1;
+  return launch_kernel(attn_sm100_kernel, dim3(max_tiles * md.Hkv), dim3(kAttnThreads), ATTN_SMEM, st, pdl, tmQ, tmK, tmV,
+                       p);
 }
 
 }  // namespace hsd

@@ -1,14 +1,21 @@
 // tcgen05 / TMEM GEMM for sm_100a:  C = A W^T,  A [M,K] bf16 (activations), W [n_out,K] bf16 (weights),
 // fp32 accumulation in tensor memory, operands staged in shared memory by TMA (128-byte swizzle).
 //
-// One persistent CTA per SM walks 128 x BN output tiles (M fastest, so CTAs running side by side share a
-// weight tile through L2).  Warp roles: warp 0 = TMA producer (one elected lane), warp 1 = MMA issuer (one
-// lane) and TMEM owner, warps 2..5 = epilogue (one TMEM lane quarter each).  Two accumulator buffers in
-// TMEM let the epilogue of tile i overlap the main loop of tile i+1.
+// One persistent CTA per SM walks work units (128 x BN output tile, optionally one slice of K), M fastest so
+// CTAs running side by side share a weight tile through L2.  Warp roles:
+//   warp 0      A producer (one lane): activation tile, one 128-row TMA box per stage
+//   warp 1      MMA issuer (one lane) and TMEM owner
+//   warps 2, 3  B producers (one lane each): the two halves of the weight tile, one TMA box each per stage.
+//               A TMA instruction costs its issuing thread ~0.25 us whatever the box size, so a stage is three
+//               large boxes issued from three warps instead of many small ones from one.  Weights do not depend
+//               on the previous kernel, so these two start before the programmatic-launch wait.
+//   warps 4..7  epilogue, one TMEM lane quarter each
+// Two accumulator buffers in TMEM let the epilogue of unit i overlap the main loop of unit i+1.
 //
-// Epilogues (all fused, nothing but the final result goes to HBM):
+// Epilogues (all fused; results leave the SM through swizzled staging buffers and TMA stores, so global
+// writes are full 128-byte lines whatever the thread-to-row mapping in TMEM):
 //   GS_STORE_BF16  C bf16 = acc
-//   GS_ADD_F32     C fp32 += acc                         (O and down projections into the residual stream)
+//   GS_ADD_F32     C fp32 += acc   (TMA reduce-add into the residual stream; with split-K every K slice adds)
 //   GS_SWIGLU      C bf16 = silu(gate) * up              (gate rows and up rows of W land in one tile)
 //   GS_ARGMAX      per-row running argmax over the vocabulary + the next draft token's logit; logits never
 //                  leave the SM (Eq. 10 of the paper fused into the LM head)
@@ -46,6 +53,18 @@ int make_tmap_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t col
   return r == CUDA_SUCCESS ? 0 : -1;
 }
 
+int make_tmap_2d_f32(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  if (!g_encode) return -1;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 4};
+  cuuint32_t box[2] = {32, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? 0 : -1;
+}
+
 int make_tmap_3d(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t stride1_bytes,
                  uint64_t stride2_bytes, uint32_t b0, uint32_t b1, uint32_t b2) {
   if (!g_encode) return -1;
@@ -59,11 +78,19 @@ int make_tmap_3d(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, u
   return r == CUDA_SUCCESS ? 0 : -1;
 }
 
+int make_weight_tmaps(WeightMaps* w, const void* base, uint64_t rows, uint64_t cols) {
+  int bad = 0;
+  for (int i = 0; i < 3; ++i) bad |= make_tmap_2d(&w->m[i], base, rows, cols, 32u << i);
+  return bad;
+}
+
 // ------------------------------------------------------------------------------------------------
 constexpr int BM = 128;
 constexpr int BK = 64;
 constexpr int A_BYTES = BM * BK * 2;
-constexpr int kGemmThreads = 192;
+constexpr int kGemmThreads = 256;
+constexpr int STG_BYTES = 4096;                  // one epilogue staging buffer: 32 rows x 128 bytes
+constexpr int STG_TOTAL = 4 * 2 * STG_BYTES;     // four epilogue warps, two buffers each
 
 template <int BN>
 struct Cfg {
@@ -71,24 +98,59 @@ struct Cfg {
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
   static constexpr int TMEM_COLS = 2 * BN;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STG_TOTAL + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
 struct GemmDev {
   int M, n_cols, K, n_up_off;   // n_cols: output columns; n_up_off: row offset of the `up` half (SwiGLU)
+  int splits, kb_per_split;     // K slices per tile (GS_ADD_F32 only) and k-blocks per slice
   GemmOut out;
   QkvEpilogue qkv;
   int* status;
 };
 
+// TMA store / reduce of one staging buffer and the bulk-group bookkeeping around it (issued by one lane).
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* smem_src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(smem_src)), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, const void* smem_src, int x, int y) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(smem_src)), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// 16-byte chunk `c` of this lane's 128-byte staging row, at its 128-byte-swizzle position.
+__device__ __forceinline__ uint4* stg_chunk(uint8_t* buf, int lane, int c) {
+  return reinterpret_cast<uint4*>(buf + lane * 128 + ((c ^ (lane & 7)) << 4));
+}
+__device__ __forceinline__ uint4 pack8(const uint32_t* r) {
+  uint4 o;
+  o.x = pack_bf16(__uint_as_float(r[0]), __uint_as_float(r[1]));
+  o.y = pack_bf16(__uint_as_float(r[2]), __uint_as_float(r[3]));
+  o.z = pack_bf16(__uint_as_float(r[4]), __uint_as_float(r[5]));
+  o.w = pack_bf16(__uint_as_float(r[6]), __uint_as_float(r[7]));
+  return o;
+}
+
 template <int BN, int MODE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmDev p) {
+gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                  const __grid_constant__ CUtensorMap tmC, GemmDev p) {
   using C = Cfg<BN>;
   constexpr int OUT_N = (MODE == GS_SWIGLU) ? BN / 2 : BN;   // output columns per tile
+  constexpr int HALF_B = BN / 2 * BK * 2;                    // bytes of one weight half-tile
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::STAGES * C::STAGE_BYTES);
+  uint8_t* stg = smem + C::STAGES * C::STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(stg + STG_TOTAL);
   uint64_t* full = bars;
   uint64_t* empty = bars + C::STAGES;
   uint64_t* tfull = bars + 2 * C::STAGES;
@@ -99,7 +161,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) {
-      mbar_init(full + s, 1);
+      mbar_init(full + s, 3);      // A producer + two B producers, each with its own byte count
       mbar_init(empty + s, 1);
     }
     for (int b = 0; b < 2; ++b) {
@@ -110,6 +172,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     fence_mbar_init();
     tma_prefetch_desc(&tmA);
     tma_prefetch_desc(&tmB);
+    if (MODE != GS_ARGMAX) tma_prefetch_desc(&tmC);
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, C::TMEM_COLS);
@@ -122,33 +185,44 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
   const int m_tiles = (p.M + BM - 1) / BM;
   const int n_tiles = p.n_cols / OUT_N;
-  const int total = m_tiles * n_tiles;
+  const int tiles = m_tiles * n_tiles;
+  const int total = tiles * p.splits;
   const int k_blocks = p.K / BK;
 
-  pdl_wait();
-
   if (warp == 0) {
+    // ---- A producer: activations, written by the previous kernel
     if (lane == 0) {
+      pdl_wait();
+      pdl_launch_dependents();
       int s = 0;
       uint32_t ph = 0;
       for (int t = blockIdx.x; t < total; t += gridDim.x) {
-        const int m0 = (t % m_tiles) * BM, n0 = (t / m_tiles) * OUT_N;
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        const int tile = t % tiles, split = t / tiles;
+        const int m0 = (tile % m_tiles) * BM;
+        const int kb0 = split * p.kb_per_split, kb1 = min(k_blocks, kb0 + p.kb_per_split);
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty + s, ph ^ 1u, abort_flag, p.status, 100)) goto done;
-          uint8_t* sa = smem + s * C::STAGE_BYTES;
-          uint8_t* sb = sa + A_BYTES;
-          mbar_expect_tx(full + s, C::STAGE_BYTES);
-          tma_load_2d(sa, &tmA, full + s, kb * BK, m0);
-          if (MODE == GS_SWIGLU) {
-#pragma unroll
-            for (int j = 0; j < OUT_N / 64; ++j) {
-              tma_load_2d(sb + j * 8192, &tmB, full + s, kb * BK, n0 + j * 64);
-              tma_load_2d(sb + (OUT_N / 64 + j) * 8192, &tmB, full + s, kb * BK, p.n_up_off + n0 + j * 64);
-            }
-          } else {
-#pragma unroll
-            for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * 8192, &tmB, full + s, kb * BK, n0 + j * 64);
-          }
+          mbar_expect_tx(full + s, A_BYTES);
+          tma_load_2d(smem + s * C::STAGE_BYTES, &tmA, full + s, kb * BK, m0);
+          if (++s == C::STAGES) { s = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 2 || warp == 3) {
+    // ---- B producers: one half of the weight tile each (for SwiGLU: gate rows / up rows)
+    if (lane == 0) {
+      const int half = warp - 2;
+      int s = 0;
+      uint32_t ph = 0;
+      for (int t = blockIdx.x; t < total; t += gridDim.x) {
+        const int tile = t % tiles, split = t / tiles;
+        const int n0 = (tile / m_tiles) * OUT_N;
+        const int kb0 = split * p.kb_per_split, kb1 = min(k_blocks, kb0 + p.kb_per_split);
+        const int row = (MODE == GS_SWIGLU) ? (half ? p.n_up_off + n0 : n0) : n0 + half * (BN / 2);
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(empty + s, ph ^ 1u, abort_flag, p.status, 110 + half)) goto done;
+          mbar_expect_tx(full + s, HALF_B);
+          tma_load_2d(smem + s * C::STAGE_BYTES + A_BYTES + half * HALF_B, &tmB, full + s, kb * BK, row);
           if (++s == C::STAGES) { s = 0; ph ^= 1u; }
         }
       }
@@ -160,19 +234,22 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       uint32_t ph = 0;
       int it = 0;
       for (int t = blockIdx.x; t < total; t += gridDim.x, ++it) {
+        const int split = t / tiles;
+        const int kb0 = split * p.kb_per_split, kb1 = min(k_blocks, kb0 + p.kb_per_split);
         const int b = it & 1;
         const uint32_t aph = (it >> 1) & 1;
         if (!mbar_wait(tempty + b, aph ^ 1u, abort_flag, p.status, 200)) goto done;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + b * BN;
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full + s, ph, abort_flag, p.status, 201)) goto done;
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + s * C::STAGE_BYTES);
           const uint32_t sb = sa + A_BYTES;
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k) {
-            umma_bf16(d_tmem, umma_desc_sw128(sa + k * 32), umma_desc_sw128(sb + k * 32), idesc, (kb | k) != 0);
+            umma_bf16(d_tmem, umma_desc_sw128(sa + k * 32), umma_desc_sw128(sb + k * 32), idesc,
+                      (kb != kb0 || k != 0) ? 1u : 0u);
           }
           umma_commit(empty + s);      // smem stage reusable once these MMAs have read it
           if (++s == C::STAGES) { s = 0; ph ^= 1u; }
@@ -181,78 +258,102 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       }
     }
   } else {
+    // ---- epilogue warps 4..7
     const int quarter = warp & 3;                 // TMEM lanes [32*quarter, +32) belong to this warp
     const int row_in_tile = quarter * 32 + lane;
+    uint8_t* my_stg = stg + quarter * 2 * STG_BYTES;
+    int n_stores = 0;                             // staging buffers handed to TMA so far (selects the buffer)
+    pdl_wait();
     int it = 0;
     for (int t = blockIdx.x; t < total; t += gridDim.x, ++it) {
       const int b = it & 1;
       const uint32_t aph = (it >> 1) & 1;
-      const int m0 = (t % m_tiles) * BM, n0 = (t / m_tiles) * OUT_N;
+      const int tile = t % tiles;
+      const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * OUT_N;
       const int row = m0 + row_in_tile;
       const bool row_ok = row < p.M;
+      const int wrow0 = m0 + quarter * 32;        // first row of this warp's 32-row slab
+      const bool slab_ok = wrow0 < p.M;           // warp-uniform: the slab has at least one real row
       bool ok = mbar_wait(tfull + b, aph, abort_flag, p.status, 300);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) goto done;
       tc_fence_after();
       const uint32_t t_acc = tmem_base + (uint32_t(quarter * 32) << 16) + b * BN;
 
-      if (MODE == GS_STORE_BF16 || MODE == GS_ADD_F32) {
+      // A slab wholly beyond M stages nothing: every staged chunk commits exactly one bulk group, which is what
+      // lets "at most one group pending" protect the buffer about to be rewritten.
+      if (MODE == GS_STORE_BF16) {
 #pragma unroll 1
-        for (int c = 0; c < BN; c += 32) {
+        for (int c = 0; slab_ok && c < BN; c += 64) {
+          uint8_t* buf = my_stg + (n_stores & 1) * STG_BYTES;
+          if (lane == 0) bulk_wait_read<1>();      // the store that last read this buffer has drained
+          __syncwarp();
+          uint32_t r0[32], r1[32];
+          tmem_ld32(t_acc + c, r0);
+          tmem_ld32(t_acc + c + 32, r1);
+          tmem_ld_wait();
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            *stg_chunk(buf, lane, v) = pack8(r0 + 8 * v);
+            *stg_chunk(buf, lane, 4 + v) = pack8(r1 + 8 * v);
+          }
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(&tmC, buf, n0 + c, wrow0);
+            bulk_commit();
+          }
+          ++n_stores;
+        }
+      } else if (MODE == GS_ADD_F32) {
+#pragma unroll 1
+        for (int c = 0; slab_ok && c < BN; c += 32) {
+          uint8_t* buf = my_stg + (n_stores & 1) * STG_BYTES;
+          if (lane == 0) bulk_wait_read<1>();
+          __syncwarp();
           uint32_t r[32];
           tmem_ld32(t_acc + c, r);
           tmem_ld_wait();
-          if (row_ok) {
-            if (MODE == GS_STORE_BF16) {
-              uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(p.out.C) + (size_t)row * p.out.ldc + n0 + c);
 #pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                uint4 o;
-                o.x = pack_bf16(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1]));
-                o.y = pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
-                o.z = pack_bf16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]));
-                o.w = pack_bf16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]));
-                dst[v] = o;
-              }
-            } else {
-              float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out.C) + (size_t)row * p.out.ldc + n0 + c);
-#pragma unroll
-              for (int v = 0; v < 8; ++v) {
-                float4 o = dst[v];
-                o.x += __uint_as_float(r[4 * v + 0]);
-                o.y += __uint_as_float(r[4 * v + 1]);
-                o.z += __uint_as_float(r[4 * v + 2]);
-                o.w += __uint_as_float(r[4 * v + 3]);
-                dst[v] = o;
-              }
-            }
+          for (int v = 0; v < 8; ++v)
+            *stg_chunk(buf, lane, v) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_reduce_add_2d(&tmC, buf, n0 + c, wrow0);
+            bulk_commit();
           }
+          ++n_stores;
         }
       } else if (MODE == GS_SWIGLU) {
 #pragma unroll 1
-        for (int c = 0; c < OUT_N; c += 32) {
-          uint32_t g[32], u[32];
-          tmem_ld32(t_acc + c, g);
-          tmem_ld32(t_acc + OUT_N + c, u);
-          tmem_ld_wait();
-          if (row_ok) {
-            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(p.out.C) + (size_t)row * p.out.ldc + n0 + c);
+        for (int c = 0; slab_ok && c < OUT_N; c += 64) {
+          uint8_t* buf = my_stg + (n_stores & 1) * STG_BYTES;
+          if (lane == 0) bulk_wait_read<1>();
+          __syncwarp();
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              float o[8];
+          for (int hf = 0; hf < 2; ++hf) {
+            uint32_t g[32], u[32];
+            tmem_ld32(t_acc + c + hf * 32, g);
+            tmem_ld32(t_acc + OUT_N + c + hf * 32, u);
+            tmem_ld_wait();
 #pragma unroll
-              for (int e = 0; e < 8; ++e) {
-                const float gv = __uint_as_float(g[8 * v + e]);
-                o[e] = gv / (1.f + __expf(-gv)) * __uint_as_float(u[8 * v + e]);
-              }
-              uint4 w;
-              w.x = pack_bf16(o[0], o[1]);
-              w.y = pack_bf16(o[2], o[3]);
-              w.z = pack_bf16(o[4], o[5]);
-              w.w = pack_bf16(o[6], o[7]);
-              dst[v] = w;
+            for (int e = 0; e < 32; ++e) {
+              // silu(g) * u; the approximate divide (reciprocal + multiply, 2 ulp) has no slow-path branch, so the
+              // 32 elements interleave; the result is rounded to bf16 anyway
+              const float gv = __uint_as_float(g[e]);
+              g[e] = __float_as_uint(__fdividef(gv, 1.f + __expf(-gv)) * __uint_as_float(u[e]));
             }
+#pragma unroll
+            for (int v = 0; v < 4; ++v) *stg_chunk(buf, lane, hf * 4 + v) = pack8(g + 8 * v);
           }
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(&tmC, buf, n0 + c, wrow0);
+            bulk_commit();
+          }
+          ++n_stores;
         }
       } else if (MODE == GS_ARGMAX) {
         const int nxt = (row_ok && p.out.row_next) ? p.out.row_next[row] : -1;
@@ -280,44 +381,55 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const int blk = phys >> 6, off = phys & 63;
 #pragma unroll 1
         for (int hh = 0; hh < BN / 64; ++hh) {
+          const int head = n0 / 64 + hh;
+          const bool is_q = head < p.qkv.Hq;
+          if (!slab_ok) break;
+          uint8_t* buf = my_stg + (n_stores & 1) * STG_BYTES;
+          if (is_q) {
+            if (lane == 0) bulk_wait_read<1>();
+            __syncwarp();
+          }
           uint32_t lo[32], hi[32];
           tmem_ld32(t_acc + hh * 64, lo);
           tmem_ld32(t_acc + hh * 64 + 32, hi);
           tmem_ld_wait();
-          if (!row_ok) continue;
-          const int head = n0 / 64 + hh;
           if (head < p.qkv.Hq + p.qkv.Hkv) {
-            const float4* cs = reinterpret_cast<const float4*>(p.qkv.rope_cs + (size_t)row * 32);
+            if (row_ok) {
+              const float4* cs = reinterpret_cast<const float4*>(p.qkv.rope_cs + (size_t)row * 32);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const float4 c2 = cs[i];   // (cos, sin) of frequencies 2i and 2i+1
-              const float a0 = __uint_as_float(lo[2 * i]), b0 = __uint_as_float(hi[2 * i]);
-              const float a1 = __uint_as_float(lo[2 * i + 1]), b1 = __uint_as_float(hi[2 * i + 1]);
-              lo[2 * i] = __float_as_uint(a0 * c2.x - b0 * c2.y);
-              hi[2 * i] = __float_as_uint(b0 * c2.x + a0 * c2.y);
-              lo[2 * i + 1] = __float_as_uint(a1 * c2.z - b1 * c2.w);
-              hi[2 * i + 1] = __float_as_uint(b1 * c2.z + a1 * c2.w);
+              for (int i = 0; i < 16; ++i) {
+                const float4 c2 = cs[i];   // (cos, sin) of frequencies 2i and 2i+1
+                const float a0 = __uint_as_float(lo[2 * i]), b0 = __uint_as_float(hi[2 * i]);
+                const float a1 = __uint_as_float(lo[2 * i + 1]), b1 = __uint_as_float(hi[2 * i + 1]);
+                lo[2 * i] = __float_as_uint(a0 * c2.x - b0 * c2.y);
+                hi[2 * i] = __float_as_uint(b0 * c2.x + a0 * c2.y);
+                lo[2 * i + 1] = __float_as_uint(a1 * c2.z - b1 * c2.w);
+                hi[2 * i + 1] = __float_as_uint(b1 * c2.z + a1 * c2.w);
+              }
             }
-            bf16* dst = (head < p.qkv.Hq)
-                            ? p.qkv.q_out + (size_t)row * p.qkv.Hq * 64 + head * 64
-                            : p.qkv.k_pool_layer + (((size_t)blk * p.qkv.Hkv + (head - p.qkv.Hq)) * 64 + off) * 64;
-            uint4* d4 = reinterpret_cast<uint4*>(dst);
+            if (is_q) {
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              uint4 o;
-              o.x = pack_bf16(__uint_as_float(lo[8 * v + 0]), __uint_as_float(lo[8 * v + 1]));
-              o.y = pack_bf16(__uint_as_float(lo[8 * v + 2]), __uint_as_float(lo[8 * v + 3]));
-              o.z = pack_bf16(__uint_as_float(lo[8 * v + 4]), __uint_as_float(lo[8 * v + 5]));
-              o.w = pack_bf16(__uint_as_float(lo[8 * v + 6]), __uint_as_float(lo[8 * v + 7]));
-              d4[v] = o;
-              uint4 q;
-              q.x = pack_bf16(__uint_as_float(hi[8 * v + 0]), __uint_as_float(hi[8 * v + 1]));
-              q.y = pack_bf16(__uint_as_float(hi[8 * v + 2]), __uint_as_float(hi[8 * v + 3]));
-              q.z = pack_bf16(__uint_as_float(hi[8 * v + 4]), __uint_as_float(hi[8 * v + 5]));
-              q.w = pack_bf16(__uint_as_float(hi[8 * v + 6]), __uint_as_float(hi[8 * v + 7]));
-              d4[4 + v] = q;
+              for (int v = 0; v < 4; ++v) {
+                *stg_chunk(buf, lane, v) = pack8(lo + 8 * v);
+                *stg_chunk(buf, lane, 4 + v) = pack8(hi + 8 * v);
+              }
+              fence_proxy_async_smem();
+              __syncwarp();
+              if (lane == 0) {
+                tma_store_2d(&tmC, buf, head * 64, wrow0);
+                bulk_commit();
+              }
+              ++n_stores;
+            } else if (row_ok) {
+              uint4* d4 = reinterpret_cast<uint4*>(
+                  p.qkv.k_pool_layer + (((size_t)blk * p.qkv.Hkv + (head - p.qkv.Hq)) * 64 + off) * 64);
+#pragma unroll
+              for (int v = 0; v < 4; ++v) {
+                d4[v] = pack8(lo + 8 * v);
+                d4[4 + v] = pack8(hi + 8 * v);
+              }
             }
-          } else {
+          } else if (row_ok) {
             // V is stored transposed per block: [dim][token]; consecutive lanes hold consecutive tokens
             bf16* dst = p.qkv.v_pool_layer + ((size_t)blk * p.qkv.Hkv + (head - p.qkv.Hq - p.qkv.Hkv)) * 4096 + off;
 #pragma unroll
@@ -332,10 +444,10 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty + b);
     }
+    if (lane == 0) bulk_wait_all();               // staged rows have reached global memory
   }
 
 done:
-  pdl_launch_dependents();
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -346,8 +458,9 @@ done:
 
 // ------------------------------------------------------------------------------------------------
 template <int BN, int MODE>
-static int launch_one(cudaStream_t st, const GemmSm100Args& a, int out_n_per_tile) {
+static int launch_one(cudaStream_t st, const GemmSm100Args& a, int splits) {
   using C = Cfg<BN>;
+  constexpr int OUT_N = (MODE == GS_SWIGLU) ? BN / 2 : BN;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(gemm_sm100_kernel<BN, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) !=
@@ -360,53 +473,75 @@ static int launch_one(cudaStream_t st, const GemmSm100Args& a, int out_n_per_til
   p.K = a.K;
   p.n_cols = (MODE == GS_SWIGLU) ? a.n_out / 2 : a.n_out;
   p.n_up_off = a.n_out / 2;
+  const int k_blocks = a.K / BK;
+  p.splits = splits;
+  p.kb_per_split = (k_blocks + splits - 1) / splits;
   p.out = a.out;
   p.qkv = a.qkv;
   p.status = a.status;
   const int m_tiles = (a.M + BM - 1) / BM;
-  const int total = m_tiles * (p.n_cols / out_n_per_tile);
+  const int total = m_tiles * (p.n_cols / OUT_N) * splits;
   const int grid = total < a.n_sms ? total : a.n_sms;
-  gemm_sm100_kernel<BN, MODE><<<grid, kGemmThreads, C::SMEM_BYTES, st>>>(a.tmA, a.tmB, p);
-  return cudaGetLastError() == cudaSuccess ? 0 : -1;
+  const CUtensorMap& tmB = a.tmB->m[BN == 64 ? 0 : (BN == 128 ? 1 : 2)];
+  return launch_kernel(gemm_sm100_kernel<BN, MODE>, dim3(grid), dim3(kGemmThreads), C::SMEM_BYTES, st, a.pdl, a.tmA, tmB,
+                       a.tmC, p);
 }
 
-// Tile width: fewest (waves x per-tile time), narrow tiles discounted for their lower MMA efficiency.
-static int pick_bn(int mode, int n_cols, int M, int n_sms) {
+// Tile width and K slices: fewest cycles by a simple model.  A k-block of a 128 x BN tile is bound by the
+// ~64 bytes per clock an SM gets from L2 (16 KB of A + 128 BN bytes of B), not by the MMA (2 BN clocks);
+// the epilogue of the last unit of a CTA is exposed.
+static void pick_tile(int mode, int n_cols, int M, int K, int n_sms, int max_splits, int* bn_out, int* splits_out) {
   const int m_tiles = (M + BM - 1) / BM;
+  const int k_blocks = K / BK;
   const int cands[3] = {256, 128, 64};
-  const double eff[3] = {1.0, 0.9, 0.6};
-  int best = (mode == GS_SWIGLU) ? 128 : 64;
   double best_cost = 1e30;
+  *bn_out = (mode == GS_SWIGLU) ? 128 : 64;
+  *splits_out = 1;
   for (int i = 0; i < 3; ++i) {
     const int bn = cands[i];
     const int out_n = (mode == GS_SWIGLU) ? bn / 2 : bn;
-    if (n_cols % out_n || out_n % 64) continue;   // B rows arrive in 64-row TMA boxes
+    if (n_cols % out_n || out_n % 64) continue;
     const long long tiles = (long long)m_tiles * (n_cols / out_n);
-    const long long waves = (tiles + n_sms - 1) / n_sms;
-    const double cost = (double)waves * bn / eff[i];
-    if (cost < best_cost) { best_cost = cost; best = bn; }
+    for (int sp = 1; sp <= max_splits; ++sp) {
+      const int kbs = (k_blocks + sp - 1) / sp;
+      if (sp > 1 && (kbs < 4 || (long long)(sp - 1) * kbs >= k_blocks)) continue;
+      const long long units = tiles * sp;
+      const long long rounds = (units + n_sms - 1) / n_sms;
+      const double per_kb = 256.0 + 2.0 * bn;
+      const double epi = 700.0 + 10.0 * bn;
+      const double cost = (double)rounds * (kbs * per_kb + 300.0) + epi + (sp > 1 ? 200.0 * sp : 0.0);
+      if (cost < best_cost) { best_cost = cost; *bn_out = bn; *splits_out = sp; }
+    }
   }
-  return best;
 }
-
-int gemm_sm100_box_rows(int, int, int, int) { return 64; }
 
 template <int MODE>
 static int launch_mode(cudaStream_t st, const GemmSm100Args& a) {
   const int n_cols = (MODE == GS_SWIGLU) ? a.n_out / 2 : a.n_out;
-  const int bn = pick_bn(MODE, n_cols, a.M, a.n_sms);
+  int bn = 64, splits = 1;
+  pick_tile(MODE, n_cols, a.M, a.K, a.n_sms, (MODE == GS_ADD_F32 && a.max_splits > 1) ? a.max_splits : 1, &bn, &splits);
+  if (a.force_bn) {
+    const int out_n = (MODE == GS_SWIGLU) ? a.force_bn / 2 : a.force_bn;
+    if ((a.force_bn != 64 && a.force_bn != 128 && a.force_bn != 256) || out_n % 64 || n_cols % out_n) return -1;
+    bn = a.force_bn;
+  }
+  if (a.force_splits) {
+    const int kbs = (a.K / BK + a.force_splits - 1) / a.force_splits;
+    if (MODE != GS_ADD_F32 || (a.force_splits - 1) * kbs >= a.K / BK) return -1;
+    splits = a.force_splits;
+  }
   switch (bn) {
-    case 256: return launch_one<256, MODE>(st, a, MODE == GS_SWIGLU ? 128 : 256);
-    case 128: return launch_one<128, MODE>(st, a, MODE == GS_SWIGLU ? 64 : 128);
+    case 256: return launch_one<256, MODE>(st, a, splits);
+    case 128: return launch_one<128, MODE>(st, a, splits);
     default:
-      if (MODE == GS_SWIGLU) return launch_one<128, MODE>(st, a, 64);
-      return launch_one<64, MODE>(st, a, 64);
+      if (MODE == GS_SWIGLU) return launch_one<128, MODE>(st, a, splits);
+      return launch_one<64, MODE>(st, a, splits);
   }
 }
 
 int launch_gemm_sm100(cudaStream_t st, const GemmSm100Args& a) {
   if (a.M <= 0) return 0;
-  if (a.K % BK || a.n_out % 64) return -1;
+  if (a.K % BK || a.n_out % 64 || !a.tmB) return -1;
   switch (a.mode) {
     case GS_STORE_BF16: return launch_mode<GS_STORE_BF16>(st, a);
     case GS_ADD_F32: return launch_mode<GS_ADD_F32>(st, a);

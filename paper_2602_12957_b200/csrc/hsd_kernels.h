@@ -23,8 +23,25 @@ struct KvView {
   int n_slots;
 };
 
-// Launch bookkeeping: counts launches and, when profiling is on, brackets each with CUDA events.
-struct Launcher;
+// One launch path for every kernel: with `pdl` the launch carries the programmatic-stream-serialization
+// attribute, so the kernel may start while its predecessor in the stream drains; such a kernel executes
+// griddepcontrol.wait before it touches anything the predecessor wrote (or anything that is read by it).
+template <typename... KArgs, typename... Args>
+inline int launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
+                         Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...) == cudaSuccess ? 0 : -1;
+}
+
 enum KernelClass {
   KC_SETUP = 0, KC_EMBED, KC_RMSNORM, KC_GEMM_QKV, KC_ROPE_KV, KC_ATTN, KC_ATTN_COMBINE, KC_GEMM_O, KC_GEMM_GATEUP,
   KC_GEMM_DOWN, KC_LMHEAD, KC_ACCEPT, KC_COMMIT, KC_DEBUG, KC_COUNT
@@ -44,15 +61,17 @@ struct SetupArgs {
   float rope_base;
   int head_dim;
 };
+// `pdl` (here and below): launch with programmatic stream serialization; these kernels wait for their
+// predecessor at their first instruction, so the flag only hides launch latency.
 void launch_setup_rows(cudaStream_t st, const SetupArgs& a, const KvView& kv, const RowMeta& rm, int* status,
-                       int* tile_count);
+                       int* tile_count, bool pdl);
 void launch_embed(cudaStream_t st, const RowMeta& rm, const bf16* table, const bf16* embeds, float* x, int T, int d,
-                  const int* status);
+                  const int* status, bool pdl);
 // h[r] = bf16(rmsnorm(x[src]) * gain), src = sel_rows ? sel_rows[r] : r
 void launch_rmsnorm(cudaStream_t st, const float* x, const bf16* gain, bf16* h, int rows, int d, float eps,
-                    const int* sel_rows);
+                    const int* sel_rows, bool pdl);
 // last row of every sequence (prefill's LM-head rows)
-void launch_select_last_rows(cudaStream_t st, const RowMeta& rm, int n_seqs, int* sel_rows);
+void launch_select_last_rows(cudaStream_t st, const RowMeta& rm, int n_seqs, int* sel_rows, bool pdl);
 void launch_rope_kvwrite(cudaStream_t st, const float* qkv, const RowMeta& rm, const KvView& kv, const ModelDims& md,
                          int layer, bf16* q, int T, const int* status);
 void launch_attn_simt(cudaStream_t st, const bf16* q, const RowMeta& rm, const KvView& kv, const ModelDims& md,
@@ -69,13 +88,14 @@ struct AcceptArgs {
   float* row_zmax;
   float* row_zdraft;
 };
-void launch_accept(cudaStream_t st, const AcceptArgs& a, const RowMeta& rm, const int* status);
+void launch_accept(cudaStream_t st, const AcceptArgs& a, const RowMeta& rm, const int* status, bool pdl);
 void launch_first_token(cudaStream_t st, const unsigned long long* row_best, int n_seqs, int* first_token,
-                        const RowMeta& rm, const KvView& kv, const int* status);
+                        const RowMeta& rm, const KvView& kv, const int* status, bool pdl);
 void launch_commit(cudaStream_t st, const KvView& kv, int n_seqs, const int* seq_slots, const int* accept_len,
-                   int* blocks_in_use);
-void launch_clear_best(cudaStream_t st, unsigned long long* row_best, float* zdraft, int rows);
-void launch_unpack_best(cudaStream_t st, const unsigned long long* row_best, int rows, int* argmax, float* zmax);
+                   int* blocks_in_use, bool pdl);
+void launch_clear_best(cudaStream_t st, unsigned long long* row_best, float* zdraft, int rows, bool pdl);
+void launch_unpack_best(cudaStream_t st, const unsigned long long* row_best, int rows, int* argmax, float* zmax,
+                        bool pdl);
 
 // ---- plain SIMT GEMM (hsd_gemm_simt.cu): the debug cross-check and hsd_debug_logits --------------
 enum GemmMode { GM_STORE_BF16 = 0, GM_ADD_F32 = 1, GM_SWIGLU = 2, GM_STORE_F32 = 3, GM_ARGMAX = 4 };
@@ -90,9 +110,15 @@ void launch_gemm_simt(cudaStream_t st, const bf16* A, const bf16* W, int M, int 
                       const GemmOut& out);
 
 // ---- tcgen05 GEMM (hsd_gemm_sm100.cu) ------------------------------------------------------------
-struct TmaFns;   // driver entry points
 // Encode a 2-D bf16 row-major [rows, cols] tensor map with a {64, box_rows} box and 128-byte swizzle.
 int make_tmap_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+// Same for fp32 with a {32, box_rows} box (128-byte rows): the residual stream as a TMA reduce-add target.
+int make_tmap_2d_f32(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
+// The three maps of one weight matrix, box heights 32 / 64 / 128 rows = half a tile of width 64 / 128 / 256.
+struct WeightMaps {
+  CUtensorMap m[3];
+};
+int make_weight_tmaps(WeightMaps* w, const void* base, uint64_t rows, uint64_t cols);
 int make_tmap_3d(CUtensorMap* map, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t stride1_bytes,
                  uint64_t stride2_bytes, uint32_t b0, uint32_t b1, uint32_t b2);
 int tma_init();   // resolves cuTensorMapEncodeTiled; 0 on success
@@ -106,15 +132,20 @@ struct QkvEpilogue {      // fused RoPE + paged KV write (QKV projection)
   int Hq, Hkv;
 };
 struct GemmSm100Args {
-  CUtensorMap tmA, tmB;
+  CUtensorMap tmA;             // activations, box {64, 128}
+  const WeightMaps* tmB;       // weights
+  CUtensorMap tmC;             // output through TMA: bf16 box {64, 32} (store) or fp32 box {32, 32} (reduce-add);
+                               // the q buffer for GS_QKV_ROPE; unused for GS_ARGMAX
   int M, n_out, K, mode;
   GemmOut out;
   QkvEpilogue qkv;
   int* status;
   int n_sms;
+  int max_splits;              // GS_ADD_F32: most K slices per tile (1 = none; slices add in arrival order)
+  bool pdl;                    // launch with programmatic stream serialization
+  int force_bn, force_splits;  // tests: tile width / K slices to use instead of the model's choice (0 = choose)
 };
 enum GemmSm100Mode { GS_STORE_BF16 = 0, GS_ADD_F32 = 1, GS_SWIGLU = 2, GS_ARGMAX = 4, GS_QKV_ROPE = 5 };
 int launch_gemm_sm100(cudaStream_t st, const GemmSm100Args& a);
-int gemm_sm100_box_rows(int mode, int n_out, int M, int n_sms);   // B-operand TMA box height for this problem
 
 }  // namespace hsd

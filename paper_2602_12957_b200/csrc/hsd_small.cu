@@ -16,6 +16,8 @@ const char* kernel_class_name(int kc) {
 // tables); any violation sets the status words, and every kernel that follows an indirection returns early.
 constexpr int kSetupRows = 64;   // rows of one sequence handled by one CTA
 __global__ void setup_rows_kernel(SetupArgs a, KvView kv, RowMeta rm, int* status, int* tile_count) {
+  pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
+  pdl_launch_dependents();
   const int i = blockIdx.x;
   const int tid = threadIdx.x;
   __shared__ int s_red[32];
@@ -108,15 +110,17 @@ __global__ void setup_rows_kernel(SetupArgs a, KvView kv, RowMeta rm, int* statu
 }
 
 void launch_setup_rows(cudaStream_t st, const SetupArgs& a, const KvView& kv, const RowMeta& rm, int* status,
-                       int* tile_count) {
+                       int* tile_count, bool pdl) {
   dim3 grid(a.n_seqs, (a.max_q_len + kSetupRows - 1) / kSetupRows);
-  setup_rows_kernel<<<grid, 256, 0, st>>>(a, kv, rm, status, tile_count);
+  launch_kernel(setup_rows_kernel, grid, dim3(256), 0, st, pdl, a, kv, rm, status, tile_count);
 }
 
 // ------------------------------------------------------------------------------------------------
 // Embedding gather: x[r] = fp32(table[tok]) or fp32(embeds[r]).  One warp per row, 16-byte loads.
 __global__ void embed_kernel(RowMeta rm, const bf16* __restrict__ table, const bf16* __restrict__ embeds,
                              float* __restrict__ x, int T, int d, const int* status) {
+  pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
+  pdl_launch_dependents();
   if (*status) return;
   const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (r >= T) return;
@@ -133,8 +137,8 @@ __global__ void embed_kernel(RowMeta rm, const bf16* __restrict__ table, const b
   }
 }
 void launch_embed(cudaStream_t st, const RowMeta& rm, const bf16* table, const bf16* embeds, float* x, int T, int d,
-                  const int* status) {
-  embed_kernel<<<(T + 7) / 8, 256, 0, st>>>(rm, table, embeds, x, T, d, status);
+                  const int* status, bool pdl) {
+  launch_kernel(embed_kernel, dim3((T + 7) / 8), dim3(256), 0, st, pdl, rm, table, embeds, x, T, d, status);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -143,6 +147,8 @@ void launch_embed(cudaStream_t st, const RowMeta& rm, const bf16* table, const b
 template <int VEC>   // VEC float4 per lane: d = 128 * VEC
 __global__ void rmsnorm_kernel(const float* __restrict__ x, const bf16* __restrict__ gain, bf16* __restrict__ h,
                                int rows, int d, float eps, const int* __restrict__ sel_rows) {
+  pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
+  pdl_launch_dependents();
   const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (r >= rows) return;
   const int lane = threadIdx.x & 31;
@@ -169,39 +175,45 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const bf16* __restri
   }
 }
 void launch_rmsnorm(cudaStream_t st, const float* x, const bf16* gain, bf16* h, int rows, int d, float eps,
-                    const int* sel_rows) {
+                    const int* sel_rows, bool pdl) {
   if (rows <= 0) return;
   dim3 grid((rows + 7) / 8), block(256);
   switch (d / 128) {
-    case 1: rmsnorm_kernel<1><<<grid, block, 0, st>>>(x, gain, h, rows, d, eps, sel_rows); break;
-    case 2: rmsnorm_kernel<2><<<grid, block, 0, st>>>(x, gain, h, rows, d, eps, sel_rows); break;
-    case 4: rmsnorm_kernel<4><<<grid, block, 0, st>>>(x, gain, h, rows, d, eps, sel_rows); break;
-    case 8: rmsnorm_kernel<8><<<grid, block, 0, st>>>(x, gain, h, rows, d, eps, sel_rows); break;
-    case 16: rmsnorm_kernel<16><<<grid, block, 0, st>>>(x, gain, h, rows, d, eps, sel_rows); break;
+    case 1: launch_kernel(rmsnorm_kernel<1>, grid, block, 0, st, pdl, x, gain, h, rows, d, eps, sel_rows); break;
+    case 2: launch_kernel(rmsnorm_kernel<2>, grid, block, 0, st, pdl, x, gain, h, rows, d, eps, sel_rows); break;
+    case 4: launch_kernel(rmsnorm_kernel<4>, grid, block, 0, st, pdl, x, gain, h, rows, d, eps, sel_rows); break;
+    case 8: launch_kernel(rmsnorm_kernel<8>, grid, block, 0, st, pdl, x, gain, h, rows, d, eps, sel_rows); break;
+    case 16: launch_kernel(rmsnorm_kernel<16>, grid, block, 0, st, pdl, x, gain, h, rows, d, eps, sel_rows); break;
     default: break;   // hsd_create rejects other widths
   }
 }
 
 __global__ void select_last_rows_kernel(RowMeta rm, int n_seqs, int* sel_rows) {
+  pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
+  pdl_launch_dependents();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n_seqs) sel_rows[i] = rm.seq_q0[i] + max(rm.seq_n[i], 1) - 1;
 }
-void launch_select_last_rows(cudaStream_t st, const RowMeta& rm, int n_seqs, int* sel_rows) {
-  select_last_rows_kernel<<<(n_seqs + 127) / 128, 128, 0, st>>>(rm, n_seqs, sel_rows);
+void launch_select_last_rows(cudaStream_t st, const RowMeta& rm, int n_seqs, int* sel_rows, bool pdl) {
+  launch_kernel(select_last_rows_kernel, dim3((n_seqs + 127) / 128), dim3(128), 0, st, pdl, rm, n_seqs, sel_rows);
 }
 
 __global__ void clear_best_kernel(unsigned long long* row_best, float* zdraft, int rows) {
+  pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
+  pdl_launch_dependents();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < rows) {
     row_best[i] = 0ull;
     if (zdraft) zdraft[i] = __int_as_float(0x7fc00000);
   }
 }
-void launch_clear_best(cudaStream_t st, unsigned long long* row_best, float* zdraft, int rows) {
-  clear_best_kernel<<<(rows + 255) / 256, 256, 0, st>>>(row_best, zdraft, rows);
+void launch_clear_best(cudaStream_t st, unsigned long long* row_best, float* zdraft, int rows, bool pdl) {
+  launch_kernel(clear_best_kernel, dim3((rows + 255) / 256), dim3(256), 0, st, pdl, row_best, zdraft, rows);
 }
 
 __global__ void unpack_best_kernel(const unsigned long long* row_best, int rows, int* argmax, float* zmax) {
+  pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
+  pdl_launch_dependents();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < rows) {
     const unsigned long long b = row_best[i];
@@ -209,8 +221,9 @@ __global__ void unpack_best_kernel(const unsigned long long* row_best, int rows,
     if (zmax) zmax[i] = key_value(b);
   }
 }
-void launch_unpack_best(cudaStream_t st, const unsigned long long* row_best, int rows, int* argmax, float* zmax) {
-  unpack_best_kernel<<<(rows + 255) / 256, 256, 0, st>>>(row_best, rows, argmax, zmax);
+void launch_unpack_best(cudaStream_t st, const unsigned long long* row_best, int rows, int* argmax, float* zmax,
+                        bool pdl) {
+  launch_kernel(unpack_best_kernel, dim3((rows + 255) / 256), dim3(256), 0, st, pdl, row_best, rows, argmax, zmax);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -326,6 +339,8 @@ void launch_attn_simt(cudaStream_t st, const bf16* q, const RowMeta& rm, const K
 // d_{j+1}.  a = first j < k whose test fails (or k).  Exact mode: argmax == d_{j+1}.  Threshold mode:
 // z[d_{j+1}] - z_max >= log_tau.
 __global__ void accept_kernel(AcceptArgs a, RowMeta rm, const int* status) {
+  pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
+  pdl_launch_dependents();
   if (*status) return;
   const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (i >= a.n_seqs) return;
@@ -363,13 +378,15 @@ __global__ void accept_kernel(AcceptArgs a, RowMeta rm, const int* status) {
     if (a.row_zdraft) a.row_zdraft[q0 + j] = a.zdraft[q0 + j];
   }
 }
-void launch_accept(cudaStream_t st, const AcceptArgs& a, const RowMeta& rm, const int* status) {
-  accept_kernel<<<(a.n_seqs + 3) / 4, 128, 0, st>>>(a, rm, status);
+void launch_accept(cudaStream_t st, const AcceptArgs& a, const RowMeta& rm, const int* status, bool pdl) {
+  launch_kernel(accept_kernel, dim3((a.n_seqs + 3) / 4), dim3(128), 0, st, pdl, a, rm, status);
 }
 
 // Prefill epilogue: first pending token per sequence, and seq_lens += rows.
 __global__ void first_token_kernel(const unsigned long long* row_best, int n_seqs, int* first_token, RowMeta rm,
                                    KvView kv, const int* status) {
+  pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
+  pdl_launch_dependents();
   if (*status) return;
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_seqs) return;
@@ -377,13 +394,16 @@ __global__ void first_token_kernel(const unsigned long long* row_best, int n_seq
   kv.seq_lens[rm.seq_slot[i]] = rm.seq_len[i] + rm.seq_n[i];
 }
 void launch_first_token(cudaStream_t st, const unsigned long long* row_best, int n_seqs, int* first_token,
-                        const RowMeta& rm, const KvView& kv, const int* status) {
-  first_token_kernel<<<(n_seqs + 127) / 128, 128, 0, st>>>(row_best, n_seqs, first_token, rm, kv, status);
+                        const RowMeta& rm, const KvView& kv, const int* status, bool pdl) {
+  launch_kernel(first_token_kernel, dim3((n_seqs + 127) / 128), dim3(128), 0, st, pdl, row_best, n_seqs, first_token, rm,
+                kv, status);
 }
 
 // ------------------------------------------------------------------------------------------------
 // KV commit / rollback: the pending row and the accepted rows stay, the rest is dead and gets overwritten.
 __global__ void commit_kernel(KvView kv, int n_seqs, const int* seq_slots, const int* accept_len, int* blocks_in_use) {
+  pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
+  pdl_launch_dependents();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_seqs) return;
   const int slot = seq_slots ? seq_slots[i] : i;
@@ -395,8 +415,9 @@ __global__ void commit_kernel(KvView kv, int n_seqs, const int* seq_slots, const
   if (blocks_in_use) blocks_in_use[i] = (L + HSD_KV_BLOCK - 1) / HSD_KV_BLOCK;
 }
 void launch_commit(cudaStream_t st, const KvView& kv, int n_seqs, const int* seq_slots, const int* accept_len,
-                   int* blocks_in_use) {
-  commit_kernel<<<(n_seqs + 127) / 128, 128, 0, st>>>(kv, n_seqs, seq_slots, accept_len, blocks_in_use);
+                   int* blocks_in_use, bool pdl) {
+  launch_kernel(commit_kernel, dim3((n_seqs + 127) / 128), dim3(128), 0, st, pdl, kv, n_seqs, seq_slots, accept_len,
+                blocks_in_use);
 }
 
 }  // namespace hsd

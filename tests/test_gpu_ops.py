@@ -101,3 +101,47 @@ def test_lm_head_argmax_matches_float64(models, flags, rows):
     assert np.all(z[np.arange(rows), am] >= srt[:, -1] - 5e-3)
     assert np.isnan(zd[0])
     assert np.abs(zd[1:] - z[np.arange(1, rows), nxt[1:]]).max() < 2e-3 if rows > 1 else True
+
+
+@pytest.mark.parametrize("shape", [(513, 8192, 128), (1323, 2048, 192), (513, 2048, 1024), (1323, 1024, 4096)])
+@pytest.mark.parametrize("mode", [0, 1, 2])
+def test_linear_every_tile_width_and_k_slicing(models, mode, shape):
+    """Every tile width (64/128/256) and, for the residual-add epilogue, 1 to 8 slices of K, on shapes whose last
+    row tile is mostly beyond M and whose K loop is short (the epilogue, not the main loop, sets the pace, so
+    several staged stores are in flight per warp).  Repeated, because a staging-buffer race shows up only sometimes."""
+    import torch
+    from paper_2602_12957_b200 import binding as B
+    model = models[0]
+    M, N, K = shape
+    rng = np.random.default_rng(M + N + K)
+    A = I.bf16_round(np.abs(rng.standard_normal((M, K), dtype=np.float32)) + 0.1)     # strictly positive: a zero
+    W = I.bf16_round(np.abs(rng.standard_normal((N, K), dtype=np.float32)) * 0.05 + 0.01)   # output is always wrong
+    dev = model.device
+    tA = torch.from_numpy(A).to(dev, torch.bfloat16)
+    tW = torch.from_numpy(W).to(dev, torch.bfloat16)
+    ref = A.astype(np.float64) @ W.astype(np.float64).T
+    if mode == 2:
+        g, u = ref[:, :N // 2], ref[:, N // 2:]
+        ref = g / (1.0 + np.exp(-g)) * u
+    st = torch.cuda.current_stream().cuda_stream
+    try:
+        for bn in (64, 128, 256):
+            if mode == 2 and bn == 64:
+                continue
+            for sp in ((1, 2, 3, 4, 8) if mode == 1 else (0,)):
+                if mode == 1 and sp > 1 and (K // 64 + sp - 1) // sp * (sp - 1) >= K // 64:
+                    continue
+                B.check(B.hsd_debug_set_gemm_tile(model.ctx, bn, sp))
+                for trial in range(3):
+                    if mode == 1:
+                        C = torch.full((M, N), 7.0, dtype=torch.float32, device=dev)
+                    else:
+                        C = torch.full((M, ref.shape[1]), 7.0, dtype=torch.bfloat16, device=dev)
+                    B.check(B.hsd_op_linear(model.ctx, tA, tW, C, M, N, K, mode, st))
+                    torch.cuda.synchronize()
+                    got = C.float().cpu().numpy().astype(np.float64) - (7.0 if mode == 1 else 0.0)
+                    tol = (1e-4 if mode == 1 else 2.0 ** -7) * np.abs(ref).max() + 1e-3
+                    err = np.abs(got - ref).max()
+                    assert err <= tol, f"shape {shape} mode {mode} tile {bn} slices {sp} trial {trial}: max err {err:.3e}"
+    finally:
+        B.hsd_debug_set_gemm_tile(model.ctx, 0, 0)

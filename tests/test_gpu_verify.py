@@ -46,12 +46,13 @@ def test_one_verify_call_equals_sequential_single_token_steps_on_gpu():
     """The library against itself: k+1 plain decode steps (empty drafts, commit each) must reproduce the rows of
     one verify call over the tokens they emitted — same kernels, same K/V rows, same tile boundaries."""
     import torch
+    from paper_2602_12957_b200 import binding as B
     from paper_2602_12957_b200 import runtime as R
     cfg = I.small_decoder(2, 8192)
     wl = I.region_workload(seed=91, n_regions=3, prefix_lo=60, prefix_hi=200, draft_mean=40, draft_lo=20, draft_hi=70,
                            cfg=cfg)
     weights = I.make_weights(cfg, 5)
-    model = R.DeviceModel(cfg, weights, 0)
+    model = R.DeviceModel(cfg, weights, B.HSD_FLAG_DETERMINISTIC)   # bit-equality needs a fixed summation order
     S = len(wl.seqs)
     k = 20
     kv = R.KvCache(model, [s.prefix_len + k + 2 for s in wl.seqs], seed=1)
