@@ -213,6 +213,11 @@ HSD_API int hsd_op_linear(hsd_ctx *ctx, const void *A, const void *W, void *C, i
  * problem does not allow makes hsd_op_linear return HSD_ERR_CUDA.  Lets the parity tests reach every tile shape. */
 HSD_API int hsd_debug_set_gemm_tile(hsd_ctx *ctx, int tile_n, int k_slices);
 
+/* Test-only: the attention launch cuts the KV range of every query tile into slices so that it has about
+ * `target_items` work items, none shorter than `min_kv_tiles` 64-token KV tiles (0 = the library's defaults).
+ * Results do not depend on the setting beyond fp32 summation order; tests use it to force many or no slices. */
+HSD_API int hsd_debug_set_attn_plan(hsd_ctx *ctx, int target_items, int min_kv_tiles);
+
 /* hsd_op_lm_head_argmax: the fused LM head on its own (Eq. 10 per row): for `rows` already-normalised hidden rows
  * h (dev bf16 [rows, d_model]) compute z = h W_lm^T tile by tile and keep only, per row, the argmax (lowest id on
  * ties), its logit, and the logit of next_tokens[row] (dev int32 [rows] or NULL; entries < 0 give NaN).  Logits

@@ -28,7 +28,7 @@ EXPORTS = [
     "hsd_status_string", "hsd_create", "hsd_destroy", "hsd_workspace_bytes", "hsd_prefill", "hsd_verify_regions",
     "hsd_verify_page", "hsd_kv_commit", "hsd_device_status", "hsd_last_cuda_error", "hsd_launch_count",
     "hsd_profile_enable", "hsd_profile_read", "hsd_debug_logits", "hsd_debug_buffer", "hsd_op_linear",
-    "hsd_op_lm_head_argmax", "hsd_op_lm_head_argmax_noalloc", "hsd_debug_set_gemm_tile",
+    "hsd_op_lm_head_argmax", "hsd_op_lm_head_argmax_noalloc", "hsd_debug_set_gemm_tile", "hsd_debug_set_attn_plan",
 ]
 
 
@@ -83,6 +83,7 @@ def _load():
     lib.hsd_debug_logits.argtypes = [vp, vp, i, i, vp, vp]
     lib.hsd_debug_buffer.argtypes = [vp, vp, i, i, C.c_char_p, C.POINTER(vp), C.POINTER(sz)]
     lib.hsd_debug_set_gemm_tile.argtypes = [vp, i, i]
+    lib.hsd_debug_set_attn_plan.argtypes = [vp, i, i]
     lib.hsd_op_linear.argtypes = [vp, vp, vp, vp, i, i, i, i, vp]
     lib.hsd_op_lm_head_argmax.argtypes = [vp, vp, i, vp, vp, sz, vp, vp, vp, vp]
     lib.hsd_op_lm_head_argmax_noalloc.argtypes = [vp, vp, i, vp, vp, vp, vp, vp]
@@ -230,6 +231,10 @@ def hsd_debug_buffer(ctx, workspace, total_q, n_seqs, name: str):
 
 def hsd_debug_set_gemm_tile(ctx, tile_n: int, k_slices: int) -> int:
     return _lib.hsd_debug_set_gemm_tile(ctx, tile_n, k_slices)
+
+
+def hsd_debug_set_attn_plan(ctx, target_items: int, min_kv_tiles: int) -> int:
+    return _lib.hsd_debug_set_attn_plan(ctx, target_items, min_kv_tiles)
 
 
 def hsd_op_linear(ctx, A, W, Cout, M, n_out, K, mode, stream) -> int:

@@ -10,12 +10,6 @@
 
 using namespace hsd;
 
-namespace hsd {
-int launch_attn_sm100(cudaStream_t st, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
-                      const RowMeta& rm, const KvView& kv, const ModelDims& md, int layer, bf16* out, int n_seqs,
-                      int max_tiles, const int* tile_count, int* status, float* split_ws, bool pdl);
-}
-
 struct ProfEvent {
   int kc;
   cudaEvent_t a, b;
@@ -31,6 +25,7 @@ struct hsd_ctx {
   int max_splits;     // K slices the residual-add projections may use (1 with HSD_FLAG_DETERMINISTIC)
   bool pdl;           // kernels are launched with programmatic stream serialization
   int force_bn, force_splits;   // hsd_debug_set_gemm_tile
+  int attn_target_items, attn_min_chunk;   // attention plan: items aimed at per launch, fewest KV tiles per slice
   int n_sms;
   int device;
   bool simt;
@@ -47,7 +42,8 @@ struct hsd_ctx {
 namespace {
 
 struct Ws {
-  int* status;        // 16 ints; [4] = attention q-tile count
+  int* status;        // 16 ints; [4] = attention q-tile count, [5] = attention items
+  AttnPlan plan;
   RowMeta rm;
   int* sel_rows;
   int* cu_one;        // {0, n} offsets of a single-sequence call
@@ -65,11 +61,11 @@ struct Ws {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// Split-KV partial results: per (q-tile row, q head, split) an fp32 accumulator row plus (max, sum).
-constexpr int kMaxSplits = 16;
+// Split-KV partial results: per (query row, q head, slice) an fp32 accumulator row plus (max, sum).
 inline size_t split_ws_floats(const ModelDims& md, int T) {
-  return (size_t)T * md.Hq * kMaxSplits * (md.D + 2);
+  return (size_t)T * md.Hq * kAttnMaxSplits * (md.D + 2);
 }
+inline int attn_max_tiles(const ModelDims& md, int T, int S) { return T / (128 / md.group) + S; }
 
 Ws carve(const hsd_ctx* c, void* base, int T, int S) {
   const ModelDims& md = c->md;
@@ -104,6 +100,15 @@ Ws carve(const hsd_ctx* c, void* base, int T, int S) {
   w.row_best = static_cast<unsigned long long*>(take(sizeof(unsigned long long) * T));
   w.zdraft = static_cast<float*>(take(sizeof(float) * T));
   w.split_ws = c->simt ? nullptr : static_cast<float*>(take(sizeof(float) * split_ws_floats(md, T)));
+  {
+    const int mt = attn_max_tiles(md, T, S);
+    w.plan.items = static_cast<int4*>(take(sizeof(int4) * 2 * (size_t)mt * kAttnMaxSplits));
+    w.plan.tile_seq = static_cast<int*>(take(sizeof(int) * mt));
+    w.plan.tile_nkv = static_cast<int*>(take(sizeof(int) * mt));
+    w.plan.counters = static_cast<int*>(take(sizeof(int) * (size_t)mt * md.Hkv));
+    w.plan.n_items = w.status ? w.status + 5 : nullptr;
+    w.plan.n_kv_heads = md.Hkv;
+  }
   w.bytes = off;
   return w;
 }
@@ -215,7 +220,12 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
   }
 
   CUtensorMap tm_h, tm_attn, tm_act, tm_q, tm_k, tm_v, tm_x_add, tm_q_st, tm_act_st;
-  const int max_tiles = T / tokens_per_tile + a.n_seqs;
+  if (!c->attn_simt) {
+    Scope s(c, st, KC_SETUP);
+    // items per launch: a few per CTA slot (two CTAs per SM), at least attn_min_chunk KV tiles each
+    launch_attn_plan(st, w.rm, w.plan, a.n_seqs, tokens_per_tile, c->attn_target_items / md.Hkv + 1, c->attn_min_chunk,
+                     w.status + 4, w.status, c->pdl);
+  }
   if (!c->simt) {
     if (make_tmap_2d(&tm_h, w.h, T, md.d, 128) || make_tmap_2d(&tm_attn, w.attn, T, md.Hq * md.D, 128) ||
         make_tmap_2d(&tm_act, w.act, T, md.ffn, 128))
@@ -279,8 +289,8 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         Scope s(c, st, KC_ATTN);
         if (c->attn_simt) {
           launch_attn_simt(st, w.q, w.rm, kv, md, l, w.attn, T, w.status);
-        } else if (launch_attn_sm100(st, tm_q, tm_k, tm_v, w.rm, kv, md, l, w.attn, a.n_seqs, max_tiles, w.status + 4,
-                                     w.status, w.split_ws, c->pdl)) {
+        } else if (launch_attn_sm100(st, tm_q, tm_k, tm_v, w.plan, kv, md, l, w.attn, c->n_sms, w.status, w.split_ws,
+                                     c->pdl)) {
           return fail_cuda(c);
         }
       }
@@ -470,6 +480,8 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
   c->max_splits = (cfg->flags & HSD_FLAG_DETERMINISTIC) ? 1 : 8;
   c->pdl = (cfg->flags & HSD_FLAG_NO_PDL) == 0;
   c->force_bn = c->force_splits = 0;
+  c->attn_target_items = 5 * c->n_sms;
+  c->attn_min_chunk = 4;
   c->last_cuda_error = 0;
   c->launches = 0;
   c->profiling = false;
@@ -755,6 +767,13 @@ int hsd_debug_set_gemm_tile(hsd_ctx* c, int tile_n, int k_slices) {
   if (!c || tile_n < 0 || k_slices < 0) return HSD_ERR_INVALID_ARG;
   c->force_bn = tile_n;
   c->force_splits = k_slices;
+  return HSD_OK;
+}
+
+int hsd_debug_set_attn_plan(hsd_ctx* c, int target_items, int min_kv_tiles) {
+  if (!c || target_items < 0 || min_kv_tiles < 0) return HSD_ERR_INVALID_ARG;
+  c->attn_target_items = target_items ? target_items : 5 * c->n_sms;
+  c->attn_min_chunk = min_kv_tiles ? min_kv_tiles : 4;
   return HSD_OK;
 }
 

@@ -97,6 +97,23 @@ void launch_clear_best(cudaStream_t st, unsigned long long* row_best, float* zdr
 void launch_unpack_best(cudaStream_t st, const unsigned long long* row_best, int rows, int* argmax, float* zmax,
                         bool pdl);
 
+// ---- attention plan (hsd_attn_sm100.cu): made once per step on the device, read by every layer's launch ----
+constexpr int kAttnMaxSplits = 16;     // most KV slices one q-tile is cut into
+struct AttnPlan {
+  int4* items;      // two int4 per (q-tile, slice) item: {first packed row, position of the first token, tokens, KV slot},
+                    // {first | (last + 1) << 16 KV tile, slice | slices << 16, q-tile, 0}
+  int* n_items;
+  int* tile_seq;    // [max_tiles] sequence of a q-tile
+  int* tile_nkv;    // [max_tiles] KV tiles it can see
+  int* counters;    // [max_tiles, n_kv_heads] slices that have delivered their partial
+  int n_kv_heads;
+};
+void launch_attn_plan(cudaStream_t st, const RowMeta& rm, const AttnPlan& pl, int n_seqs, int tokens_per_tile,
+                      int target_items, int min_chunk, const int* tile_count, const int* status, bool pdl);
+int launch_attn_sm100(cudaStream_t st, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
+                      const AttnPlan& plan, const KvView& kv, const ModelDims& md, int layer, bf16* out, int n_sms,
+                      int* status, float* split_ws, bool pdl);
+
 // ---- plain SIMT GEMM (hsd_gemm_simt.cu): the debug cross-check and hsd_debug_logits --------------
 enum GemmMode { GM_STORE_BF16 = 0, GM_ADD_F32 = 1, GM_SWIGLU = 2, GM_STORE_F32 = 3, GM_ARGMAX = 4 };
 struct GemmOut {

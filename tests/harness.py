@@ -87,7 +87,7 @@ def compare_sequence(tag, res: O.VerifyResult, draft, g_accept, g_emit, g_n_emit
 # ------------------------------------------------------------------------------------------------ GPU side
 def gpu_regions(wl: I.Workload, weights, pendings: Dict[int, int], drafts: Dict[int, np.ndarray], flags: int = 0,
                 seed: int = 0, poison: bool = True, order: Optional[List[int]] = None, log_tau: float = 0.0,
-                commit: bool = False, model=None):
+                commit: bool = False, model=None, attn_plan=None):
     """Run prefill + one verify step of the listed sequences through the C-ABI.  Returns numpy outputs per
     sequence index plus the engine (for follow-up calls)."""
     import torch
@@ -97,6 +97,9 @@ def gpu_regions(wl: I.Workload, weights, pendings: Dict[int, int], drafts: Dict[
     own_model = model is None
     if own_model:
         model = R.DeviceModel(wl.cfg, weights, flags)
+    if attn_plan is not None:
+        from paper_2602_12957_b200 import binding as B
+        B.check(B.hsd_debug_set_attn_plan(model.ctx, attn_plan[0], attn_plan[1]))
     caps = [s.prefix_len + s.draft_len + 1 + 64 for s in seqs]
     kv = R.KvCache(model, caps, seed=seed, poison=poison)
     total_prefix = sum(s.prefix_len for s in seqs)

@@ -9,11 +9,11 @@ from . import harness as H
 pytestmark = pytest.mark.gpu
 
 
-def run_region_parity(wl, flags=0, dtype=np.float64, which=None):
+def run_region_parity(wl, flags=0, dtype=np.float64, which=None, attn_plan=None):
     weights = I.make_weights(wl.cfg, wl.seed)
     orc = H.oracle_regions(wl, weights, dtype, which)
     per, eng, _ = H.gpu_regions(wl, weights, {i: o.pending for i, o in orc.items()},
-                                {i: o.draft for i, o in orc.items()}, flags)
+                                {i: o.draft for i, o in orc.items()}, flags, attn_plan=attn_plan)
     stats = {}
     for i, o in orc.items():
         g = per[i]
@@ -39,6 +39,17 @@ def test_small_decoder_regions_match_oracle(flags):
                            cfg=I.small_decoder(2, 8192), name="small_regions")
     stats, orc, per, _ = run_region_parity(wl, flags)
     print("small", flags, stats, [(len(o.draft), o.res.accept_len) for o in orc.values()])
+    assert stats["max_dz"] < H.LOGIT_TOL
+
+
+@pytest.mark.parametrize("plan", [(1 << 20, 1), (1, 1 << 20)], ids=["sixteen_slices", "no_slices"])
+def test_attention_kv_slicing_does_not_change_the_result(plan):
+    """The KV range of a query tile cut into as many slices as allowed (partials combined by the last slice to
+    finish) and not cut at all: both within the oracle's tolerance, on contexts of 2 to 9 KV tiles."""
+    wl = I.region_workload(seed=78, n_regions=4, prefix_lo=100, prefix_hi=520, draft_mean=50, draft_lo=8, draft_hi=150,
+                           cfg=I.small_decoder(2, 8192), name="small_regions_slicing")
+    stats, orc, per, _ = run_region_parity(wl, 0, attn_plan=plan)
+    print("slicing", plan, stats)
     assert stats["max_dz"] < H.LOGIT_TOL
 
 
