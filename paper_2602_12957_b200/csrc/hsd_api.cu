@@ -61,11 +61,11 @@ struct Ws {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// Split-KV partial results: per (query row, q head, slice) an fp32 accumulator row plus (max, sum).
-inline size_t split_ws_floats(const ModelDims& md, int T) {
-  return (size_t)T * md.Hq * kAttnMaxSplits * (md.D + 2);
-}
 inline int attn_max_tiles(const ModelDims& md, int T, int S) { return T / (128 / md.group) + S; }
+// Split-KV partial results: per (q-tile, kv head, slice) 128 rows of an fp32 accumulator row plus (max, sum).
+inline size_t split_ws_floats(const ModelDims& md, int T, int S) {
+  return (size_t)attn_max_tiles(md, T, S) * md.Hkv * kAttnMaxSplits * (md.D + 2) * 128;
+}
 
 Ws carve(const hsd_ctx* c, void* base, int T, int S) {
   const ModelDims& md = c->md;
@@ -99,7 +99,7 @@ Ws carve(const hsd_ctx* c, void* base, int T, int S) {
   w.qkv_f32 = c->simt ? static_cast<float*>(take(sizeof(float) * (size_t)T * md.qkv_out)) : nullptr;
   w.row_best = static_cast<unsigned long long*>(take(sizeof(unsigned long long) * T));
   w.zdraft = static_cast<float*>(take(sizeof(float) * T));
-  w.split_ws = c->simt ? nullptr : static_cast<float*>(take(sizeof(float) * split_ws_floats(md, T)));
+  w.split_ws = c->simt ? nullptr : static_cast<float*>(take(sizeof(float) * split_ws_floats(md, T, S)));
   {
     const int mt = attn_max_tiles(md, T, S);
     w.plan.items = static_cast<int4*>(take(sizeof(int4) * 2 * (size_t)mt * kAttnMaxSplits));
@@ -480,8 +480,8 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
   c->max_splits = (cfg->flags & HSD_FLAG_DETERMINISTIC) ? 1 : 8;
   c->pdl = (cfg->flags & HSD_FLAG_NO_PDL) == 0;
   c->force_bn = c->force_splits = 0;
-  c->attn_target_items = 5 * c->n_sms;
-  c->attn_min_chunk = 4;
+  c->attn_target_items = 2 * c->n_sms;   // one item per CTA slot: slicing costs a partial hand-over per slice
+  c->attn_min_chunk = 16;
   c->last_cuda_error = 0;
   c->launches = 0;
   c->profiling = false;
@@ -772,8 +772,8 @@ int hsd_debug_set_gemm_tile(hsd_ctx* c, int tile_n, int k_slices) {
 
 int hsd_debug_set_attn_plan(hsd_ctx* c, int target_items, int min_kv_tiles) {
   if (!c || target_items < 0 || min_kv_tiles < 0) return HSD_ERR_INVALID_ARG;
-  c->attn_target_items = target_items ? target_items : 5 * c->n_sms;
-  c->attn_min_chunk = min_kv_tiles ? min_kv_tiles : 4;
+  c->attn_target_items = target_items ? target_items : 2 * c->n_sms;
+  c->attn_min_chunk = min_kv_tiles ? min_kv_tiles : 16;
   return HSD_OK;
 }
 

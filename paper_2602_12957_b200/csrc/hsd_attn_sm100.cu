@@ -13,34 +13,30 @@
 // the workspace and the last slice to finish combines them in slice order, so the result does not depend
 // on which CTA ran what.
 //
-// Persistent CTAs, two per SM, walk the item list.  Warp roles: warps 0..3 = softmax (one TMEM lane quarter
-// each, one thread per q row, no shuffles), warp 4 = TMA producer, warp 5 = MMA issuer + TMEM owner.  The
-// second warpgroup hands most of its registers to the softmax warpgroup (setmaxnreg), which keeps a whole
-// tile of scores and probabilities in registers.
-// Per KV tile: S = Q K^T (TMEM, double-buffered) -> softmax in registers -> P (bf16, shared memory,
-// 128B-swizzled, double-buffered) -> O += P V accumulated in TMEM.  The softmax keeps a reference maximum
-// per row that is raised only when a tile's maximum exceeds it by more than 2^8; O and the running sum are
-// rescaled (in TMEM, by the row's own thread) only then, so most tiles cost one exp per score and nothing
-// else.  The final O / sum is exact whatever the reference was.
+// Persistent CTAs, two per SM, walk the item list.  Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer +
+// TMEM owner, warps 2..5 = softmax (one TMEM lane quarter each, one thread per q row, no shuffles).
+// Per KV tile: S = Q K^T (TMEM) -> online softmax in registers -> P (bf16, shared memory, 128B-swizzled) ->
+// PV = P V (TMEM) -> accumulated into registers with the running-max rescale.  S, P and PV are double-buffered
+// so the tensor pipe works on tile j+1 while the softmax warps are on tile j; two CTAs per SM interleave
+// further.  Every wait is a bounded mbarrier wait, so one that gives up takes the whole CTA to the common exit.
 #include "hsd_kernels.h"
 
 namespace hsd {
 
-constexpr int kAttnThreads = 256;                  // warps 0-3 softmax, 4 TMA producer, 5 MMA issuer, 6-7 idle
+constexpr int kAttnThreads = 192;
 constexpr int KV_STAGES = 3;
 constexpr int Q_BYTES = 128 * 128;
 constexpr int KV_TILE_BYTES = 64 * 128;            // one K tile or one V^T tile
 constexpr int P_BYTES = 128 * 128;
 constexpr int ATTN_SMEM = Q_BYTES + KV_STAGES * 2 * KV_TILE_BYTES + 2 * P_BYTES + 1024 + 256;
-constexpr int ATTN_TMEM_COLS = 256;                // S0 S1 O (64 fp32 columns each) + 64 spare (power of two)
-constexpr float kRescaleLog2 = 8.f;                // raise the reference maximum only beyond 2^8
+constexpr int ATTN_TMEM_COLS = 256;                // S0 S1 PV0 PV1, 64 fp32 columns each
 
 struct AttnParams {
   AttnPlan plan;
   const int* block_table;
   int max_blocks, n_blocks, Hq, Hkv, group, layer;
   bf16* out;            // [T, Hq*64]
-  float* split_ws;      // partials of sliced items: [row][q head][slice][2 + 64]
+  float* split_ws;      // partials of sliced items: [q-tile][kv head][slice][2 + 64][128 rows]
   int* status;
 };
 
@@ -54,24 +50,16 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
   return y;
 }
-// registers -> TMEM: 32 lanes x 32 consecutive fp32 columns (the mirror of tmem_ld32)
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
-        "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
-        "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
+// Barrier among whole warps on an mbarrier whose count is the number of warps: every lane's earlier shared-memory
+// writes are visible to every participant afterwards.  `phase` counts this thread's uses of `bar`.
+__device__ __forceinline__ bool warps_sync(uint64_t* bar, uint32_t& phase, int lane, volatile int* abort_flag,
+                                           int* status, int where) {
+  __syncwarp();
+  if (lane == 0) mbar_arrive(bar);
+  const bool ok = mbar_wait(bar, phase & 1u, abort_flag, status, where);
+  ++phase;
+  return __all_sync(0xffffffffu, ok);
 }
-__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void softmax_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
-template <int N>
-__device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 
 // ------------------------------------------------------------------------------------------------
 // Plan: one CTA.  For every q-tile the KV tiles it can see and into how many slices that range is cut, then
@@ -145,14 +133,14 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   uint64_t* bars = reinterpret_cast<uint64_t*>(sP + 2 * P_BYTES);
   uint64_t* q_full = bars;                 // Q tile landed                       (one phase per item)
   uint64_t* q_empty = bars + 1;            // every S MMA of the item has read Q   (one phase per item)
-  uint64_t* o_empty = bars + 2;            // softmax warps have read the final O  (one phase per item, 4 arrivals)
-  uint64_t* kv_full = bars + 3;
+  uint64_t* kv_full = bars + 2;
   uint64_t* kv_empty = kv_full + KV_STAGES;
   uint64_t* s_full = kv_empty + KV_STAGES;
   uint64_t* s_empty = s_full + 2;
   uint64_t* p_full = s_empty + 2;
-  uint64_t* pv_done = p_full + 2;          // the PV MMA that read P[b] has completed
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pv_done + 2);
+  uint64_t* pv_full = p_full + 2;
+  uint64_t* group_bar = pv_full + 2;       // the four softmax warps (slice hand-over)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(group_bar + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* s_flag = abort_flag + 1;   // combine: "this CTA ran the last slice to finish"
 
@@ -160,7 +148,6 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
     mbar_init(q_empty, 1);
-    mbar_init(o_empty, 4);
     for (int s = 0; s < KV_STAGES; ++s) {
       mbar_init(kv_full + s, 1);
       mbar_init(kv_empty + s, 1);
@@ -168,16 +155,17 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     for (int b = 0; b < 2; ++b) {
       mbar_init(s_full + b, 1);
       mbar_init(s_empty + b, 4);
-      mbar_init(p_full + b, 4);
-      mbar_init(pv_done + b, 1);
+      mbar_init(p_full + b, 128);
+      mbar_init(pv_full + b, 1);
     }
+    mbar_init(group_bar, 4);
     *abort_flag = 0;
     fence_mbar_init();
     tma_prefetch_desc(&tmQ);
     tma_prefetch_desc(&tmK);
     tma_prefetch_desc(&tmV);
   }
-  if (warp == 5) {
+  if (warp == 1) {
     tmem_alloc(tmem_slot, ATTN_TMEM_COLS);
     tmem_relinquish();
   }
@@ -191,96 +179,89 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
   const int total = (*p.status) ? 0 : *p.plan.n_items * p.Hkv;
 
-  // Global tile counter g (all items of this CTA): S / P buffer = g & 1, KV stage = g % KV_STAGES, and every
-  // barrier's parity follows from how often g has used it; n counts items (Q / O hand-over barriers).
-  // 128 x (48 + 200) registers <= half the SM's register file; each role's code follows its own setmaxnreg.
-  if (warp >= 4) {
-    reg_dealloc<48>();
-    if (warp == 4) {
-      if (lane == 0) {
-        uint32_t g = 0;
-        int n = 0;
-        for (int w = blockIdx.x; w < total; w += gridDim.x, ++n) {
-          const int4 ia = p.plan.items[2 * (w / p.Hkv)], ib = p.plan.items[2 * (w / p.Hkv) + 1];
-          const int kvh = w % p.Hkv;
-          const int kt_lo = ib.x & 0xffff, kt_hi = ib.x >> 16;
-          const int* bt = p.block_table + (size_t)ia.w * p.max_blocks;
-          int phys = bt[kt_lo];
-          if (!mbar_wait(q_empty, (n & 1) ^ 1u, abort_flag, p.status, 400)) goto done;
-          mbar_expect_tx(q_full, Q_BYTES);
-          tma_load_3d(sQ, &tmQ, q_full, 0, kvh * p.group, ia.x);
-          for (int j = kt_lo; j < kt_hi; ++j, ++g) {
-            const int phys_next = (j + 1 < kt_hi) ? bt[j + 1] : 0;    // block-table entry of the next tile, ahead of need
-            const int st = g % KV_STAGES;
-            if (!mbar_wait(kv_empty + st, ((g / KV_STAGES) & 1) ^ 1u, abort_flag, p.status, 401)) goto done;
-            const int row = (((p.layer * p.n_blocks) + phys) * p.Hkv + kvh) * 64;
-            uint8_t* k_dst = sKV + st * 2 * KV_TILE_BYTES;
-            mbar_expect_tx(kv_full + st, 2 * KV_TILE_BYTES);
-            tma_load_2d(k_dst, &tmK, kv_full + st, 0, row);
-            tma_load_2d(k_dst + KV_TILE_BYTES, &tmV, kv_full + st, 0, row);
-            phys = phys_next;
-          }
+  // Global tile counter g (all items of this CTA): S / P / PV buffer = g & 1, KV stage = g % KV_STAGES, and every
+  // barrier's parity follows from how often g has used it; n counts items (Q hand-over barriers).
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t g = 0;
+      int n = 0;
+      for (int w = blockIdx.x; w < total; w += gridDim.x, ++n) {
+        const int4 ia = p.plan.items[2 * (w / p.Hkv)], ib = p.plan.items[2 * (w / p.Hkv) + 1];
+        const int kvh = w % p.Hkv;
+        const int kt_lo = ib.x & 0xffff, kt_hi = ib.x >> 16;
+        const int* bt = p.block_table + (size_t)ia.w * p.max_blocks;
+        int phys = bt[kt_lo];
+        if (!mbar_wait(q_empty, (n & 1) ^ 1u, abort_flag, p.status, 400)) goto done;
+        mbar_expect_tx(q_full, Q_BYTES);
+        tma_load_3d(sQ, &tmQ, q_full, 0, kvh * p.group, ia.x);
+        for (int j = kt_lo; j < kt_hi; ++j, ++g) {
+          const int phys_next = (j + 1 < kt_hi) ? bt[j + 1] : 0;      // block-table entry of the next tile, ahead of need
+          const int st = g % KV_STAGES;
+          if (!mbar_wait(kv_empty + st, ((g / KV_STAGES) & 1) ^ 1u, abort_flag, p.status, 401)) goto done;
+          const int row = (((p.layer * p.n_blocks) + phys) * p.Hkv + kvh) * 64;
+          uint8_t* k_dst = sKV + st * 2 * KV_TILE_BYTES;
+          mbar_expect_tx(kv_full + st, 2 * KV_TILE_BYTES);
+          tma_load_2d(k_dst, &tmK, kv_full + st, 0, row);
+          tma_load_2d(k_dst + KV_TILE_BYTES, &tmV, kv_full + st, 0, row);
+          phys = phys_next;
         }
-      }
-    } else if (warp == 5) {
-      if (lane == 0) {
-        constexpr uint32_t idesc = umma_idesc_bf16(64);
-        const uint32_t q_addr = smem_u32(sQ);
-        uint32_t g = 0;
-        int n = 0;
-        for (int w = blockIdx.x; w < total; w += gridDim.x, ++n) {
-          const int4 ib = p.plan.items[2 * (w / p.Hkv) + 1];
-          const int n_it = (ib.x >> 16) - (ib.x & 0xffff);
-          auto issue_s = [&](uint32_t gi) -> bool {
-            const int st = gi % KV_STAGES;
-            if (!mbar_wait(kv_full + st, (gi / KV_STAGES) & 1, abort_flag, p.status, 410)) return false;
-            if (!mbar_wait(s_empty + (gi & 1), ((gi >> 1) & 1) ^ 1u, abort_flag, p.status, 411)) return false;
-            tc_fence_after();
-            const uint32_t k_addr = smem_u32(sKV + st * 2 * KV_TILE_BYTES);
-            const uint32_t d = tmem_base + (gi & 1) * 64;
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              umma_bf16(d, umma_desc_sw128(q_addr + k * 32), umma_desc_sw128(k_addr + k * 32), idesc, k != 0);
-            umma_commit(s_full + (gi & 1));
-            return true;
-          };
-          if (!mbar_wait(q_full, n & 1, abort_flag, p.status, 412)) goto done;
-          if (!issue_s(g)) goto done;
-          if (n_it == 1) umma_commit(q_empty);
-          // the previous item's O has been read out of TMEM
-          if (!mbar_wait(o_empty, (n & 1) ^ 1u, abort_flag, p.status, 415)) goto done;
-          for (int j = 0; j < n_it; ++j, ++g) {
-            if (j + 1 < n_it) {
-              if (!issue_s(g + 1)) goto done;
-              if (j + 2 == n_it) umma_commit(q_empty);    // last S MMA of the item issued: Q is free once it completes
-            }
-            if (!mbar_wait(p_full + (g & 1), (g >> 1) & 1, abort_flag, p.status, 413)) goto done;
-            tc_fence_after();
-            const int st = g % KV_STAGES;
-            const uint32_t p_addr = smem_u32(sP + (g & 1) * P_BYTES);
-            const uint32_t v_addr = smem_u32(sKV + st * 2 * KV_TILE_BYTES + KV_TILE_BYTES);
-            const uint32_t d = tmem_base + 128;
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              umma_bf16(d, umma_desc_sw128(p_addr + k * 32), umma_desc_sw128(v_addr + k * 32), idesc, (j | k) != 0);
-            umma_commit(kv_empty + st);
-            umma_commit(pv_done + (g & 1));
-          }
-        }
-        // every stage-release arrival must land before the CTA's shared memory can be handed on
-        if (g > 0 && !mbar_wait(pv_done + ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag, p.status, 414)) goto done;
       }
     }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(64);
+      const uint32_t q_addr = smem_u32(sQ);
+      uint32_t g = 0;
+      int n = 0;
+      for (int w = blockIdx.x; w < total; w += gridDim.x, ++n) {
+        const int4 ib = p.plan.items[2 * (w / p.Hkv) + 1];
+        const int n_it = (ib.x >> 16) - (ib.x & 0xffff);
+        auto issue_s = [&](uint32_t gi) -> bool {
+          const int st = gi % KV_STAGES;
+          if (!mbar_wait(kv_full + st, (gi / KV_STAGES) & 1, abort_flag, p.status, 410)) return false;
+          if (!mbar_wait(s_empty + (gi & 1), ((gi >> 1) & 1) ^ 1u, abort_flag, p.status, 411)) return false;
+          tc_fence_after();
+          const uint32_t k_addr = smem_u32(sKV + st * 2 * KV_TILE_BYTES);
+          const uint32_t d = tmem_base + (gi & 1) * 64;
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            umma_bf16(d, umma_desc_sw128(q_addr + k * 32), umma_desc_sw128(k_addr + k * 32), idesc, k != 0);
+          umma_commit(s_full + (gi & 1));
+          return true;
+        };
+        if (!mbar_wait(q_full, n & 1, abort_flag, p.status, 412)) goto done;
+        if (!issue_s(g)) goto done;
+        if (n_it == 1) umma_commit(q_empty);
+        for (int j = 0; j < n_it; ++j, ++g) {
+          if (j + 1 < n_it) {
+            if (!issue_s(g + 1)) goto done;
+            if (j + 2 == n_it) umma_commit(q_empty);      // last S MMA of the item issued: Q is free once it completes
+          }
+          // P(g) is written; the softmax warps have also folded PV(g-2) out of the buffer PV(g) is about to overwrite
+          if (!mbar_wait(p_full + (g & 1), (g >> 1) & 1, abort_flag, p.status, 413)) goto done;
+          tc_fence_after();
+          const int st = g % KV_STAGES;
+          const uint32_t p_addr = smem_u32(sP + (g & 1) * P_BYTES);
+          const uint32_t v_addr = smem_u32(sKV + st * 2 * KV_TILE_BYTES + KV_TILE_BYTES);
+          const uint32_t d = tmem_base + 128 + (g & 1) * 64;
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            umma_bf16(d, umma_desc_sw128(p_addr + k * 32), umma_desc_sw128(v_addr + k * 32), idesc, k != 0);
+          umma_commit(kv_empty + st);
+          umma_commit(pv_full + (g & 1));
+        }
+      }
+      // every stage-release arrival must land before the CTA's shared memory can be handed on
+      if (g > 0 && !mbar_wait(pv_full + ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag, p.status, 414)) goto done;
+    }
   } else {
-    reg_alloc<200>();
-    const int quarter = warp;
+    const int quarter = warp & 3;
     const int row = quarter * 32 + lane;               // q row of the tile = TMEM lane
     const int tok = row / p.group;
     const uint32_t t_lane = tmem_base + (uint32_t(quarter * 32) << 16);
     const float sc = 0.125f * 1.4426950408889634f;     // 1/sqrt(64) * log2(e)
-    uint32_t g = 0;
-    int n = 0;
-    for (int w = blockIdx.x; w < total; w += gridDim.x, ++n) {
+    uint32_t g = 0, group_ph = 0;
+    for (int w = blockIdx.x; w < total; w += gridDim.x) {
       const int4 ia = p.plan.items[2 * (w / p.Hkv)], ib = p.plan.items[2 * (w / p.Hkv) + 1];
       const int kvh = w % p.Hkv;
       const int q_row0 = ia.x, pos0 = ia.y, n_tok = ia.z;
@@ -288,8 +269,29 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       const int split = ib.y & 0xffff, n_split = ib.y >> 16;
       const int pos_row = pos0 + tok;
       const bool row_ok = tok < n_tok;
-      const bool warp_ok = (quarter * 32) / p.group < n_tok;   // warp-uniform: some row of this warp is real
-      float m_ref = -INFINITY, l = 0.f;
+      float m = -INFINITY, l = 0.f, alpha_prev = 1.f;
+      float o[64];
+#pragma unroll
+      for (int e = 0; e < 64; ++e) o[e] = 0.f;
+
+      // fold PV(gi) into the row accumulator; the rescale for what was accumulated before it is alpha_prev
+      auto fold_pv = [&](uint32_t gi, int where) -> bool {
+        const int pb = gi & 1;
+        bool ok = mbar_wait(pv_full + pb, (gi >> 1) & 1, abort_flag, p.status, where);
+        if (!__all_sync(0xffffffffu, ok)) return false;
+        tc_fence_after();
+        uint32_t t0[32], t1[32];
+        tmem_ld32(t_lane + 128 + pb * 64, t0);
+        tmem_ld32(t_lane + 128 + pb * 64 + 32, t1);
+        tmem_ld_wait();
+        tc_fence_before();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          o[e] = o[e] * alpha_prev + __uint_as_float(t0[e]);
+          o[32 + e] = o[32 + e] * alpha_prev + __uint_as_float(t1[e]);
+        }
+        return true;
+      };
 
       for (int j = kt_lo; j < kt_hi; ++j, ++g) {
         const int b = g & 1;
@@ -297,182 +299,116 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (!__all_sync(0xffffffffu, ok)) goto done;
         tc_fence_after();
         uint32_t s0[32], s1[32];
-        if (warp_ok) {
-          tmem_ld32(t_lane + b * 64, s0);
-          tmem_ld32(t_lane + b * 64 + 32, s1);
-          tmem_ld_wait();
-        }
+        tmem_ld32(t_lane + b * 64, s0);
+        tmem_ld32(t_lane + b * 64 + 32, s1);
+        tmem_ld_wait();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(s_empty + b);
-        // P[b] was last read by the PV MMA two tiles ago
-        if (g >= 2) {
-          ok = mbar_wait(pv_done + b, ((g - 2) >> 1) & 1, abort_flag, p.status, 421);
-          if (!__all_sync(0xffffffffu, ok)) goto done;
-        }
-        if (warp_ok) {
-          const int kbase = j * 64;
-          if (kbase + 63 > pos0) {                        // some row of the tile masks part of this KV tile
-#pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              if (kbase + e > pos_row) s0[e] = 0xff800000u;          // -inf
-              if (kbase + 32 + e > pos_row) s1[e] = 0xff800000u;
-            }
-          }
-          float mx = -INFINITY;
-#pragma unroll
-          for (int e = 0; e < 32; ++e) mx = max3(mx, __uint_as_float(s0[e]), __uint_as_float(s1[e]));
-          const float m_tile = mx * sc;
-          // raise the reference only when this tile overshoots it by more than 2^8 (always on the first tile)
-          const bool raise = m_tile > m_ref + kRescaleLog2;
-          if (__any_sync(0xffffffffu, raise && j > kt_lo)) {
-            // O holds the sum of the tiles up to j-1: rescale this lane's row in TMEM once PV(j-1) has landed
-            ok = mbar_wait(pv_done + ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag, p.status, 422);
-            if (!__all_sync(0xffffffffu, ok)) goto done;
-            tc_fence_after();
-            const float alpha = raise ? ex2(m_ref - m_tile) : 1.f;
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-              uint32_t o[32];
-              tmem_ld32(t_lane + 128 + h * 32, o);
-              tmem_ld_wait();
-#pragma unroll
-              for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-              tmem_st32(t_lane + 128 + h * 32, o);
-            }
-            tmem_st_wait();
-            tc_fence_before();
-            l *= alpha;
-          }
-          if (raise) m_ref = m_tile;                      // (first tile: l is still 0, O is overwritten by PV)
-          const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-          float sum0 = 0.f, sum1 = 0.f;
-          uint8_t* prow = sP + b * P_BYTES + row * 128;
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            float a[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) a[e] = ex2(fmaf(__uint_as_float(s0[8 * c + e]), sc, -m_use));
-            sum0 += (a[0] + a[1]) + (a[2] + a[3]);
-            sum1 += (a[4] + a[5]) + (a[6] + a[7]);
-            // P row -> shared memory, K-major 128B-swizzled: 16-byte chunk c of row r sits at chunk c ^ (r & 7)
-            *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) =
-                make_uint4(pack_bf16(a[0], a[1]), pack_bf16(a[2], a[3]), pack_bf16(a[4], a[5]), pack_bf16(a[6], a[7]));
-          }
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            float a[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) a[e] = ex2(fmaf(__uint_as_float(s1[8 * c + e]), sc, -m_use));
-            sum0 += (a[0] + a[1]) + (a[2] + a[3]);
-            sum1 += (a[4] + a[5]) + (a[6] + a[7]);
-            *reinterpret_cast<uint4*>(prow + (((4 + c) ^ (row & 7)) << 4)) =
-                make_uint4(pack_bf16(a[0], a[1]), pack_bf16(a[2], a[3]), pack_bf16(a[4], a[5]), pack_bf16(a[6], a[7]));
-          }
-          l += sum0 + sum1;
-          fence_proxy_async_smem();
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(p_full + b);
-      }
 
-      // ---- item epilogue: O is complete once the last PV has landed
-      {
-        bool ok = mbar_wait(pv_done + ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag, p.status, 423);
-        if (!__all_sync(0xffffffffu, ok)) goto done;
-        tc_fence_after();
+        const int kbase = j * 64;
+        if (kbase + 63 > pos0) {                          // some row of the tile masks part of this KV tile
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            if (kbase + e > pos_row) s0[e] = 0xff800000u;          // -inf
+            if (kbase + 32 + e > pos_row) s1[e] = 0xff800000u;
+          }
+        }
+        float mx = -INFINITY;
+#pragma unroll
+        for (int e = 0; e < 32; ++e) mx = max3(mx, __uint_as_float(s0[e]), __uint_as_float(s1[e]));
+        const float m_new = fmaxf(m, mx * sc);
+        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+        const float alpha = ex2(m - m_use);
+        float sum = 0.f;
+        uint32_t pk[32];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          const float a0 = ex2(fmaf(__uint_as_float(s0[2 * e]), sc, -m_use));
+          const float a1 = ex2(fmaf(__uint_as_float(s0[2 * e + 1]), sc, -m_use));
+          sum += a0 + a1;
+          pk[e] = pack_bf16(a0, a1);
+        }
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          const float a0 = ex2(fmaf(__uint_as_float(s1[2 * e]), sc, -m_use));
+          const float a1 = ex2(fmaf(__uint_as_float(s1[2 * e + 1]), sc, -m_use));
+          sum += a0 + a1;
+          pk[16 + e] = pack_bf16(a0, a1);
+        }
+        l = l * alpha + sum;
+        // P row -> shared memory, K-major 128B-swizzled: 16-byte chunk c of row r sits at chunk c ^ (r & 7)
+        uint8_t* prow = sP + b * P_BYTES + row * 128;
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) =
+              make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+        fence_proxy_async_smem();
+        mbar_arrive(p_full + b);
+        m = m_new;
+        // the rescale for everything accumulated so far is applied when PV(g-1) is folded in
+        if (j > kt_lo && !fold_pv(g - 1, 421)) goto done;
+        alpha_prev = alpha;
       }
-      uint32_t o0[32], o1[32];
-      if (warp_ok) {
-        tmem_ld32(t_lane + 128, o0);
-        tmem_ld32(t_lane + 128 + 32, o1);
-        tmem_ld_wait();
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(o_empty);
+      if (!fold_pv(g - 1, 422)) goto done;
 
+      // ---- item epilogue
       const int head = kvh * p.group + row % p.group;
       if (n_split == 1) {
         if (row_ok) {
           const float inv = 1.f / l;
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            o0[e] = __float_as_uint(__uint_as_float(o0[e]) * inv);
-            o1[e] = __float_as_uint(__uint_as_float(o1[e]) * inv);
-          }
           uint4* dst = reinterpret_cast<uint4*>(p.out + (size_t)(q_row0 + tok) * p.Hq * 64 + head * 64);
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            dst[c] = make_uint4(pack_bf16(__uint_as_float(o0[8 * c]), __uint_as_float(o0[8 * c + 1])),
-                                pack_bf16(__uint_as_float(o0[8 * c + 2]), __uint_as_float(o0[8 * c + 3])),
-                                pack_bf16(__uint_as_float(o0[8 * c + 4]), __uint_as_float(o0[8 * c + 5])),
-                                pack_bf16(__uint_as_float(o0[8 * c + 6]), __uint_as_float(o0[8 * c + 7])));
-            dst[4 + c] = make_uint4(pack_bf16(__uint_as_float(o1[8 * c]), __uint_as_float(o1[8 * c + 1])),
-                                    pack_bf16(__uint_as_float(o1[8 * c + 2]), __uint_as_float(o1[8 * c + 3])),
-                                    pack_bf16(__uint_as_float(o1[8 * c + 4]), __uint_as_float(o1[8 * c + 5])),
-                                    pack_bf16(__uint_as_float(o1[8 * c + 6]), __uint_as_float(o1[8 * c + 7])));
-          }
+          for (int c = 0; c < 8; ++c)
+            dst[c] = make_uint4(pack_bf16(o[8 * c] * inv, o[8 * c + 1] * inv), pack_bf16(o[8 * c + 2] * inv, o[8 * c + 3] * inv),
+                                pack_bf16(o[8 * c + 4] * inv, o[8 * c + 5] * inv), pack_bf16(o[8 * c + 6] * inv, o[8 * c + 7] * inv));
         }
       } else {
-        // partial of this slice: the reference maximum (log2 units), the sum, 64 unnormalised outputs
-        float* part = p.split_ws + (((size_t)(q_row0 + tok) * p.Hq + head) * kAttnMaxSplits) * 66;
-        if (row_ok) {
-          float2* d2 = reinterpret_cast<float2*>(part + (size_t)split * 66);
-          d2[0] = make_float2(m_ref, l);
+        // partials of this (q-tile, kv head): [slice][66][128 rows] floats, entry 0 the running maximum (log2
+        // units), 1 the row sum, 2.. the 64 unnormalised outputs; a warp's accesses are 128-byte lines
+        float* tile_part = p.split_ws + ((size_t)(ib.z * p.Hkv + kvh) * kAttnMaxSplits) * (66 * 128) + row;
+        {
+          float* part = tile_part + (size_t)split * (66 * 128);
+          part[0] = m;
+          part[128] = l;
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            d2[1 + e] = make_float2(__uint_as_float(o0[2 * e]), __uint_as_float(o0[2 * e + 1]));
-            d2[17 + e] = make_float2(__uint_as_float(o1[2 * e]), __uint_as_float(o1[2 * e + 1]));
-          }
+          for (int e = 0; e < 64; ++e) part[(2 + e) * 128] = o[e];
         }
         __threadfence();
-        softmax_bar();
-        if (warp == 0 && lane == 0) {
+        if (!warps_sync(group_bar, group_ph, lane, abort_flag, p.status, 427)) goto done;
+        if (warp == 2 && lane == 0) {
           int* ctr = p.plan.counters + ib.z * p.Hkv + kvh;
           const int old = atomicAdd(ctr, 1);
           *s_flag = (old == n_split - 1);
           if (old == n_split - 1) *ctr = 0;             // ready for the next layer
         }
-        softmax_bar();
+        if (!warps_sync(group_bar, group_ph, lane, abort_flag, p.status, 428)) goto done;
         if (*s_flag) {
           __threadfence();
+          float M = -INFINITY;
+          for (int s = 0; s < n_split; ++s) M = fmaxf(M, __ldcg(tile_part + (size_t)s * (66 * 128)));
+          float Lsum = 0.f;
+#pragma unroll
+          for (int e = 0; e < 64; ++e) o[e] = 0.f;
+          for (int s = 0; s < n_split; ++s) {             // fixed slice order: the result does not depend on arrival
+            const float* ps = tile_part + (size_t)s * (66 * 128);
+            const float mx = __ldcg(ps);
+            const float wgt = (mx == -INFINITY) ? 0.f : ex2(mx - M);
+            Lsum += wgt * __ldcg(ps + 128);
+#pragma unroll
+            for (int e = 0; e < 64; ++e) o[e] += wgt * __ldcg(ps + (2 + e) * 128);
+          }
           if (row_ok) {
-            float M = -INFINITY;
-            for (int s = 0; s < n_split; ++s) M = fmaxf(M, __ldcg(part + s * 66));
-            float L = 0.f;
-            for (int s = 0; s < n_split; ++s) {
-              const float2 ml = __ldcg(reinterpret_cast<const float2*>(part + s * 66));
-              L += ((ml.x == -INFINITY) ? 0.f : ex2(ml.x - M)) * ml.y;
-            }
-            const float inv = 1.f / L;
+            const float inv = 1.f / Lsum;
             uint4* dst = reinterpret_cast<uint4*>(p.out + (size_t)(q_row0 + tok) * p.Hq * 64 + head * 64);
-#pragma unroll 1
-            for (int hf = 0; hf < 2; ++hf) {              // 32 outputs at a time keeps the register count down
-              float acc[32];
 #pragma unroll
-              for (int e = 0; e < 32; ++e) acc[e] = 0.f;
-              for (int s = 0; s < n_split; ++s) {         // fixed slice order: the result does not depend on arrival
-                const float2* src = reinterpret_cast<const float2*>(part + s * 66);
-                const float mx = __ldcg(part + s * 66);
-                const float wgt = (mx == -INFINITY) ? 0.f : ex2(mx - M);
-#pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                  const float2 v = __ldcg(src + 1 + hf * 16 + e);
-                  acc[2 * e] += wgt * v.x;
-                  acc[2 * e + 1] += wgt * v.y;
-                }
-              }
-#pragma unroll
-              for (int c = 0; c < 4; ++c)
-                dst[hf * 4 + c] = make_uint4(pack_bf16(acc[8 * c] * inv, acc[8 * c + 1] * inv),
-                                             pack_bf16(acc[8 * c + 2] * inv, acc[8 * c + 3] * inv),
-                                             pack_bf16(acc[8 * c + 4] * inv, acc[8 * c + 5] * inv),
-                                             pack_bf16(acc[8 * c + 6] * inv, acc[8 * c + 7] * inv));
-            }
+            for (int c = 0; c < 8; ++c)
+              dst[c] = make_uint4(pack_bf16(o[8 * c] * inv, o[8 * c + 1] * inv), pack_bf16(o[8 * c + 2] * inv, o[8 * c + 3] * inv),
+                                  pack_bf16(o[8 * c + 4] * inv, o[8 * c + 5] * inv), pack_bf16(o[8 * c + 6] * inv, o[8 * c + 7] * inv));
           }
         }
-        softmax_bar();                                  // s_flag is rewritten by the next item only after all have read it
+        // s_flag is rewritten by the next item only after all have read it
+        if (!warps_sync(group_bar, group_ph, lane, abort_flag, p.status, 429)) goto done;
       }
     }
   }
@@ -480,7 +416,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 done:
   tc_fence_before();
   __syncthreads();
-  if (warp == 5) {
+  if (warp == 1) {
     if (*abort_flag) __nanosleep(20000);
     tmem_dealloc(tmem_base, ATTN_TMEM_COLS);
   }

@@ -97,14 +97,17 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
+// One probe of the barrier.  The suspend-time hint lets the hardware park the warp until the phase completes
+// (or the hint expires) instead of returning at once: a parked warp takes no issue slots from the warps that
+// share its scheduler, which matters because most warps of these kernels spend most of their time waiting.
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred P;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2, %3;\n\t"
       "selp.b32 %0, 1, 0, P;\n\t}\n"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(20000u)
       : "memory");
   return ok != 0;
 }
@@ -112,7 +115,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait.  Every spin in these kernels has an iteration limit: when it runs out (or another thread
 // of the CTA has already given up) the wait records DEV_WAIT_TIMEOUT in the status words, raises the
 // CTA-wide abort flag and returns false; callers then fall through to the common teardown.
-constexpr uint32_t kWaitSpins = 1u << 24;
+constexpr uint32_t kWaitSpins = 1u << 22;
 constexpr unsigned long long kWaitNs = 2000000000ull;   // 2 s of wall clock
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
@@ -121,15 +124,15 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
                                           int where) {
+  if (mbar_try_wait(bar, parity)) return true;
   unsigned long long t0 = 0;
   for (uint32_t i = 0; i < kWaitSpins; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 63u) == 63u) {
+    if ((i & 7u) == 7u) {
       if (*abort_flag) return false;
       const unsigned long long now = global_ns();
       if (t0 == 0) t0 = now;
       if (now - t0 > kWaitNs) break;
-      __nanosleep(64);
     }
   }
   *abort_flag = 1;

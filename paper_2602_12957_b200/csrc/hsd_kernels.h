@@ -98,7 +98,7 @@ void launch_unpack_best(cudaStream_t st, const unsigned long long* row_best, int
                         bool pdl);
 
 // ---- attention plan (hsd_attn_sm100.cu): made once per step on the device, read by every layer's launch ----
-constexpr int kAttnMaxSplits = 16;     // most KV slices one q-tile is cut into
+constexpr int kAttnMaxSplits = 8;      // most KV slices one q-tile is cut into
 struct AttnPlan {
   int4* items;      // two int4 per (q-tile, slice) item: {first packed row, position of the first token, tokens, KV slot},
                     // {first | (last + 1) << 16 KV tile, slice | slices << 16, q-tile, 0}
