@@ -240,24 +240,30 @@ def run_ours(args):
     draft_tokens = sum(st["ks"])
     value = draft_tokens * world / (ms_step * 1e-3)
 
-    # ---- end to end through the C-ABI with host buffers (pinned): H2D inputs, verify + commit, D2H results
+    # ---- end to end through the C-ABI call that takes HOST buffers (pinned): every step copies the packed drafts
+    # host->device, runs verify + commit, copies accept_len / n_emit / emitted tokens device->host and synchronises
     h_toks = torch.from_numpy(st["toks"]).pin_memory()
     h_cu = torch.from_numpy(st["cu"]).pin_memory()
     h_acc = torch.empty(S, dtype=torch.int32).pin_memory()
     h_nem = torch.empty(S, dtype=torch.int32).pin_memory()
     h_emit = torch.empty(S, max_q, dtype=torch.int32).pin_memory()
     e2e_steps = max(3, min(args.steps, 200))
+    ctx = eng.model.ctx
+
+    def e2e_step():
+        rc, _ = B.hsd_verify_regions_host(ctx, kv.c, S, h_cu, h_toks, None, 0.0, 1, h_acc, h_emit, h_nem, eng.ws.ptr,
+                                          eng.ws.bytes, stream.cuda_stream)
+        B.check(rc, "hsd_verify_regions_host")
+        kv.seq_lens.copy_(st["prefix_lens"])          # rewind (bench artefact: every step sees the same state)
+
     with torch.cuda.stream(stream):
+        for _ in range(3):
+            e2e_step()
         barrier()
         t0 = time.perf_counter()
         for _ in range(e2e_steps):
-            d_toks.copy_(h_toks, non_blocking=True)
-            d_cu.copy_(h_cu, non_blocking=True)
-            run()
-            h_acc.copy_(out["accept_len"], non_blocking=True)
-            h_nem.copy_(out["n_emit"], non_blocking=True)
-            h_emit.copy_(out["emit_tokens"], non_blocking=True)
-            stream.synchronize()
+            e2e_step()
+        stream.synchronize()
         t1 = time.perf_counter()
         barrier()
     e2e_ms = (t1 - t0) * 1e3 / e2e_steps
@@ -267,7 +273,8 @@ def run_ours(args):
         e2e_ms = float(tt.item())
     e2e = {"value": draft_tokens * world / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
            "h2d_bytes_per_step": int(h_toks.numel() * 4 + h_cu.numel() * 4),
-           "d2h_bytes_per_step": int((h_acc.numel() + h_nem.numel() + h_emit.numel()) * 4)}
+           "d2h_bytes_per_step": int((h_acc.numel() + h_nem.numel() + h_emit.numel()) * 4 + 16),
+           "call": "hsd_verify_regions_host (eager launches, pinned host buffers, stream synchronised per step)"}
     accept_mean = float(np.mean([a / k for a, k in zip(h_acc.numpy().tolist(), st["ks"])]))
 
     # ---- per-kernel durations (CUDA events around every launch, eager) for the roofline of the top kernel

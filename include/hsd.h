@@ -31,8 +31,8 @@
  *      w_down    [d_model, d_ffn]
  *      embed, lm_head [vocab, d_model];  *_norm [d_model] (bf16 gains)
  *  - Paged KV pool, block = kv_block (64) tokens:
- *      k_pool bf16 [n_layers][n_blocks][n_kv_heads][64 tokens][head_dim]
- *      v_pool bf16 [n_layers][n_blocks][n_kv_heads][head_dim][64 tokens]      (V is stored transposed)
+ *      k_pool, v_pool bf16 [n_layers][n_blocks][n_kv_heads][64 tokens][head_dim]
+ *    (one 128-byte line per token and kv head; a (block, kv head) tile is 8 KB contiguous)
  *    block_table int32 [n_slots, max_blocks_per_seq]: physical block of logical block j of slot s.
  *    seq_lens int32 [n_slots]: committed K/V rows per slot.
  *  - Packed query tokens: q_tokens[cu_q[i] .. cu_q[i+1]) = [pending_i, d_i1 .. d_ik].
@@ -168,6 +168,21 @@ HSD_API int hsd_verify_page(hsd_ctx *ctx, const hsd_kv *kv, int seq_slot, const 
  * receives ceil(new_len / 64). */
 HSD_API int hsd_kv_commit(hsd_ctx *ctx, const hsd_kv *kv, int n_seqs, const int *seq_slots, const int *accept_len,
                   int *blocks_in_use, void *cuda_stream);
+
+/* Stage 1 with HOST buffers: the same step as hsd_verify_regions followed (if commit != 0) by hsd_kv_commit, for
+ * callers whose drafts and results live in host memory (Eq. 2 and Eq. 12 end to end, including the transfers the
+ * paper counts in T_decode, Sec. 4.2).
+ *   cu_q, q_tokens        HOST int32 [n_seqs+1], [cu_q[n_seqs]] (pinned memory makes the copies asynchronous)
+ *   seq_slots             dev int32 [n_seqs] or NULL, as above
+ *   accept_len, n_emit    HOST int32 [n_seqs] out
+ *   emit_tokens           HOST int32 [n_seqs, max_q_len] out, max_q_len = max_i(cu_q[i+1]-cu_q[i]), also
+ *                         returned through max_q_len_out (may be NULL); the buffer must hold n_seqs * max_q_len ints
+ * Copies the inputs into staging areas inside `workspace`, runs the step on the stream, copies the results back and
+ * SYNCHRONISES the stream before returning; a device-side check that tripped is returned as HSD_ERR_DEVICE_CHECK.
+ * Errors otherwise as hsd_verify_regions. */
+HSD_API int hsd_verify_regions_host(hsd_ctx *ctx, const hsd_kv *kv, int n_seqs, const int *cu_q, const int *q_tokens,
+                            const int *seq_slots, float log_tau, int commit, int *accept_len, int *emit_tokens,
+                            int *n_emit, int *max_q_len_out, void *workspace, size_t ws_bytes, void *cuda_stream);
 
 /* Device status words written by the last call that used `workspace` (synchronises the stream).
  * status[0] = 0 if every device-side check passed, else a code (1 cu_q not monotone, 2 sequence too long,

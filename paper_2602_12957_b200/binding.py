@@ -26,7 +26,7 @@ HSD_NOALLOC_MAX_ROWS = 8192
 
 EXPORTS = [
     "hsd_status_string", "hsd_create", "hsd_destroy", "hsd_workspace_bytes", "hsd_prefill", "hsd_verify_regions",
-    "hsd_verify_page", "hsd_kv_commit", "hsd_device_status", "hsd_last_cuda_error", "hsd_launch_count",
+    "hsd_verify_page", "hsd_kv_commit", "hsd_verify_regions_host", "hsd_device_status", "hsd_last_cuda_error", "hsd_launch_count",
     "hsd_profile_enable", "hsd_profile_read", "hsd_debug_logits", "hsd_debug_buffer", "hsd_op_linear",
     "hsd_op_lm_head_argmax", "hsd_op_lm_head_argmax_noalloc", "hsd_debug_set_gemm_tile", "hsd_debug_set_attn_plan",
 ]
@@ -74,6 +74,7 @@ def _load():
     lib.hsd_verify_regions.argtypes = [vp, C.POINTER(hsd_kv), i, vp, vp, vp, i, i, f, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.hsd_verify_page.argtypes = [vp, C.POINTER(hsd_kv), i, vp, vp, i, f, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.hsd_kv_commit.argtypes = [vp, C.POINTER(hsd_kv), i, vp, vp, vp, vp]
+    lib.hsd_verify_regions_host.argtypes = [vp, C.POINTER(hsd_kv), i, vp, vp, vp, f, i, vp, vp, vp, C.POINTER(C.c_int), vp, sz, vp]
     lib.hsd_device_status.argtypes = [vp, vp, vp, C.POINTER(C.c_int)]
     lib.hsd_last_cuda_error.argtypes = [vp]
     lib.hsd_launch_count.restype = C.c_longlong
@@ -179,6 +180,17 @@ def hsd_verify_page(ctx, kv, seq_slot, pending_token, draft_chunk, chunk_len, lo
     return _lib.hsd_verify_page(ctx, C.byref(kv) if kv is not None else None, seq_slot, _p(pending_token),
                                 _p(draft_chunk), chunk_len, log_tau, _p(accept_len), _p(emit_tokens), _p(n_emit),
                                 _p(row_argmax), _p(row_zmax), _p(row_zdraft), _p(workspace), ws_bytes, _p(stream))
+
+
+def hsd_verify_regions_host(ctx, kv, n_seqs, cu_q, q_tokens, seq_slots, log_tau, commit, accept_len, emit_tokens, n_emit,
+                            workspace, ws_bytes, stream):
+    """Host-buffer form: cu_q, q_tokens, accept_len, emit_tokens, n_emit are HOST tensors (CPU torch tensors or
+    addresses).  Returns (status, max_q_len)."""
+    mq = C.c_int(0)
+    st = _lib.hsd_verify_regions_host(ctx, C.byref(kv) if kv is not None else None, n_seqs, _p(cu_q), _p(q_tokens),
+                                      _p(seq_slots), log_tau, int(commit), _p(accept_len), _p(emit_tokens), _p(n_emit),
+                                      C.byref(mq), _p(workspace), ws_bytes, _p(stream))
+    return st, mq.value
 
 
 def hsd_kv_commit(ctx, kv, n_seqs, seq_slots, accept_len, blocks_in_use, stream) -> int:

@@ -47,6 +47,8 @@ struct Ws {
   RowMeta rm;
   int* sel_rows;
   int* cu_one;        // {0, n} offsets of a single-sequence call
+  int *h_tokens, *h_cu, *h_accept, *h_nemit, *h_emit;   // device staging of hsd_verify_regions_host
+  size_t h_emit_ints;
   float* x;
   bf16* h;
   bf16* q;
@@ -91,6 +93,12 @@ Ws carve(const hsd_ctx* c, void* base, int T, int S) {
   w.rm.seq_tile0 = static_cast<int*>(take(sizeof(int) * (S + 1)));
   w.sel_rows = static_cast<int*>(take(sizeof(int) * S));
   w.cu_one = static_cast<int*>(take(sizeof(int) * 2));
+  w.h_tokens = static_cast<int*>(take(sizeof(int) * T));
+  w.h_cu = static_cast<int*>(take(sizeof(int) * (S + 1)));
+  w.h_accept = static_cast<int*>(take(sizeof(int) * S));
+  w.h_nemit = static_cast<int*>(take(sizeof(int) * S));
+  w.h_emit_ints = (size_t)S * (T < HSD_MAX_Q_LEN ? T : HSD_MAX_Q_LEN);
+  w.h_emit = static_cast<int*>(take(sizeof(int) * w.h_emit_ints));
   w.x = static_cast<float*>(take(sizeof(float) * (size_t)T * md.d));
   w.h = static_cast<bf16*>(take(2 * (size_t)T * md.d));
   w.q = static_cast<bf16*>(take(2 * (size_t)T * md.Hq * md.D));
@@ -237,7 +245,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
     // q as [T][Hq][64]: one box = (128/group) tokens x group heads x 64 dims -> a 128-row MMA operand
     if (make_tmap_3d(&tm_q, w.q, 64, md.Hq, T, 128, (uint64_t)md.Hq * 128, 64, md.group, tokens_per_tile))
       return HSD_ERR_CUDA;
-    // K / V^T pools as 2-D [rows, 64]: one (layer, block, kv head) tile = 64 consecutive rows
+    // K / V pools as 2-D [rows, 64]: one (layer, block, kv head) tile = 64 consecutive rows
     const uint64_t pool_rows = (uint64_t)md.n_layers * kv.n_blocks * md.Hkv * 64;
     if (make_tmap_2d(&tm_k, kv.k_pool, pool_rows, 64, 64) || make_tmap_2d(&tm_v, kv.v_pool, pool_rows, 64, 64))
       return HSD_ERR_CUDA;
@@ -283,6 +291,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         g.qkv.v_pool_layer = kv.v_pool + (size_t)l * layer_elems;
         g.qkv.Hq = md.Hq; g.qkv.Hkv = md.Hkv;
         g.status = w.status; g.n_sms = c->n_sms; g.max_splits = 1; g.pdl = c->pdl;
+        g.force_bn = c->force_bn;
         if (launch_gemm_sm100(st, g)) return fail_cuda(c);
       }
       {
@@ -621,6 +630,46 @@ int hsd_kv_commit(hsd_ctx* c, const hsd_kv* kv, int n_seqs, const int* seq_slots
   Scope s(c, st, KC_COMMIT);
   launch_commit(st, kv_view(kv), n_seqs, seq_slots, accept_len, blocks_in_use, c->pdl);
   return check_cuda(c);
+}
+
+int hsd_verify_regions_host(hsd_ctx* c, const hsd_kv* kv, int n_seqs, const int* cu_q, const int* q_tokens,
+                            const int* seq_slots, float log_tau, int commit, int* accept_len, int* emit_tokens,
+                            int* n_emit, int* max_q_len_out, void* workspace, size_t ws_bytes, void* cuda_stream) {
+  if (!c || !cu_q || !q_tokens || !accept_len || !emit_tokens || !n_emit || n_seqs <= 0) return HSD_ERR_INVALID_ARG;
+  if (cu_q[0] != 0) return HSD_ERR_INVALID_ARG;
+  int max_q = 0;
+  for (int i = 0; i < n_seqs; ++i) {
+    const int q = cu_q[i + 1] - cu_q[i];
+    if (q <= 0) return HSD_ERR_INVALID_ARG;
+    if (q > max_q) max_q = q;
+  }
+  const int total_q = cu_q[n_seqs];
+  if (max_q > HSD_MAX_Q_LEN) return HSD_ERR_TOO_LONG;
+  int rc = check_ws(c, workspace, ws_bytes, total_q, n_seqs);
+  if (rc) return rc;
+  const Ws w = carve(c, workspace, total_q, n_seqs);
+  if ((size_t)n_seqs * max_q > w.h_emit_ints) return HSD_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(w.h_cu, cu_q, sizeof(int) * (n_seqs + 1), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(w.h_tokens, q_tokens, sizeof(int) * total_q, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return fail_cuda(c);
+  rc = hsd_verify_regions(c, kv, n_seqs, w.h_cu, w.h_tokens, seq_slots, max_q, total_q, log_tau, w.h_accept, w.h_emit,
+                          w.h_nemit, nullptr, nullptr, nullptr, workspace, ws_bytes, cuda_stream);
+  if (rc) return rc;
+  if (commit) {
+    rc = hsd_kv_commit(c, kv, n_seqs, seq_slots, w.h_accept, nullptr, cuda_stream);
+    if (rc) return rc;
+  }
+  if (cudaMemcpyAsync(accept_len, w.h_accept, sizeof(int) * n_seqs, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaMemcpyAsync(n_emit, w.h_nemit, sizeof(int) * n_seqs, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaMemcpyAsync(emit_tokens, w.h_emit, sizeof(int) * (size_t)n_seqs * max_q, cudaMemcpyDeviceToHost, st) !=
+          cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return fail_cuda(c);
+  if (max_q_len_out) *max_q_len_out = max_q;
+  int status[4];
+  if (cudaMemcpy(status, workspace, sizeof(status), cudaMemcpyDeviceToHost) != cudaSuccess) return fail_cuda(c);
+  return status[0] ? HSD_ERR_DEVICE_CHECK : HSD_OK;
 }
 
 int hsd_device_status(hsd_ctx* c, const void* workspace, void* cuda_stream, int status[4]) {

@@ -5,8 +5,8 @@
 //
 // Work item = (q-tile, kv slice, kv head).  A q-tile is 128 MMA rows: 128/group consecutive tokens of one
 // sequence x the `group` query heads that share the kv head (GQA packing, so K/V tiles are read once per
-// group).  K tiles [64 keys][64 dims] and V^T tiles [64 dims][64 keys] are exactly one paged block per kv
-// head, fetched by TMA through the block table.  The KV range a q-tile can see is cut into up to
+// group).  K and V tiles [64 keys][64 dims] are exactly one paged block per kv head, fetched by TMA through
+// the block table; K is the K-major B operand of S = Q K^T, V the MN-major B operand of P V.  The KV range a q-tile can see is cut into up to
 // kAttnMaxSplits slices so that a launch has a few items per CTA slot whatever the mix of context lengths
 // (one page chunk over a long context, or many short regions); the plan is made once per step on the
 // device (attn_plan_kernel) and reused by every layer.  Slices leave (unnormalised O, max, sum) partials in
@@ -26,7 +26,7 @@ namespace hsd {
 constexpr int kAttnThreads = 192;
 constexpr int KV_STAGES = 3;
 constexpr int Q_BYTES = 128 * 128;
-constexpr int KV_TILE_BYTES = 64 * 128;            // one K tile or one V^T tile
+constexpr int KV_TILE_BYTES = 64 * 128;            // one K tile or one V tile
 constexpr int P_BYTES = 128 * 128;
 constexpr int ATTN_SMEM = Q_BYTES + KV_STAGES * 2 * KV_TILE_BYTES + 2 * P_BYTES + 1024 + 256;
 constexpr int ATTN_TMEM_COLS = 256;                // S0 S1 PV0 PV1, 64 fp32 columns each
@@ -128,7 +128,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sQ = smem;
-  uint8_t* sKV = sQ + Q_BYTES;                         // stage s: K at s*2*KV_TILE_BYTES, V^T right after
+  uint8_t* sKV = sQ + Q_BYTES;                         // stage s: K at s*2*KV_TILE_BYTES, V right after
   uint8_t* sP = sKV + KV_STAGES * 2 * KV_TILE_BYTES;   // two P buffers
   uint64_t* bars = reinterpret_cast<uint64_t*>(sP + 2 * P_BYTES);
   uint64_t* q_full = bars;                 // Q tile landed                       (one phase per item)
@@ -210,6 +210,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16(64);
+      constexpr uint32_t idesc_pv = umma_idesc_bf16(64, true);
       const uint32_t q_addr = smem_u32(sQ);
       uint32_t g = 0;
       int n = 0;
@@ -245,8 +246,8 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           const uint32_t v_addr = smem_u32(sKV + st * 2 * KV_TILE_BYTES + KV_TILE_BYTES);
           const uint32_t d = tmem_base + 128 + (g & 1) * 64;
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            umma_bf16(d, umma_desc_sw128(p_addr + k * 32), umma_desc_sw128(v_addr + k * 32), idesc, k != 0);
+          for (int k = 0; k < 4; ++k)   // V [key][dim] is MN-major: a K step of 16 keys is 16 rows of 128 bytes
+            umma_bf16(d, umma_desc_sw128(p_addr + k * 32), umma_desc_sw128(v_addr + k * 2048), idesc_pv, k != 0);
           umma_commit(kv_empty + st);
           umma_commit(pv_full + (g & 1));
         }

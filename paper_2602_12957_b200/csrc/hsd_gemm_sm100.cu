@@ -274,6 +274,13 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       const bool row_ok = row < p.M;
       const int wrow0 = m0 + quarter * 32;        // first row of this warp's 32-row slab
       const bool slab_ok = wrow0 < p.M;           // warp-uniform: the slab has at least one real row
+      // rotary (cos, sin) of this thread's row: fetched while the main loop still runs, reused by every head
+      float4 cs[MODE == GS_QKV_ROPE ? 16 : 1];
+      if (MODE == GS_QKV_ROPE && row_ok) {
+        const float4* src = reinterpret_cast<const float4*>(p.qkv.rope_cs + (size_t)row * 32);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) cs[i] = __ldg(src + i);
+      }
       bool ok = mbar_wait(tfull + b, aph, abort_flag, p.status, 300);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) goto done;
@@ -393,49 +400,41 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           tmem_ld32(t_acc + hh * 64, lo);
           tmem_ld32(t_acc + hh * 64 + 32, hi);
           tmem_ld_wait();
-          if (head < p.qkv.Hq + p.qkv.Hkv) {
-            if (row_ok) {
-              const float4* cs = reinterpret_cast<const float4*>(p.qkv.rope_cs + (size_t)row * 32);
+          if (head < p.qkv.Hq + p.qkv.Hkv && row_ok) {
 #pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                const float4 c2 = cs[i];   // (cos, sin) of frequencies 2i and 2i+1
-                const float a0 = __uint_as_float(lo[2 * i]), b0 = __uint_as_float(hi[2 * i]);
-                const float a1 = __uint_as_float(lo[2 * i + 1]), b1 = __uint_as_float(hi[2 * i + 1]);
-                lo[2 * i] = __float_as_uint(a0 * c2.x - b0 * c2.y);
-                hi[2 * i] = __float_as_uint(b0 * c2.x + a0 * c2.y);
-                lo[2 * i + 1] = __float_as_uint(a1 * c2.z - b1 * c2.w);
-                hi[2 * i + 1] = __float_as_uint(b1 * c2.z + a1 * c2.w);
-              }
+            for (int i = 0; i < 16; ++i) {
+              const float4 c2 = cs[i];   // (cos, sin) of frequencies 2i and 2i+1
+              const float a0 = __uint_as_float(lo[2 * i]), b0 = __uint_as_float(hi[2 * i]);
+              const float a1 = __uint_as_float(lo[2 * i + 1]), b1 = __uint_as_float(hi[2 * i + 1]);
+              lo[2 * i] = __float_as_uint(a0 * c2.x - b0 * c2.y);
+              hi[2 * i] = __float_as_uint(b0 * c2.x + a0 * c2.y);
+              lo[2 * i + 1] = __float_as_uint(a1 * c2.z - b1 * c2.w);
+              hi[2 * i + 1] = __float_as_uint(b1 * c2.z + a1 * c2.w);
             }
-            if (is_q) {
+          }
+          if (is_q) {
 #pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                *stg_chunk(buf, lane, v) = pack8(lo + 8 * v);
-                *stg_chunk(buf, lane, 4 + v) = pack8(hi + 8 * v);
-              }
-              fence_proxy_async_smem();
-              __syncwarp();
-              if (lane == 0) {
-                tma_store_2d(&tmC, buf, head * 64, wrow0);
-                bulk_commit();
-              }
-              ++n_stores;
-            } else if (row_ok) {
-              uint4* d4 = reinterpret_cast<uint4*>(
-                  p.qkv.k_pool_layer + (((size_t)blk * p.qkv.Hkv + (head - p.qkv.Hq)) * 64 + off) * 64);
-#pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                d4[v] = pack8(lo + 8 * v);
-                d4[4 + v] = pack8(hi + 8 * v);
-              }
+            for (int v = 0; v < 4; ++v) {
+              *stg_chunk(buf, lane, v) = pack8(lo + 8 * v);
+              *stg_chunk(buf, lane, 4 + v) = pack8(hi + 8 * v);
             }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&tmC, buf, head * 64, wrow0);
+              bulk_commit();
+            }
+            ++n_stores;
           } else if (row_ok) {
-            // V is stored transposed per block: [dim][token]; consecutive lanes hold consecutive tokens
-            bf16* dst = p.qkv.v_pool_layer + ((size_t)blk * p.qkv.Hkv + (head - p.qkv.Hq - p.qkv.Hkv)) * 4096 + off;
+            // K and V rows go to the paged pool: one 128-byte line per (token, kv head)
+            const bool is_k = head < p.qkv.Hq + p.qkv.Hkv;
+            bf16* pool = is_k ? p.qkv.k_pool_layer : p.qkv.v_pool_layer;
+            const int kvh = head - p.qkv.Hq - (is_k ? 0 : p.qkv.Hkv);
+            uint4* d4 = reinterpret_cast<uint4*>(pool + (((size_t)blk * p.qkv.Hkv + kvh) * 64 + off) * 64);
 #pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              dst[(size_t)e * 64] = __float2bfloat16(__uint_as_float(lo[e]));
-              dst[(size_t)(e + 32) * 64] = __float2bfloat16(__uint_as_float(hi[e]));
+            for (int v = 0; v < 4; ++v) {
+              d4[v] = pack8(lo + 8 * v);
+              d4[4 + v] = pack8(hi + 8 * v);
             }
           }
         }

@@ -254,9 +254,9 @@ __global__ void rope_kvwrite_kernel(const float* __restrict__ qkv, RowMeta rm, K
       dst[lane + 32] = __float2bfloat16(rb);
     }
   } else {
-    bf16* dst = kv.v_pool + (blk_base + (hd - md.Hq - md.Hkv)) * 4096;
-    dst[(size_t)lane * 64 + off] = __float2bfloat16(a);
-    dst[(size_t)(lane + 32) * 64 + off] = __float2bfloat16(b);
+    bf16* dst = kv.v_pool + ((blk_base + (hd - md.Hq - md.Hkv)) * 64 + off) * 64;
+    dst[lane] = __float2bfloat16(a);
+    dst[lane + 32] = __float2bfloat16(b);
   }
 }
 void launch_rope_kvwrite(cudaStream_t st, const float* qkv, const RowMeta& rm, const KvView& kv, const ModelDims& md,
@@ -313,14 +313,14 @@ __global__ void attn_simt_kernel(const bf16* __restrict__ q, RowMeta rm, KvView 
     o0 *= scale;
     o1 *= scale;
     m = m_new;
-    // V^T tile [dim][tok]: lane owns dims lane and lane + 32
+    // V tile [tok][dim]: lane owns dims lane and lane + 32
     const bf16* vt = kv.v_pool + tile * 4096;
     const int tok0 = k0 % 64;
     const int cnt = min(32, n_keys - k0);
     for (int t = 0; t < cnt; ++t) {
       const float pt = __shfl_sync(0xffffffffu, p, t);
-      o0 += pt * __bfloat162float(vt[(size_t)lane * 64 + tok0 + t]);
-      o1 += pt * __bfloat162float(vt[(size_t)(lane + 32) * 64 + tok0 + t]);
+      o0 += pt * __bfloat162float(vt[(size_t)(tok0 + t) * 64 + lane]);
+      o1 += pt * __bfloat162float(vt[(size_t)(tok0 + t) * 64 + lane + 32]);
     }
   }
   bf16* op = out + (size_t)r * md.Hq * 64 + hq * 64;

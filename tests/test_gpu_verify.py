@@ -90,3 +90,37 @@ def test_one_verify_call_equals_sequential_single_token_steps_on_gpu():
     assert np.array_equal(am, greedy), "teacher-forced rows must reproduce the sequential greedy tokens"
     assert np.array_equal(z, seq_z), f"max |dz| {np.abs(z - seq_z).max()}"
     assert o["accept_len"].cpu().numpy().tolist() == [k] * S
+
+
+def test_host_buffer_call_matches_the_device_call_and_commits():
+    """hsd_verify_regions_host (host buffers in, host buffers out, commit folded in) against hsd_verify_regions +
+    hsd_kv_commit on the same inputs: identical integers, and the committed lengths advance by accept_len + 1."""
+    import torch
+    from paper_2602_12957_b200 import binding as B
+    wl = I.tiny_workload()
+    weights = I.make_weights(wl.cfg, wl.seed)
+    orc = H.oracle_regions(wl, weights, np.float64)
+    per, eng, (toks, cu, total_q) = H.gpu_regions(wl, weights, {i: o.pending for i, o in orc.items()},
+                                                  {i: o.draft for i, o in orc.items()}, B.HSD_FLAG_DETERMINISTIC)
+    S = len(orc)
+    before = eng.kv.seq_lens.cpu().numpy().copy()
+    h_toks, h_cu = torch.from_numpy(toks).pin_memory(), torch.from_numpy(cu).pin_memory()
+    max_q = int(np.diff(cu).max())
+    h_acc = torch.full((S,), -7, dtype=torch.int32).pin_memory()
+    h_nem = torch.full((S,), -7, dtype=torch.int32).pin_memory()
+    h_emit = torch.full((S, max_q), -7, dtype=torch.int32).pin_memory()
+    rc, mq = B.hsd_verify_regions_host(eng.model.ctx, eng.kv.c, S, h_cu, h_toks, None, 0.0, 1, h_acc, h_emit, h_nem,
+                                       eng.ws.ptr, eng.ws.bytes, torch.cuda.current_stream().cuda_stream)
+    B.check(rc, "hsd_verify_regions_host")
+    assert mq == max_q
+    for j, i in enumerate(sorted(orc)):
+        a = int(per[i]["accept_len"])
+        assert int(h_acc[j]) == a and int(h_nem[j]) == a + 1
+        assert h_emit[j, :a + 1].tolist() == per[i]["emit"][:a + 1].tolist()
+    after = eng.kv.seq_lens.cpu().numpy()
+    assert (after - before).tolist() == [int(h_acc[j]) + 1 for j in range(S)]
+    # malformed host offsets are refused before anything is launched
+    bad = h_cu.clone(); bad[0] = 1
+    rc, _ = B.hsd_verify_regions_host(eng.model.ctx, eng.kv.c, S, bad, h_toks, None, 0.0, 0, h_acc, h_emit, h_nem,
+                                      eng.ws.ptr, eng.ws.bytes, torch.cuda.current_stream().cuda_stream)
+    assert rc == B.HSD_ERR_INVALID_ARG
