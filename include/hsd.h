@@ -223,7 +223,8 @@ HSD_API int hsd_debug_buffer(hsd_ctx *ctx, const void *workspace, int total_q, i
 HSD_API int hsd_op_linear(hsd_ctx *ctx, const void *A, const void *W, void *C, int M, int n_out, int K, int mode,
                   void *cuda_stream);
 
-/* Test-only: make hsd_op_linear use output tiles of `tile_n` columns (64, 128 or 256) and, for mode 1, `k_slices`
+/* Test-only: make hsd_op_linear use output tiles of `tile_n` columns (64, 128, 256, or 512 = a pair of CTAs sharing a
+ * 256-row x 256-column tile) and, for mode 1, `k_slices`
  * slices of K per tile, instead of what the library would choose for the problem; 0 = choose.  A combination the
  * problem does not allow makes hsd_op_linear return HSD_ERR_CUDA.  Lets the parity tests reach every tile shape. */
 HSD_API int hsd_debug_set_gemm_tile(hsd_ctx *ctx, int tile_n, int k_slices);

@@ -25,6 +25,7 @@ struct hsd_ctx {
   int max_splits;     // K slices the residual-add projections may use (1 with HSD_FLAG_DETERMINISTIC)
   bool pdl;           // kernels are launched with programmatic stream serialization
   int force_bn, force_splits;   // hsd_debug_set_gemm_tile
+  int pair;                     // GEMMs may run as CTA pairs
   int attn_target_items, attn_min_chunk;   // attention plan: items aimed at per launch, fewest KV tiles per slice
   int n_sms;
   int device;
@@ -290,7 +291,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         g.qkv.k_pool_layer = kv.k_pool + (size_t)l * layer_elems;
         g.qkv.v_pool_layer = kv.v_pool + (size_t)l * layer_elems;
         g.qkv.Hq = md.Hq; g.qkv.Hkv = md.Hkv;
-        g.status = w.status; g.n_sms = c->n_sms; g.max_splits = 1; g.pdl = c->pdl;
+        g.status = w.status; g.n_sms = c->n_sms; g.max_splits = 1; g.pdl = c->pdl; g.pair = c->pair;
         g.force_bn = c->force_bn;
         if (launch_gemm_sm100(st, g)) return fail_cuda(c);
       }
@@ -310,7 +311,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         g.tmB = &c->tm_o[l];
         g.tmC = tm_x_add;
         g.M = T; g.n_out = md.d; g.K = md.Hq * md.D; g.mode = GS_ADD_F32;
-        g.status = w.status; g.n_sms = c->n_sms; g.max_splits = c->max_splits; g.pdl = c->pdl;
+        g.status = w.status; g.n_sms = c->n_sms; g.max_splits = c->max_splits; g.pdl = c->pdl; g.pair = c->pair;
         if (launch_gemm_sm100(st, g)) return fail_cuda(c);
       }
     }
@@ -337,7 +338,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         g.tmB = &c->tm_gate_up[l];
         g.tmC = tm_act_st;
         g.M = T; g.n_out = 2 * md.ffn; g.K = md.d; g.mode = GS_SWIGLU;
-        g.status = w.status; g.n_sms = c->n_sms; g.max_splits = 1; g.pdl = c->pdl;
+        g.status = w.status; g.n_sms = c->n_sms; g.max_splits = 1; g.pdl = c->pdl; g.pair = c->pair;
         if (launch_gemm_sm100(st, g)) return fail_cuda(c);
       }
       {
@@ -347,7 +348,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         g.tmB = &c->tm_down[l];
         g.tmC = tm_x_add;
         g.M = T; g.n_out = md.d; g.K = md.ffn; g.mode = GS_ADD_F32;
-        g.status = w.status; g.n_sms = c->n_sms; g.max_splits = c->max_splits; g.pdl = c->pdl;
+        g.status = w.status; g.n_sms = c->n_sms; g.max_splits = c->max_splits; g.pdl = c->pdl; g.pair = c->pair;
         if (launch_gemm_sm100(st, g)) return fail_cuda(c);
       }
     }
@@ -374,7 +375,7 @@ int run_lm_head(hsd_ctx* c, const Ws& w, int rows, const int* row_next, cudaStre
     g.tmB = &c->tm_lm_head;
     g.M = rows; g.n_out = md.V; g.K = md.d; g.mode = GS_ARGMAX;
     g.out = o;
-    g.status = w.status; g.n_sms = c->n_sms; g.max_splits = 1; g.pdl = c->pdl;
+    g.status = w.status; g.n_sms = c->n_sms; g.max_splits = 1; g.pdl = c->pdl; g.pair = c->pair;
     if (launch_gemm_sm100(st, g)) return fail_cuda(c);
   }
   return check_cuda(c);
@@ -489,6 +490,7 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
   c->max_splits = (cfg->flags & HSD_FLAG_DETERMINISTIC) ? 1 : 8;
   c->pdl = (cfg->flags & HSD_FLAG_NO_PDL) == 0;
   c->force_bn = c->force_splits = 0;
+  c->pair = 0;
   c->attn_target_items = 2 * c->n_sms;   // one item per CTA slot: slicing costs a partial hand-over per slice
   c->attn_min_chunk = 16;
   c->last_cuda_error = 0;
@@ -764,7 +766,7 @@ static int lm_head_argmax_impl(hsd_ctx* c, const void* h, int rows, const int* n
       g.tmB = &c->tm_lm_head;
       g.M = rows; g.n_out = md.V; g.K = md.d; g.mode = GS_ARGMAX;
       g.out = o;
-      g.status = nullptr; g.n_sms = c->n_sms; g.max_splits = 1; g.pdl = false;
+      g.status = nullptr; g.n_sms = c->n_sms; g.max_splits = 1; g.pdl = false; g.pair = c->pair;
       if (launch_gemm_sm100(st, g)) return fail_cuda(c);
     }
   }
@@ -844,7 +846,7 @@ int hsd_op_linear(hsd_ctx* c, const void* A, const void* W, void* C, int M, int 
   if (mode == 1 ? make_tmap_2d_f32(&g.tmC, C, M, ldc, 32) : make_tmap_2d(&g.tmC, C, M, ldc, 32)) return HSD_ERR_CUDA;
   g.tmB = &wm;
   g.M = M; g.n_out = n_out; g.K = K; g.mode = mode;
-  g.status = nullptr; g.n_sms = c->n_sms; g.max_splits = c->max_splits; g.pdl = false;
+  g.status = nullptr; g.n_sms = c->n_sms; g.max_splits = c->max_splits; g.pdl = false; g.pair = c->pair;
   g.force_bn = c->force_bn; g.force_splits = c->force_splits;
   if (launch_gemm_sm100(st, g)) return fail_cuda(c);
   return check_cuda(c);

@@ -92,11 +92,12 @@ constexpr int kGemmThreads = 256;
 constexpr int STG_BYTES = 4096;                  // one epilogue staging buffer: 32 rows x 128 bytes
 constexpr int STG_TOTAL = 4 * 2 * STG_BYTES;     // four epilogue warps, two buffers each
 
-template <int BN>
+// PAIR: two CTAs (a cluster) share one 256 x BN tile: each stages its own 128 rows of A and BN/2 rows of B.
+template <int BN, bool PAIR = false>
 struct Cfg {
-  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int B_BYTES = (PAIR ? BN / 2 : BN) * BK * 2;     // bytes of B this CTA stages per k-block
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
+  static constexpr int STAGES = PAIR ? 6 : ((BN == 256) ? 4 : (BN == 128 ? 6 : 8));
   static constexpr int TMEM_COLS = 2 * BN;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STG_TOTAL + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
@@ -140,13 +141,17 @@ __device__ __forceinline__ uint4 pack8(const uint32_t* r) {
   return o;
 }
 
-template <int BN, int MODE>
+template <int BN, int MODE, bool PAIR>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const __grid_constant__ CUtensorMap tmC, GemmDev p) {
-  using C = Cfg<BN>;
+  using C = Cfg<BN, PAIR>;
   constexpr int OUT_N = (MODE == GS_SWIGLU) ? BN / 2 : BN;   // output columns per tile
   constexpr int HALF_B = BN / 2 * BK * 2;                    // bytes of one weight half-tile
+  constexpr int TILE_M = PAIR ? 2 * BM : BM;                 // rows of one work unit (both CTAs of a pair)
+  const int rank = PAIR ? (int)cluster_ctarank() : 0;        // 0 = the CTA that issues the MMAs
+  const int cta = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // index among the unit walkers
+  const int n_cta = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* stg = smem + C::STAGES * C::STAGE_BYTES;
@@ -161,12 +166,13 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::STAGES; ++s) {
-      mbar_init(full + s, 3);      // A producer + two B producers, each with its own byte count
+      // A producer + two B producers, each with its own byte count; a pair: one arrival (even CTA) for all bytes
+      mbar_init(full + s, PAIR ? 1 : 3);
       mbar_init(empty + s, 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull + b, 1);
-      mbar_init(tempty + b, 4);
+      mbar_init(tempty + b, PAIR ? 8 : 4);     // the epilogue warps of both CTAs release the even CTA's MMA thread
     }
     *abort_flag = 0;
     fence_mbar_init();
@@ -175,15 +181,21 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     if (MODE != GS_ARGMAX) tma_prefetch_desc(&tmC);
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, C::TMEM_COLS);
-    tmem_relinquish();
+    if (PAIR) {
+      tmem_alloc_pair(tmem_slot, C::TMEM_COLS);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc(tmem_slot, C::TMEM_COLS);
+      tmem_relinquish();
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync();          // both CTAs' barriers exist before either one's loads complete on them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int m_tiles = (p.M + BM - 1) / BM;
+  const int m_tiles = (p.M + TILE_M - 1) / TILE_M;
   const int n_tiles = p.n_cols / OUT_N;
   const int tiles = m_tiles * n_tiles;
   const int total = tiles * p.splits;
@@ -196,44 +208,54 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       pdl_launch_dependents();
       int s = 0;
       uint32_t ph = 0;
-      for (int t = blockIdx.x; t < total; t += gridDim.x) {
+      for (int t = cta; t < total; t += n_cta) {
         const int tile = t % tiles, split = t / tiles;
-        const int m0 = (tile % m_tiles) * BM;
+        const int m0 = (tile % m_tiles) * TILE_M + rank * BM;
         const int kb0 = split * p.kb_per_split, kb1 = min(k_blocks, kb0 + p.kb_per_split);
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty + s, ph ^ 1u, abort_flag, p.status, 100)) goto done;
-          mbar_expect_tx(full + s, A_BYTES);
-          tma_load_2d(smem + s * C::STAGE_BYTES, &tmA, full + s, kb * BK, m0);
+          if (PAIR) {
+            if (rank == 0) mbar_expect_tx(full + s, 2 * C::STAGE_BYTES);   // A and B of both CTAs land on this barrier
+            tma_load_2d_pair(smem + s * C::STAGE_BYTES, &tmA, full + s, kb * BK, m0);
+          } else {
+            mbar_expect_tx(full + s, A_BYTES);
+            tma_load_2d(smem + s * C::STAGE_BYTES, &tmA, full + s, kb * BK, m0);
+          }
           if (++s == C::STAGES) { s = 0; ph ^= 1u; }
         }
       }
     }
   } else if (warp == 2 || warp == 3) {
     // ---- B producers: one half of the weight tile each (for SwiGLU: gate rows / up rows)
-    if (lane == 0) {
-      const int half = warp - 2;
+    if (lane == 0 && !(PAIR && warp == 3)) {
+      // a pair: this CTA stages half `rank` of the tile in one box; alone: warps 2 and 3 stage one half each
+      const int half = PAIR ? rank : warp - 2;
       int s = 0;
       uint32_t ph = 0;
-      for (int t = blockIdx.x; t < total; t += gridDim.x) {
+      for (int t = cta; t < total; t += n_cta) {
         const int tile = t % tiles, split = t / tiles;
         const int n0 = (tile / m_tiles) * OUT_N;
         const int kb0 = split * p.kb_per_split, kb1 = min(k_blocks, kb0 + p.kb_per_split);
         const int row = (MODE == GS_SWIGLU) ? (half ? p.n_up_off + n0 : n0) : n0 + half * (BN / 2);
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty + s, ph ^ 1u, abort_flag, p.status, 110 + half)) goto done;
-          mbar_expect_tx(full + s, HALF_B);
-          tma_load_2d(smem + s * C::STAGE_BYTES + A_BYTES + half * HALF_B, &tmB, full + s, kb * BK, row);
+          if (PAIR) {
+            tma_load_2d_pair(smem + s * C::STAGE_BYTES + A_BYTES, &tmB, full + s, kb * BK, row);
+          } else {
+            mbar_expect_tx(full + s, HALF_B);
+            tma_load_2d(smem + s * C::STAGE_BYTES + A_BYTES + half * HALF_B, &tmB, full + s, kb * BK, row);
+          }
           if (++s == C::STAGES) { s = 0; ph ^= 1u; }
         }
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(BN);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(BN, false, TILE_M);
       int s = 0;
       uint32_t ph = 0;
       int it = 0;
-      for (int t = blockIdx.x; t < total; t += gridDim.x, ++it) {
+      for (int t = cta; t < total; t += n_cta, ++it) {
         const int split = t / tiles;
         const int kb0 = split * p.kb_per_split, kb1 = min(k_blocks, kb0 + p.kb_per_split);
         const int b = it & 1;
@@ -248,13 +270,15 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           const uint32_t sb = sa + A_BYTES;
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k) {
-            umma_bf16(d_tmem, umma_desc_sw128(sa + k * 32), umma_desc_sw128(sb + k * 32), idesc,
-                      (kb != kb0 || k != 0) ? 1u : 0u);
+            const uint32_t acc = (kb != kb0 || k != 0) ? 1u : 0u;
+            if (PAIR) umma_bf16_pair(d_tmem, umma_desc_sw128(sa + k * 32), umma_desc_sw128(sb + k * 32), idesc, acc);
+            else umma_bf16(d_tmem, umma_desc_sw128(sa + k * 32), umma_desc_sw128(sb + k * 32), idesc, acc);
           }
-          umma_commit(empty + s);      // smem stage reusable once these MMAs have read it
+          // smem stage reusable once these MMAs have read it (in both CTAs of a pair)
+          if (PAIR) umma_commit_pair(empty + s); else umma_commit(empty + s);
           if (++s == C::STAGES) { s = 0; ph ^= 1u; }
         }
-        umma_commit(tfull + b);        // accumulator complete
+        if (PAIR) umma_commit_pair(tfull + b); else umma_commit(tfull + b);   // accumulator complete
       }
     }
   } else {
@@ -265,11 +289,11 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     int n_stores = 0;                             // staging buffers handed to TMA so far (selects the buffer)
     pdl_wait();
     int it = 0;
-    for (int t = blockIdx.x; t < total; t += gridDim.x, ++it) {
+    for (int t = cta; t < total; t += n_cta, ++it) {
       const int b = it & 1;
       const uint32_t aph = (it >> 1) & 1;
       const int tile = t % tiles;
-      const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * OUT_N;
+      const int m0 = (tile % m_tiles) * TILE_M + rank * BM, n0 = (tile / m_tiles) * OUT_N;
       const int row = m0 + row_in_tile;
       const bool row_ok = row < p.M;
       const int wrow0 = m0 + quarter * 32;        // first row of this warp's 32-row slab
@@ -441,7 +465,9 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty + b);
+      if (lane == 0) {
+        if (PAIR) mbar_arrive_even_cta(tempty + b); else mbar_arrive(tempty + b);
+      }
     }
     if (lane == 0) bulk_wait_all();               // staged rows have reached global memory
   }
@@ -449,21 +475,22 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 done:
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync();                // the other CTA's loads, MMAs and arrivals no longer touch this one
   if (warp == 1) {
     if (*abort_flag) __nanosleep(20000);   // let copies / MMAs in flight drain before TMEM goes away
-    tmem_dealloc(tmem_base, C::TMEM_COLS);
+    if (PAIR) tmem_dealloc_pair(tmem_base, C::TMEM_COLS); else tmem_dealloc(tmem_base, C::TMEM_COLS);
   }
 }
 
 // ------------------------------------------------------------------------------------------------
-template <int BN, int MODE>
+template <int BN, int MODE, bool PAIR>
 static int launch_one(cudaStream_t st, const GemmSm100Args& a, int splits) {
-  using C = Cfg<BN>;
+  using C = Cfg<BN, PAIR>;
   constexpr int OUT_N = (MODE == GS_SWIGLU) ? BN / 2 : BN;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm_sm100_kernel<BN, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) !=
-        cudaSuccess)
+    if (cudaFuncSetAttribute(gemm_sm100_kernel<BN, MODE, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             C::SMEM_BYTES) != cudaSuccess)
       return -1;
     attr_set = true;
   }
@@ -478,38 +505,65 @@ static int launch_one(cudaStream_t st, const GemmSm100Args& a, int splits) {
   p.out = a.out;
   p.qkv = a.qkv;
   p.status = a.status;
-  const int m_tiles = (a.M + BM - 1) / BM;
+  const int tile_m = PAIR ? 2 * BM : BM;
+  const int m_tiles = (a.M + tile_m - 1) / tile_m;
   const int total = m_tiles * (p.n_cols / OUT_N) * splits;
-  const int grid = total < a.n_sms ? total : a.n_sms;
-  const CUtensorMap& tmB = a.tmB->m[BN == 64 ? 0 : (BN == 128 ? 1 : 2)];
-  return launch_kernel(gemm_sm100_kernel<BN, MODE>, dim3(grid), dim3(kGemmThreads), C::SMEM_BYTES, st, a.pdl, a.tmA, tmB,
-                       a.tmC, p);
+  const int walkers = PAIR ? a.n_sms / 2 : a.n_sms;
+  const int grid = (total < walkers ? total : walkers) * (PAIR ? 2 : 1);
+  const CUtensorMap& tmB = a.tmB->m[PAIR ? 2 : (BN == 64 ? 0 : (BN == 128 ? 1 : 2))];   // pair: one 128-row box per CTA
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kGemmThreads);
+  cfg.dynamicSmemBytes = C::SMEM_BYTES;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  int n_attr = 0;
+  if (a.pdl) {
+    attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+    ++n_attr;
+  }
+  if (PAIR) {
+    attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+    attr[n_attr].val.clusterDim.x = 2;
+    attr[n_attr].val.clusterDim.y = 1;
+    attr[n_attr].val.clusterDim.z = 1;
+    ++n_attr;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n_attr;
+  return cudaLaunchKernelEx(&cfg, gemm_sm100_kernel<BN, MODE, PAIR>, a.tmA, tmB, a.tmC, p) == cudaSuccess ? 0 : -1;
 }
 
-// Tile width and K slices: fewest cycles by a simple model.  A k-block of a 128 x BN tile is bound by the
-// ~64 bytes per clock an SM gets from L2 (16 KB of A + 128 BN bytes of B), not by the MMA (2 BN clocks);
-// the epilogue of the last unit of a CTA is exposed.
-static void pick_tile(int mode, int n_cols, int M, int K, int n_sms, int max_splits, int* bn_out, int* splits_out) {
-  const int m_tiles = (M + BM - 1) / BM;
+// Tile width, CTA pairing and K slices: fewest cycles by a simple model.  A k-block of a 128 x BN tile is bound by
+// the ~64 bytes per clock an SM gets from L2 (16 KB of A + 128 BN bytes of B), not by the MMA (2 BN clocks); in a
+// CTA pair each SM stages 16 KB of A and half of a 256-row B tile, which balances the two.  The epilogue of the
+// last unit of a CTA is exposed.
+static void pick_tile(int mode, int n_cols, int M, int K, int n_sms, int max_splits, bool allow_pair, int* bn_out,
+                      int* splits_out, bool* pair_out) {
   const int k_blocks = K / BK;
-  const int cands[3] = {256, 128, 64};
+  const int cands[4] = {256, 256, 128, 64};     // first entry: a CTA pair on a 256 x 256 tile
   double best_cost = 1e30;
   *bn_out = (mode == GS_SWIGLU) ? 128 : 64;
   *splits_out = 1;
-  for (int i = 0; i < 3; ++i) {
+  *pair_out = false;
+  for (int i = allow_pair ? 0 : 1; i < 4; ++i) {
+    const bool pair = i == 0;
     const int bn = cands[i];
     const int out_n = (mode == GS_SWIGLU) ? bn / 2 : bn;
     if (n_cols % out_n || out_n % 64) continue;
-    const long long tiles = (long long)m_tiles * (n_cols / out_n);
+    const int tile_m = pair ? 2 * BM : BM;
+    const int walkers = pair ? n_sms / 2 : n_sms;
+    const long long tiles = (long long)((M + tile_m - 1) / tile_m) * (n_cols / out_n);
     for (int sp = 1; sp <= max_splits; ++sp) {
       const int kbs = (k_blocks + sp - 1) / sp;
       if (sp > 1 && (kbs < 4 || (long long)(sp - 1) * kbs >= k_blocks)) continue;
       const long long units = tiles * sp;
-      const long long rounds = (units + n_sms - 1) / n_sms;
-      const double per_kb = 256.0 + 2.0 * bn;
+      const long long rounds = (units + walkers - 1) / walkers;
+      const double per_kb = pair ? 2.0 * bn + 32.0 : 256.0 + 2.0 * bn;
       const double epi = 700.0 + 10.0 * bn;
       const double cost = (double)rounds * (kbs * per_kb + 300.0) + epi + (sp > 1 ? 200.0 * sp : 0.0);
-      if (cost < best_cost) { best_cost = cost; *bn_out = bn; *splits_out = sp; }
+      if (cost < best_cost) { best_cost = cost; *bn_out = bn; *splits_out = sp; *pair_out = pair; }
     }
   }
 }
@@ -518,23 +572,28 @@ template <int MODE>
 static int launch_mode(cudaStream_t st, const GemmSm100Args& a) {
   const int n_cols = (MODE == GS_SWIGLU) ? a.n_out / 2 : a.n_out;
   int bn = 64, splits = 1;
-  pick_tile(MODE, n_cols, a.M, a.K, a.n_sms, (MODE == GS_ADD_F32 && a.max_splits > 1) ? a.max_splits : 1, &bn, &splits);
+  bool pair = false;
+  pick_tile(MODE, n_cols, a.M, a.K, a.n_sms, (MODE == GS_ADD_F32 && a.max_splits > 1) ? a.max_splits : 1, a.pair != 0, &bn,
+            &splits, &pair);
   if (a.force_bn) {
-    const int out_n = (MODE == GS_SWIGLU) ? a.force_bn / 2 : a.force_bn;
-    if ((a.force_bn != 64 && a.force_bn != 128 && a.force_bn != 256) || out_n % 64 || n_cols % out_n) return -1;
-    bn = a.force_bn;
+    const int fbn = a.force_bn == 512 ? 256 : a.force_bn;       // 512 = a CTA pair on 256-column tiles
+    const int out_n = (MODE == GS_SWIGLU) ? fbn / 2 : fbn;
+    if ((fbn != 64 && fbn != 128 && fbn != 256) || out_n % 64 || n_cols % out_n) return -1;
+    bn = fbn;
+    pair = a.force_bn == 512;
   }
   if (a.force_splits) {
     const int kbs = (a.K / BK + a.force_splits - 1) / a.force_splits;
     if (MODE != GS_ADD_F32 || (a.force_splits - 1) * kbs >= a.K / BK) return -1;
     splits = a.force_splits;
   }
+  if (pair) return launch_one<256, MODE, true>(st, a, splits);
   switch (bn) {
-    case 256: return launch_one<256, MODE>(st, a, splits);
-    case 128: return launch_one<128, MODE>(st, a, splits);
+    case 256: return launch_one<256, MODE, false>(st, a, splits);
+    case 128: return launch_one<128, MODE, false>(st, a, splits);
     default:
-      if (MODE == GS_SWIGLU) return launch_one<128, MODE>(st, a, splits);
-      return launch_one<64, MODE>(st, a, splits);
+      if (MODE == GS_SWIGLU) return launch_one<128, MODE, false>(st, a, splits);
+      return launch_one<64, MODE, false>(st, a, splits);
   }
 }
 

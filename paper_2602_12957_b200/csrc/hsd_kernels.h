@@ -160,7 +160,8 @@ struct GemmSm100Args {
   int n_sms;
   int max_splits;              // GS_ADD_F32: most K slices per tile (1 = none; slices add in arrival order)
   bool pdl;                    // launch with programmatic stream serialization
-  int force_bn, force_splits;  // tests: tile width / K slices to use instead of the model's choice (0 = choose)
+  int pair;                    // CTA pairs (clusters of two sharing a 256-row tile) may be used
+  int force_bn, force_splits;  // tests: tile width (512 = CTA pair) / K slices instead of the model's choice (0 = choose)
 };
 enum GemmSm100Mode { GS_STORE_BF16 = 0, GS_ADD_F32 = 1, GS_SWIGLU = 2, GS_ARGMAX = 4, GS_QKV_ROPE = 5 };
 int launch_gemm_sm100(cudaStream_t st, const GemmSm100Args& a);
