@@ -73,6 +73,7 @@ extern "C" {
 #define HSD_FLAG_DETERMINISTIC 4   /* no split-K in the residual-add projections: their K slices add into
                                       the fp32 residual in arrival order, so results can differ in the last
                                       bit from run to run; with this flag every run is bit-identical      */
+#define HSD_FLAG_NO_PAIR 16        /* debugging: no CTA-pair (cluster of two) GEMM tiles                        */
 #define HSD_FLAG_NO_PDL 8          /* debugging: plain stream-ordered launches (no programmatic dependent
                                       launch overlap between consecutive kernels)                       */
 

@@ -490,7 +490,7 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
   c->max_splits = (cfg->flags & HSD_FLAG_DETERMINISTIC) ? 1 : 8;
   c->pdl = (cfg->flags & HSD_FLAG_NO_PDL) == 0;
   c->force_bn = c->force_splits = 0;
-  c->pair = 0;
+  c->pair = (cfg->flags & HSD_FLAG_NO_PAIR) == 0;
   c->attn_target_items = 2 * c->n_sms;   // one item per CTA slot: slicing costs a partial hand-over per slice
   c->attn_min_chunk = 16;
   c->last_cuda_error = 0;

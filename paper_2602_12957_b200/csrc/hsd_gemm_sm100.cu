@@ -201,18 +201,24 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const int total = tiles * p.splits;
   const int k_blocks = p.K / BK;
 
+  // Producer warps: lanes 0 and 1 each take every other stage (kc counts k-blocks over all units of this CTA;
+  // the stage count is even, so a lane always sees the same stages).  One thread cannot issue TMA instructions
+  // faster than about one per 0.25 us, and a barrier round trip adds to that; two lanes per operand keep the
+  // issue interval below the 128 x 256 MMA time of a k-block.
   if (warp == 0) {
     // ---- A producer: activations, written by the previous kernel
-    if (lane == 0) {
+    if (lane < 2) {
       pdl_wait();
-      pdl_launch_dependents();
-      int s = 0;
-      uint32_t ph = 0;
+      if (lane == 0) pdl_launch_dependents();
+      int kc = 0;
       for (int t = cta; t < total; t += n_cta) {
         const int tile = t % tiles, split = t / tiles;
         const int m0 = (tile % m_tiles) * TILE_M + rank * BM;
         const int kb0 = split * p.kb_per_split, kb1 = min(k_blocks, kb0 + p.kb_per_split);
-        for (int kb = kb0; kb < kb1; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb, ++kc) {
+          if ((kc & 1) != lane) continue;
+          const int s = kc % C::STAGES;
+          const uint32_t ph = (kc / C::STAGES) & 1;
           if (!mbar_wait(empty + s, ph ^ 1u, abort_flag, p.status, 100)) goto done;
           if (PAIR) {
             if (rank == 0) mbar_expect_tx(full + s, 2 * C::STAGE_BYTES);   // A and B of both CTAs land on this barrier
@@ -221,23 +227,24 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             mbar_expect_tx(full + s, A_BYTES);
             tma_load_2d(smem + s * C::STAGE_BYTES, &tmA, full + s, kb * BK, m0);
           }
-          if (++s == C::STAGES) { s = 0; ph ^= 1u; }
         }
       }
     }
   } else if (warp == 2 || warp == 3) {
     // ---- B producers: one half of the weight tile each (for SwiGLU: gate rows / up rows)
-    if (lane == 0 && !(PAIR && warp == 3)) {
+    if (lane < 2 && !(PAIR && warp == 3)) {
       // a pair: this CTA stages half `rank` of the tile in one box; alone: warps 2 and 3 stage one half each
       const int half = PAIR ? rank : warp - 2;
-      int s = 0;
-      uint32_t ph = 0;
+      int kc = 0;
       for (int t = cta; t < total; t += n_cta) {
         const int tile = t % tiles, split = t / tiles;
         const int n0 = (tile / m_tiles) * OUT_N;
         const int kb0 = split * p.kb_per_split, kb1 = min(k_blocks, kb0 + p.kb_per_split);
         const int row = (MODE == GS_SWIGLU) ? (half ? p.n_up_off + n0 : n0) : n0 + half * (BN / 2);
-        for (int kb = kb0; kb < kb1; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb, ++kc) {
+          if ((kc & 1) != lane) continue;
+          const int s = kc % C::STAGES;
+          const uint32_t ph = (kc / C::STAGES) & 1;
           if (!mbar_wait(empty + s, ph ^ 1u, abort_flag, p.status, 110 + half)) goto done;
           if (PAIR) {
             tma_load_2d_pair(smem + s * C::STAGE_BYTES + A_BYTES, &tmB, full + s, kb * BK, row);
@@ -245,7 +252,6 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             mbar_expect_tx(full + s, HALF_B);
             tma_load_2d(smem + s * C::STAGE_BYTES + A_BYTES + half * HALF_B, &tmB, full + s, kb * BK, row);
           }
-          if (++s == C::STAGES) { s = 0; ph ^= 1u; }
         }
       }
     }
@@ -535,10 +541,11 @@ static int launch_one(cudaStream_t st, const GemmSm100Args& a, int splits) {
   return cudaLaunchKernelEx(&cfg, gemm_sm100_kernel<BN, MODE, PAIR>, a.tmA, tmB, a.tmC, p) == cudaSuccess ? 0 : -1;
 }
 
-// Tile width, CTA pairing and K slices: fewest cycles by a simple model.  A k-block of a 128 x BN tile is bound by
-// the ~64 bytes per clock an SM gets from L2 (16 KB of A + 128 BN bytes of B), not by the MMA (2 BN clocks); in a
-// CTA pair each SM stages 16 KB of A and half of a 256-row B tile, which balances the two.  The epilogue of the
-// last unit of a CTA is exposed.
+// Tile width, CTA pairing and K slices: fewest cycles by a model calibrated on B200 (cycles per k-block of one work
+// unit, measured in steady state: 128 x 256 tile ~820, 128 x 128 ~700, 128 x 64 ~600, CTA pair on 256 x 256 ~770 per
+// CTA for twice the rows).  None of them reaches the 512 clocks the MMAs of a 256-column tile take: the pipeline is
+// bound by the round trip stage-free -> TMA issue -> data -> MMA over the few stages shared memory holds.  A pair
+// costs a cluster launch; the epilogue of the last unit of a CTA is exposed.
 static void pick_tile(int mode, int n_cols, int M, int K, int n_sms, int max_splits, bool allow_pair, int* bn_out,
                       int* splits_out, bool* pair_out) {
   const int k_blocks = K / BK;
@@ -560,9 +567,9 @@ static void pick_tile(int mode, int n_cols, int M, int K, int n_sms, int max_spl
       if (sp > 1 && (kbs < 4 || (long long)(sp - 1) * kbs >= k_blocks)) continue;
       const long long units = tiles * sp;
       const long long rounds = (units + walkers - 1) / walkers;
-      const double per_kb = pair ? 2.0 * bn + 32.0 : 256.0 + 2.0 * bn;
+      const double per_kb = pair ? 770.0 : (bn == 256 ? 820.0 : (bn == 128 ? 700.0 : 600.0));
       const double epi = 700.0 + 10.0 * bn;
-      const double cost = (double)rounds * (kbs * per_kb + 300.0) + epi + (sp > 1 ? 200.0 * sp : 0.0);
+      const double cost = (double)rounds * (kbs * per_kb + 300.0) + epi + (sp > 1 ? 200.0 * sp : 0.0) + (pair ? 1500.0 : 0.0);
       if (cost < best_cost) { best_cost = cost; *bn_out = bn; *splits_out = sp; *pair_out = pair; }
     }
   }

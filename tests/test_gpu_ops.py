@@ -106,7 +106,7 @@ def test_lm_head_argmax_matches_float64(models, flags, rows):
 @pytest.mark.parametrize("shape", [(513, 8192, 128), (1323, 2048, 192), (513, 2048, 1024), (1323, 1024, 4096)])
 @pytest.mark.parametrize("mode", [0, 1, 2])
 def test_linear_every_tile_width_and_k_slicing(models, mode, shape):
-    """Every tile width (64/128/256) and, for the residual-add epilogue, 1 to 8 slices of K, on shapes whose last
+    """Every tile width (64/128/256 and the CTA pair) and, for the residual-add epilogue, 1 to 8 slices of K, on shapes whose last
     row tile is mostly beyond M and whose K loop is short (the epilogue, not the main loop, sets the pace, so
     several staged stores are in flight per warp).  Repeated, because a staging-buffer race shows up only sometimes."""
     import torch
@@ -125,7 +125,7 @@ def test_linear_every_tile_width_and_k_slicing(models, mode, shape):
         ref = g / (1.0 + np.exp(-g)) * u
     st = torch.cuda.current_stream().cuda_stream
     try:
-        for bn in (64, 128, 256):
+        for bn in (64, 128, 256, 512):       # 512 = a pair of CTAs on a 256 x 256 tile
             if mode == 2 and bn == 64:
                 continue
             for sp in ((1, 2, 3, 4, 8) if mode == 1 else (0,)):
