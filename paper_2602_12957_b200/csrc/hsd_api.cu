@@ -112,6 +112,7 @@ Ws carve(const hsd_ctx* c, void* base, int T, int S) {
   {
     const int mt = attn_max_tiles(md, T, S);
     w.plan.items = static_cast<int4*>(take(sizeof(int4) * 2 * (size_t)mt * kAttnMaxSplits));
+    w.plan.items_unsorted = static_cast<int4*>(take(sizeof(int4) * 2 * (size_t)mt * kAttnMaxSplits));
     w.plan.tile_seq = static_cast<int*>(take(sizeof(int) * mt));
     w.plan.tile_nkv = static_cast<int*>(take(sizeof(int) * mt));
     w.plan.counters = static_cast<int*>(take(sizeof(int) * (size_t)mt * md.Hkv));

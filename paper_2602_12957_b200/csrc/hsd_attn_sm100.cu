@@ -90,6 +90,7 @@ __global__ void attn_plan_kernel(RowMeta rm, AttnPlan pl, int n_seqs, int tokens
   }
   atomicAdd(&s_total, my);
   __syncthreads();
+  __shared__ int s_n;
   if (threadIdx.x == 0) {
     const int chunk = max(min_chunk, (s_total + target_items - 1) / max(1, target_items));
     int n = 0;
@@ -102,14 +103,29 @@ __global__ void attn_plan_kernel(RowMeta rm, AttnPlan pl, int n_seqs, int tokens
       int lo = 0;
       for (int k = 0; k < ns; ++k) {
         const int len = base + (k < rem ? 1 : 0);
-        pl.items[2 * n] = make_int4(rm.seq_q0[s] + tok0, rm.seq_len[s] + tok0, min(tokens_per_tile, rm.seq_n[s] - tok0),
-                                    rm.seq_slot[s]);
-        pl.items[2 * n + 1] = make_int4(lo | ((lo + len) << 16), k | (ns << 16), t, 0);
+        pl.items_unsorted[2 * n] = make_int4(rm.seq_q0[s] + tok0, rm.seq_len[s] + tok0,
+                                             min(tokens_per_tile, rm.seq_n[s] - tok0), rm.seq_slot[s]);
+        pl.items_unsorted[2 * n + 1] = make_int4(lo | ((lo + len) << 16), k | (ns << 16), t, len);
         ++n;
         lo += len;
       }
     }
     *pl.n_items = n;
+    s_n = n;
+  }
+  __syncthreads();
+  // longest first (rank sort, ties by creation order): the attention CTAs walk the list in boustrophedon order, so
+  // every CTA's share of KV tiles comes out about equal
+  const int n = s_n;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const int len = pl.items_unsorted[2 * i + 1].w;
+    int rank = 0;
+    for (int k = 0; k < n; ++k) {
+      const int lk = pl.items_unsorted[2 * k + 1].w;
+      rank += (lk > len) || (lk == len && k < i);
+    }
+    pl.items[2 * rank] = pl.items_unsorted[2 * i];
+    pl.items[2 * rank + 1] = pl.items_unsorted[2 * i + 1];
   }
   // slice-arrival counters of every (q-tile, kv head): zero at the start of a step, reset by the combiner
   for (int i = threadIdx.x; i < n_tiles * pl.n_kv_heads; i += blockDim.x) pl.counters[i] = 0;
@@ -178,6 +194,14 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   pdl_launch_dependents();
 
   const int total = (*p.status) ? 0 : *p.plan.n_items * p.Hkv;
+  // Round r of the walk: CTA i takes item r G + i in even rounds and r G + (G - 1 - i) in odd ones (the list is
+  // sorted longest first, so the CTA that drew a long item in one round draws a short one in the next).
+  const int n_rounds = (total + (int)gridDim.x - 1) / (int)gridDim.x;
+  auto item_of_round = [&](int r) -> int {
+    const int i = (r & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x;
+    const int w = r * (int)gridDim.x + i;
+    return w < total ? w : -1;
+  };
 
   // Global tile counter g (all items of this CTA): S / P / PV buffer = g & 1, KV stage = g % KV_STAGES, and every
   // barrier's parity follows from how often g has used it; n counts items (Q hand-over barriers).
@@ -185,7 +209,9 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     if (lane == 0) {
       uint32_t g = 0;
       int n = 0;
-      for (int w = blockIdx.x; w < total; w += gridDim.x, ++n) {
+      for (int r = 0; r < n_rounds; ++r) {
+        const int w = item_of_round(r);
+        if (w < 0) continue;
         const int4 ia = p.plan.items[2 * (w / p.Hkv)], ib = p.plan.items[2 * (w / p.Hkv) + 1];
         const int kvh = w % p.Hkv;
         const int kt_lo = ib.x & 0xffff, kt_hi = ib.x >> 16;
@@ -205,6 +231,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           tma_load_2d(k_dst + KV_TILE_BYTES, &tmV, kv_full + st, 0, row);
           phys = phys_next;
         }
+        ++n;
       }
     }
   } else if (warp == 1) {
@@ -214,7 +241,9 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       const uint32_t q_addr = smem_u32(sQ);
       uint32_t g = 0;
       int n = 0;
-      for (int w = blockIdx.x; w < total; w += gridDim.x, ++n) {
+      for (int r = 0; r < n_rounds; ++r) {
+        const int w = item_of_round(r);
+        if (w < 0) continue;
         const int4 ib = p.plan.items[2 * (w / p.Hkv) + 1];
         const int n_it = (ib.x >> 16) - (ib.x & 0xffff);
         auto issue_s = [&](uint32_t gi) -> bool {
@@ -251,6 +280,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           umma_commit(kv_empty + st);
           umma_commit(pv_full + (g & 1));
         }
+        ++n;
       }
       // every stage-release arrival must land before the CTA's shared memory can be handed on
       if (g > 0 && !mbar_wait(pv_full + ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag, p.status, 414)) goto done;
@@ -262,7 +292,9 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const uint32_t t_lane = tmem_base + (uint32_t(quarter * 32) << 16);
     const float sc = 0.125f * 1.4426950408889634f;     // 1/sqrt(64) * log2(e)
     uint32_t g = 0, group_ph = 0;
-    for (int w = blockIdx.x; w < total; w += gridDim.x) {
+    for (int r = 0; r < n_rounds; ++r) {
+      const int w = item_of_round(r);
+      if (w < 0) continue;
       const int4 ia = p.plan.items[2 * (w / p.Hkv)], ib = p.plan.items[2 * (w / p.Hkv) + 1];
       const int kvh = w % p.Hkv;
       const int q_row0 = ia.x, pos0 = ia.y, n_tok = ia.z;
@@ -270,6 +302,10 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       const int split = ib.y & 0xffff, n_split = ib.y >> 16;
       const int pos_row = pos0 + tok;
       const bool row_ok = tok < n_tok;
+      // warp-uniform: some row of this warp is a real token.  A ragged last q-tile leaves whole warps without one;
+      // they keep step with the barriers but skip the loads, the exps and the P rows (which only feed their own,
+      // never stored, output rows)
+      const bool warp_ok = (quarter * 32) / p.group < n_tok;
       float m = -INFINITY, l = 0.f, alpha_prev = 1.f;
       float o[64];
 #pragma unroll
@@ -299,6 +335,13 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         bool ok = mbar_wait(s_full + b, (g >> 1) & 1, abort_flag, p.status, 420);
         if (!__all_sync(0xffffffffu, ok)) goto done;
         tc_fence_after();
+        if (!warp_ok) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(s_empty + b);
+          mbar_arrive(p_full + b);
+          continue;
+        }
         uint32_t s0[32], s1[32];
         tmem_ld32(t_lane + b * 64, s0);
         tmem_ld32(t_lane + b * 64 + 32, s1);
@@ -351,7 +394,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (j > kt_lo && !fold_pv(g - 1, 421)) goto done;
         alpha_prev = alpha;
       }
-      if (!fold_pv(g - 1, 422)) goto done;
+      if (warp_ok && !fold_pv(g - 1, 422)) goto done;
 
       // ---- item epilogue
       const int head = kvh * p.group + row % p.group;
@@ -368,7 +411,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         // partials of this (q-tile, kv head): [slice][66][128 rows] floats, entry 0 the running maximum (log2
         // units), 1 the row sum, 2.. the 64 unnormalised outputs; a warp's accesses are 128-byte lines
         float* tile_part = p.split_ws + ((size_t)(ib.z * p.Hkv + kvh) * kAttnMaxSplits) * (66 * 128) + row;
-        {
+        if (warp_ok) {
           float* part = tile_part + (size_t)split * (66 * 128);
           part[0] = m;
           part[128] = l;
@@ -384,7 +427,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           if (old == n_split - 1) *ctr = 0;             // ready for the next layer
         }
         if (!warps_sync(group_bar, group_ph, lane, abort_flag, p.status, 428)) goto done;
-        if (*s_flag) {
+        if (*s_flag && warp_ok) {
           __threadfence();
           float M = -INFINITY;
           for (int s = 0; s < n_split; ++s) M = fmaxf(M, __ldcg(tile_part + (size_t)s * (66 * 128)));

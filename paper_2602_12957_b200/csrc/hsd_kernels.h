@@ -100,8 +100,9 @@ void launch_unpack_best(cudaStream_t st, const unsigned long long* row_best, int
 // ---- attention plan (hsd_attn_sm100.cu): made once per step on the device, read by every layer's launch ----
 constexpr int kAttnMaxSplits = 8;      // most KV slices one q-tile is cut into
 struct AttnPlan {
-  int4* items;      // two int4 per (q-tile, slice) item: {first packed row, position of the first token, tokens, KV slot},
-                    // {first | (last + 1) << 16 KV tile, slice | slices << 16, q-tile, 0}
+  int4* items;      // two int4 per (q-tile, slice) item, longest first: {first packed row, position of the first
+                    // token, tokens, KV slot}, {first | (last + 1) << 16 KV tile, slice | slices << 16, q-tile, KV tiles}
+  int4* items_unsorted;   // the same list in creation order (scratch of the plan kernel)
   int* n_items;
   int* tile_seq;    // [max_tiles] sequence of a q-tile
   int* tile_nkv;    // [max_tiles] KV tiles it can see
