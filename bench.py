@@ -104,13 +104,41 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------------ workload
+WORKLOADS = {
+    "region": "region-level stage: 24-layer decoder d1024 16q/8kv x64 ffn4096 vocab32768, 16 regions per GPU, prefix "
+              "256-1024, lognormal drafts mean 64 (8-256), acceptance 0.8, paged KV block 64",
+    "page": "page-level stage, one chunk mid-schedule: batch 1, 6400 committed tokens, chunk of 512 draft tokens",
+    "long1024": "long-document page verify, one chunk mid-schedule: batch 1, 10240 committed tokens, chunk of 1024",
+    "long2048": "long-document page verify, one chunk mid-schedule: batch 1, 10240 committed tokens, chunk of 2048",
+    "mixed": "mixed serving batch: 64 regions (prefix 128-2048, lognormal drafts mean 96, 8-512) + 2 page chunks of 1024 "
+             "over 4352-token prefixes, one varlen launch",
+}
+
+
+def make_workload(args, rank):
+    """The seeded workload of this rank.  Region: planted drafts; the others (extra, not the default bench line):
+    random drafts, since kernel time does not depend on token values."""
+    cfg = I.DECODER
+    name = getattr(args, "workload", "region")
+    if name == "region":
+        return I.region_workload(seed=I.BASE_SEED + 1 + 1000 * rank, cfg=cfg)
+    args.random_drafts = True
+    if name == "mixed":
+        return I.mixed_workload(seed=I.BASE_SEED + 4 + 1000 * rank, cfg=cfg)
+    ctx, k = {"page": (6400, 512), "long1024": (10240, 1024), "long2048": (10240, 2048)}[name]
+    rng = np.random.Generator(np.random.PCG64(I.BASE_SEED + 2 + 1000 * rank))
+    emb = I.bf16_round(rng.standard_normal((ctx, cfg.d_model), dtype=np.float32))
+    seq = I.SeqInput(emb, np.full(ctx, -1, np.int32), k, k, rng.integers(0, cfg.vocab, size=k, dtype=np.int32), True)
+    return I.Workload(name, cfg, I.BASE_SEED + 2, [seq], chunk_len=k)
+
+
 def build_gpu_state(args, rank):
     import torch
     from paper_2602_12957_b200 import runtime as R
     cfg = I.DECODER
-    wl = I.region_workload(seed=I.BASE_SEED + 1 + 1000 * rank, cfg=cfg)
+    wl = make_workload(args, rank)
     weights = I.make_weights(cfg, I.BASE_SEED + 1)
-    model = R.DeviceModel(cfg, weights, 0, f"cuda:{torch.cuda.current_device()}")
+    model = R.DeviceModel(cfg, weights, getattr(args, "flags", 0), f"cuda:{torch.cuda.current_device()}")
     del weights
     seqs = wl.seqs
     S = len(seqs)
@@ -314,16 +342,14 @@ def run_ours(args):
                  "bound": "tensor" if work.flops / pk > work.bytes / bw else "hbm"}
 
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and args.workload == "region":
         cpu = cpu_baseline_sample(st["wl"], budget_s=20.0)
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": "region-level stage: 24-layer decoder d1024 16q/8kv x64 ffn4096 vocab32768, "
-                                       "16 regions per GPU, prefix 256-1024, lognormal drafts mean 64 (8-256), "
-                                       "acceptance 0.8, paged KV block 64",
+                "config": {"workload": WORKLOADS[args.workload],
                            "regions_per_gpu": S, "query_rows_per_gpu": T, "draft_tokens_per_gpu": draft_tokens,
                            "context_tokens_per_gpu": int(sum(ctx_lens)), "mean_acceptance_rate": accept_mean,
                            "planted_acceptance_rate": float(np.mean([s.agree_len / s.draft_len for s in st["wl"].seqs])),
@@ -395,6 +421,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="region", choices=sorted(WORKLOADS),
+                    help="region = the benchmark line; the others time one step of the other configurations")
+    ap.add_argument("--flags", type=int, default=0, help="HSD_FLAG_* bits for the context (debugging / ablations)")
     ap.add_argument("--random-drafts", action="store_true",
                     help="skip the greedy-continuation pass that plants agreement (for profiler captures)")
     args = ap.parse_args()
