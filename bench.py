@@ -304,7 +304,8 @@ def run_ours(args):
     e2e = {"value": draft_tokens * world / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
            "h2d_bytes_per_step": int(h_toks.numel() * 4 + h_cu.numel() * 4),
            "d2h_bytes_per_step": int((h_acc.numel() + h_nem.numel() + h_emit.numel()) * 4 + 16),
-           "call": "hsd_verify_regions_host (eager launches, pinned host buffers, stream synchronised per step)"}
+           "call": "hsd_verify_regions_host (pinned host buffers; the library replays the step as a CUDA graph it captured "
+                   "at the second call of this shape; stream synchronised per step)"}
     accept_mean = float(np.mean([a / k for a, k in zip(h_acc.numpy().tolist(), st["ks"])]))
 
     # ---- per-kernel durations (CUDA events around every launch, eager) for the roofline of the top kernel

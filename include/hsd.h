@@ -74,6 +74,7 @@ extern "C" {
                                       the fp32 residual in arrival order, so results can differ in the last
                                       bit from run to run; with this flag every run is bit-identical      */
 #define HSD_FLAG_NO_PAIR 16        /* debugging: no CTA-pair (cluster of two) GEMM tiles                        */
+#define HSD_FLAG_NO_HOST_GRAPH 32  /* hsd_verify_regions_host launches its kernels one by one, never as a CUDA graph */
 #define HSD_FLAG_NO_PDL 8          /* debugging: plain stream-ordered launches (no programmatic dependent
                                       launch overlap between consecutive kernels)                       */
 
@@ -180,6 +181,11 @@ HSD_API int hsd_kv_commit(hsd_ctx *ctx, const hsd_kv *kv, int n_seqs, const int 
  *                         returned through max_q_len_out (may be NULL); the buffer must hold n_seqs * max_q_len ints
  * Copies the inputs into staging areas inside `workspace`, runs the step on the stream, copies the results back and
  * SYNCHRONISES the stream before returning; a device-side check that tripped is returned as HSD_ERR_DEVICE_CHECK.
+ * The transfers go through pinned staging owned by the context.  When the same call shape (every argument but the
+ * contents of cu_q / q_tokens, with equal n_seqs, total and longest query length) comes a second time on a stream
+ * other than the default one, the whole step is captured once into a CUDA graph and replayed from then on, which
+ * removes the per-kernel launch cost from the decode loop (HSD_FLAG_NO_HOST_GRAPH turns this off).  The caller
+ * must not be capturing the stream itself.
  * Errors otherwise as hsd_verify_regions. */
 HSD_API int hsd_verify_regions_host(hsd_ctx *ctx, const hsd_kv *kv, int n_seqs, const int *cu_q, const int *q_tokens,
                             const int *seq_slots, float log_tau, int commit, int *accept_len, int *emit_tokens,

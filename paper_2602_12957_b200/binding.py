@@ -23,6 +23,7 @@ HSD_FLAG_SIMT_ATTENTION = 2
 HSD_FLAG_DETERMINISTIC = 4
 HSD_FLAG_NO_PDL = 8
 HSD_FLAG_NO_PAIR = 16
+HSD_FLAG_NO_HOST_GRAPH = 32
 HSD_NOALLOC_MAX_ROWS = 8192
 
 EXPORTS = [

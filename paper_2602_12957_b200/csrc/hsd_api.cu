@@ -15,6 +15,19 @@ struct ProfEvent {
   cudaEvent_t a, b;
 };
 
+// Everything a call of hsd_verify_regions_host bakes into its launches, by value: two calls with equal keys enqueue
+// identical work (only the contents of the staged inputs differ), so the second one can replay the first one's graph.
+struct HostCallKey {
+  hsd_kv kv;
+  const int* seq_slots;
+  void* workspace;
+  size_t ws_bytes;
+  void* stream;
+  int n_seqs, total_q, max_q, commit;
+  float log_tau;
+  int pad;
+};
+
 struct hsd_ctx {
   hsd_model_config cfg;
   ModelDims md;
@@ -34,6 +47,14 @@ struct hsd_ctx {
   int last_cuda_error;
   long long launches;
   bool profiling;
+  // hsd_verify_regions_host: pinned staging and the cached graph of the last repeated call shape
+  bool host_graph_ok;
+  int* pin;
+  size_t pin_ints;
+  HostCallKey hg_key, hg_seen;
+  bool hg_seen_valid;
+  cudaGraphExec_t hg_exec;
+  long long hg_launches;
   std::vector<ProfEvent> prof_events;
   std::vector<cudaEvent_t> event_pool;
   double prof_ms[KC_COUNT];
@@ -492,6 +513,12 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
   c->pdl = (cfg->flags & HSD_FLAG_NO_PDL) == 0;
   c->force_bn = c->force_splits = 0;
   c->pair = (cfg->flags & HSD_FLAG_NO_PAIR) == 0;
+  c->host_graph_ok = (cfg->flags & HSD_FLAG_NO_HOST_GRAPH) == 0;
+  c->pin = nullptr;
+  c->pin_ints = 0;
+  c->hg_seen_valid = false;
+  c->hg_exec = nullptr;
+  c->hg_launches = 0;
   c->attn_target_items = 2 * c->n_sms;   // one item per CTA slot: slicing costs a partial hand-over per slice
   c->attn_min_chunk = 16;
   c->last_cuda_error = 0;
@@ -521,6 +548,8 @@ int hsd_destroy(hsd_ctx* c) {
   if (!c) return HSD_ERR_INVALID_ARG;
   for (auto& e : c->prof_events) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
   for (auto& e : c->event_pool) cudaEventDestroy(e);
+  if (c->hg_exec) cudaGraphExecDestroy(c->hg_exec);
+  if (c->pin) cudaFreeHost(c->pin);
   delete c;
   return HSD_OK;
 }
@@ -638,7 +667,7 @@ int hsd_kv_commit(hsd_ctx* c, const hsd_kv* kv, int n_seqs, const int* seq_slots
 int hsd_verify_regions_host(hsd_ctx* c, const hsd_kv* kv, int n_seqs, const int* cu_q, const int* q_tokens,
                             const int* seq_slots, float log_tau, int commit, int* accept_len, int* emit_tokens,
                             int* n_emit, int* max_q_len_out, void* workspace, size_t ws_bytes, void* cuda_stream) {
-  if (!c || !cu_q || !q_tokens || !accept_len || !emit_tokens || !n_emit || n_seqs <= 0) return HSD_ERR_INVALID_ARG;
+  if (!c || !kv || !cu_q || !q_tokens || !accept_len || !emit_tokens || !n_emit || n_seqs <= 0) return HSD_ERR_INVALID_ARG;
   if (cu_q[0] != 0) return HSD_ERR_INVALID_ARG;
   int max_q = 0;
   for (int i = 0; i < n_seqs; ++i) {
@@ -651,28 +680,102 @@ int hsd_verify_regions_host(hsd_ctx* c, const hsd_kv* kv, int n_seqs, const int*
   int rc = check_ws(c, workspace, ws_bytes, total_q, n_seqs);
   if (rc) return rc;
   const Ws w = carve(c, workspace, total_q, n_seqs);
-  if ((size_t)n_seqs * max_q > w.h_emit_ints) return HSD_ERR_WORKSPACE;
+  const size_t emit_ints = (size_t)n_seqs * max_q;
+  if (emit_ints > w.h_emit_ints) return HSD_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  if (cudaMemcpyAsync(w.h_cu, cu_q, sizeof(int) * (n_seqs + 1), cudaMemcpyHostToDevice, st) != cudaSuccess ||
-      cudaMemcpyAsync(w.h_tokens, q_tokens, sizeof(int) * total_q, cudaMemcpyHostToDevice, st) != cudaSuccess)
-    return fail_cuda(c);
-  rc = hsd_verify_regions(c, kv, n_seqs, w.h_cu, w.h_tokens, seq_slots, max_q, total_q, log_tau, w.h_accept, w.h_emit,
-                          w.h_nemit, nullptr, nullptr, nullptr, workspace, ws_bytes, cuda_stream);
-  if (rc) return rc;
-  if (commit) {
-    rc = hsd_kv_commit(c, kv, n_seqs, seq_slots, w.h_accept, nullptr, cuda_stream);
-    if (rc) return rc;
+
+  // pinned staging: [cu_q | q_tokens | accept_len | n_emit | status words | emit_tokens]
+  const size_t need = (size_t)(n_seqs + 1) + total_q + 2 * (size_t)n_seqs + 4 + emit_ints;
+  if (need > c->pin_ints) {
+    if (c->hg_exec) { cudaGraphExecDestroy(c->hg_exec); c->hg_exec = nullptr; }   // it names the old staging
+    c->hg_seen_valid = false;
+    if (c->pin) cudaFreeHost(c->pin);
+    c->pin = nullptr;
+    c->pin_ints = 0;
+    if (cudaHostAlloc(reinterpret_cast<void**>(&c->pin), need * sizeof(int), cudaHostAllocDefault) != cudaSuccess)
+      return fail_cuda(c);
+    c->pin_ints = need;
   }
-  if (cudaMemcpyAsync(accept_len, w.h_accept, sizeof(int) * n_seqs, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-      cudaMemcpyAsync(n_emit, w.h_nemit, sizeof(int) * n_seqs, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-      cudaMemcpyAsync(emit_tokens, w.h_emit, sizeof(int) * (size_t)n_seqs * max_q, cudaMemcpyDeviceToHost, st) !=
-          cudaSuccess ||
-      cudaStreamSynchronize(st) != cudaSuccess)
-    return fail_cuda(c);
+  int* p_cu = c->pin;
+  int* p_tok = p_cu + n_seqs + 1;
+  int* p_acc = p_tok + total_q;
+  int* p_nem = p_acc + n_seqs;
+  int* p_status = p_nem + n_seqs;
+  int* p_emit = p_status + 4;
+  memcpy(p_cu, cu_q, sizeof(int) * (n_seqs + 1));
+  memcpy(p_tok, q_tokens, sizeof(int) * total_q);
+
+  HostCallKey key;
+  memset(&key, 0, sizeof(key));
+  key.kv = *kv;
+  key.seq_slots = seq_slots;
+  key.workspace = workspace;
+  key.ws_bytes = ws_bytes;
+  key.stream = cuda_stream;
+  key.n_seqs = n_seqs;
+  key.total_q = total_q;
+  key.max_q = max_q;
+  key.commit = commit != 0;
+  key.log_tau = log_tau;
+
+  // the whole step on the stream: inputs in, verify (+ commit), results and status words out
+  auto enqueue = [&]() -> int {
+    if (cudaMemcpyAsync(w.h_cu, p_cu, sizeof(int) * (n_seqs + 1), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(w.h_tokens, p_tok, sizeof(int) * total_q, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return fail_cuda(c);
+    int r = hsd_verify_regions(c, kv, n_seqs, w.h_cu, w.h_tokens, seq_slots, max_q, total_q, log_tau, w.h_accept,
+                               w.h_emit, w.h_nemit, nullptr, nullptr, nullptr, workspace, ws_bytes, cuda_stream);
+    if (r) return r;
+    if (commit) {
+      r = hsd_kv_commit(c, kv, n_seqs, seq_slots, w.h_accept, nullptr, cuda_stream);
+      if (r) return r;
+    }
+    if (cudaMemcpyAsync(p_acc, w.h_accept, sizeof(int) * n_seqs, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemcpyAsync(p_nem, w.h_nemit, sizeof(int) * n_seqs, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemcpyAsync(p_emit, w.h_emit, sizeof(int) * emit_ints, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemcpyAsync(p_status, workspace, sizeof(int) * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+      return fail_cuda(c);
+    return HSD_OK;
+  };
+
+  const bool graph_stream = c->host_graph_ok && !c->profiling && st != nullptr && st != cudaStreamLegacy &&
+                            st != cudaStreamPerThread;
+  if (graph_stream && c->hg_exec && memcmp(&key, &c->hg_key, sizeof(key)) == 0) {
+    if (cudaGraphLaunch(c->hg_exec, st) != cudaSuccess) return fail_cuda(c);
+    c->launches += c->hg_launches;
+  } else if (graph_stream && c->hg_seen_valid && memcmp(&key, &c->hg_seen, sizeof(key)) == 0) {
+    // second call of this shape (the first one ran eagerly and set every one-time kernel attribute): capture it
+    if (c->hg_exec) { cudaGraphExecDestroy(c->hg_exec); c->hg_exec = nullptr; }
+    if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return fail_cuda(c);
+    const long long before = c->launches;
+    rc = enqueue();
+    cudaGraph_t graph = nullptr;
+    const cudaError_t end = cudaStreamEndCapture(st, &graph);
+    c->hg_launches = c->launches - before;
+    c->launches = before;
+    if (rc || end != cudaSuccess || !graph) {
+      if (graph) cudaGraphDestroy(graph);
+      c->hg_seen_valid = false;
+      return rc ? rc : fail_cuda(c);
+    }
+    const cudaError_t inst = cudaGraphInstantiate(&c->hg_exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (inst != cudaSuccess) { c->hg_exec = nullptr; c->hg_seen_valid = false; return fail_cuda(c); }
+    c->hg_key = key;
+    if (cudaGraphLaunch(c->hg_exec, st) != cudaSuccess) return fail_cuda(c);
+    c->launches += c->hg_launches;
+  } else {
+    rc = enqueue();
+    if (rc) return rc;
+    c->hg_seen = key;
+    c->hg_seen_valid = true;
+  }
+  if (cudaStreamSynchronize(st) != cudaSuccess) return fail_cuda(c);
+  memcpy(accept_len, p_acc, sizeof(int) * n_seqs);
+  memcpy(n_emit, p_nem, sizeof(int) * n_seqs);
+  memcpy(emit_tokens, p_emit, sizeof(int) * emit_ints);
   if (max_q_len_out) *max_q_len_out = max_q;
-  int status[4];
-  if (cudaMemcpy(status, workspace, sizeof(status), cudaMemcpyDeviceToHost) != cudaSuccess) return fail_cuda(c);
-  return status[0] ? HSD_ERR_DEVICE_CHECK : HSD_OK;
+  return p_status[0] ? HSD_ERR_DEVICE_CHECK : HSD_OK;
 }
 
 int hsd_device_status(hsd_ctx* c, const void* workspace, void* cuda_stream, int status[4]) {

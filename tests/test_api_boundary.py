@@ -51,7 +51,7 @@ def test_status_strings(B):
 def test_constants_match_the_header(B):
     text = open(HEADER).read()
     for name in ("HSD_MAX_Q_LEN", "HSD_KV_BLOCK", "HSD_NOALLOC_MAX_ROWS", "HSD_FLAG_SIMT_DEBUG", "HSD_FLAG_SIMT_ATTENTION",
-                 "HSD_FLAG_DETERMINISTIC", "HSD_FLAG_NO_PDL", "HSD_FLAG_NO_PAIR"):
+                 "HSD_FLAG_DETERMINISTIC", "HSD_FLAG_NO_PDL", "HSD_FLAG_NO_PAIR", "HSD_FLAG_NO_HOST_GRAPH"):
         m = re.search(rf"#define\s+{name}\s+(-?\d+)", text)
         assert m and int(m.group(1)) == getattr(B, name), name
     for name in ("INVALID_ARG", "SHAPE", "TOO_LONG", "WORKSPACE", "KV_CAPACITY", "CUDA", "DEVICE_CHECK", "NO_DEVICE"):

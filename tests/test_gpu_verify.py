@@ -92,6 +92,63 @@ def test_one_verify_call_equals_sequential_single_token_steps_on_gpu():
     assert o["accept_len"].cpu().numpy().tolist() == [k] * S
 
 
+def test_host_buffer_call_replays_a_captured_graph_with_fresh_inputs():
+    """On a side stream the host-buffer entry captures the step into a CUDA graph at the second call of one shape and
+    replays it afterwards.  Every call (eager, capturing, replayed) must give the integers of the plain device call,
+    also when the token values (hence accept lengths) change between calls, and account the same number of launches."""
+    import torch
+    from paper_2602_12957_b200 import binding as B
+    wl = I.tiny_workload()
+    weights = I.make_weights(wl.cfg, wl.seed)
+    orc = H.oracle_regions(wl, weights, np.float64)
+    per, eng, (toks, cu, total_q) = H.gpu_regions(wl, weights, {i: o.pending for i, o in orc.items()},
+                                                  {i: o.draft for i, o in orc.items()}, B.HSD_FLAG_DETERMINISTIC)
+    S = len(orc)
+    ctx = eng.model.ctx
+    max_q = int(np.diff(cu).max())
+    lens0 = eng.kv.seq_lens.clone()
+    side = torch.cuda.Stream()
+    rng = np.random.default_rng(11)
+    variants = [toks.copy()]
+    for _ in range(3):                                   # same shape, other draft tokens after the pending one
+        v = toks.copy()
+        for i in range(S):
+            lo, hi = int(cu[i]) + 1, int(cu[i + 1])
+            if hi > lo:
+                cut = int(rng.integers(lo, hi))
+                v[cut:hi] = rng.integers(0, wl.cfg.vocab, hi - cut)
+        variants.append(v)
+    variants.append(toks.copy())
+    h_cu = torch.from_numpy(cu).pin_memory()
+    counts = []
+    for v in variants:
+        # plain device call on the same inputs (no commit), as the expected integers
+        d_t, d_c = eng._i32(v), eng._i32(cu)
+        out = eng.verify_regions(d_t, d_c, max_q, total_q)
+        torch.cuda.synchronize()
+        exp_acc = out["accept_len"].cpu().numpy()
+        exp_emit = out["emit_tokens"].cpu().numpy().reshape(S, -1)
+        h_toks = torch.from_numpy(v).pin_memory()
+        h_acc = torch.full((S,), -7, dtype=torch.int32).pin_memory()
+        h_nem = torch.full((S,), -7, dtype=torch.int32).pin_memory()
+        h_emit = torch.full((S, max_q), -7, dtype=torch.int32).pin_memory()
+        n0 = B.hsd_launch_count(ctx)
+        rc, mq = B.hsd_verify_regions_host(ctx, eng.kv.c, S, h_cu, h_toks, None, 0.0, 1, h_acc, h_emit, h_nem,
+                                           eng.ws.ptr, eng.ws.bytes, side.cuda_stream)
+        B.check(rc, "hsd_verify_regions_host")
+        counts.append(B.hsd_launch_count(ctx) - n0)
+        assert mq == max_q
+        assert h_acc.numpy().tolist() == exp_acc.tolist()
+        assert h_nem.numpy().tolist() == (exp_acc + 1).tolist()
+        for j in range(S):
+            a = int(exp_acc[j])
+            assert h_emit[j, :a + 1].tolist() == exp_emit[j, :a + 1].tolist()
+        assert (eng.kv.seq_lens - lens0).cpu().numpy().tolist() == (exp_acc + 1).tolist()   # the commit ran
+        eng.kv.seq_lens.copy_(lens0)
+        torch.cuda.synchronize()
+    assert len(set(counts)) == 1 and counts[0] > 0, counts
+
+
 def test_host_buffer_call_matches_the_device_call_and_commits():
     """hsd_verify_regions_host (host buffers in, host buffers out, commit folded in) against hsd_verify_regions +
     hsd_kv_commit on the same inputs: identical integers, and the committed lengths advance by accept_len + 1."""
