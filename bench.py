@@ -36,7 +36,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM traffic per launch of the dominant kernel classes, from the ncu captures summarised under profiles/
 # (dram__bytes_read.sum + dram__bytes_write.sum); None where no capture exists yet.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {"attention": 30.96e6, "gemm_gate_up": 19.52e6, "gemm_qkv": 7.28e6, "gemm_o": 10.25e6,
+                     "gemm_down": 24.67e6}     # region workload only
 
 
 def load_peaks():
@@ -335,7 +336,7 @@ def run_ours(args):
     else:
         roof = {"kernel": top, "bound": "hbm", "achieved": nbytes / dur / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = NCU_TRAFFIC_BYTES.get(top)
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get(top) if args.workload == "region" else None
     roof["peak_source"] = f"{peak_src} (sustained bf16 figure: kernel timed inside a long step)"
     roof["us_per_launch"] = dur * 1e6
     t_roof = RF.roofline_time(work.bytes, work.flops, bw, pk)
