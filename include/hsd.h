@@ -64,6 +64,7 @@ extern "C" {
 #define HSD_ERR_NO_DEVICE (-8)     /* no usable sm_100 device                                         */
 
 #define HSD_MAX_Q_LEN 4097         /* most query rows one sequence may have in a verify call          */
+#define HSD_MAX_TREE_ROWS 128      /* most rows (root included) of one sequence in hsd_verify_tree    */
 #define HSD_KV_BLOCK 64
 
 /* hsd_model_config.flags */
@@ -164,6 +165,38 @@ HSD_API int hsd_verify_page(hsd_ctx *ctx, const hsd_kv *kv, int seq_slot, const 
                     int *n_emit, int *row_argmax, float *row_zmax, float *row_zdraft, void *workspace,
                     size_t ws_bytes, void *cuda_stream);
 
+/* One verification step over candidate TREES (Sec. 3.2: prefix tree T of Eq. 7 packed into one sequence, the
+ * tree-ancestry mask of Fig. 2(c), greedy traversal of Eq. 9-12).  Per sequence the packed rows are
+ * [pending token (the root), node 1, .., node k] in an order that puts every parent before its children;
+ *   parent          dev int32 [total_q]: the parent's row index WITHIN the sequence, -1 for row 0
+ *   max_q_len       at most HSD_MAX_TREE_ROWS rows per sequence (root included; the paper packs <= 128 tokens)
+ * A node's rotary position is committed length + depth; it attends to the committed context, itself and its
+ * ancestors.  Traversal from the root: at node s, u_hat = argmax over the vocabulary (lowest id on ties), u* = the
+ * child of s with the highest logit (log_tau = 0: the child that carries u_hat); move to it iff
+ * z[u*] - z[u_hat] >= log_tau; stop when the test fails or s is a leaf; emitted = tokens of the path, then u_hat.
+ *   accept_len      dev int32 [n_seqs] out: length of the accepted path
+ *   emit_tokens     dev int32 [n_seqs, max_q_len] out, n_emit = accept_len + 1
+ *   accept_rows     dev int32 [n_seqs, max_q_len] out: rows of the accepted path after the root
+ *   row_argmax, row_zmax   dev [total_q] out or NULL, as in hsd_verify_regions
+ *   row_zchild      dev fp32 [total_q] out or NULL: the logit of the row's own token under its parent's
+ *                   distribution (NaN on row 0)
+ * The K/V rows of ALL nodes are written at cache rows committed length + row index; hsd_kv_commit_tree keeps the
+ * accepted ones.  The workspace must be sized for 2 * total_q rows (the LM head evaluates every node once for its
+ * argmax and once more, through its parent, for its own token).  A parent pointer that does not name an earlier row
+ * sets device status 7 and turns the step into a no-op.  Errors otherwise as hsd_verify_regions; contexts created
+ * with a SIMT debug flag return HSD_ERR_INVALID_ARG. */
+HSD_API int hsd_verify_tree(hsd_ctx *ctx, const hsd_kv *kv, int n_seqs, const int *cu_q, const int *q_tokens,
+                    const int *parent, const int *seq_slots, int max_q_len, int total_q, float log_tau,
+                    int *accept_len, int *emit_tokens, int *n_emit, int *accept_rows, int *row_argmax, float *row_zmax,
+                    float *row_zchild, void *workspace, size_t ws_bytes, void *cuda_stream);
+
+/* KV maintenance after hsd_verify_tree (Sec. 4.2 counts it in the decode loop): in every layer the K/V rows of the
+ * accepted path move from cache rows L + accept_rows[i][d-1] to rows L + d (d = 1..accept_len[i]; L = committed
+ * length; the values already carry the rotary position L + d), then seq_lens[slot_i] += accept_len[i] + 1.
+ * blocks_in_use as in hsd_kv_commit. */
+HSD_API int hsd_kv_commit_tree(hsd_ctx *ctx, const hsd_kv *kv, int n_seqs, const int *seq_slots, const int *accept_len,
+                       const int *accept_rows, int max_q_len, int *blocks_in_use, void *cuda_stream);
+
 /* KV maintenance after a step: seq_lens[slot_i] += accept_len[i] + 1 (the pending row and the accepted
  * draft rows stay; rows after them are rolled back and will be overwritten by the next step).  The caller
  * may pass lengths other than the ones verify produced.  blocks_in_use (dev int32 [n_seqs] or NULL)
@@ -193,7 +226,8 @@ HSD_API int hsd_verify_regions_host(hsd_ctx *ctx, const hsd_kv *kv, int n_seqs, 
 
 /* Device status words written by the last call that used `workspace` (synchronises the stream).
  * status[0] = 0 if every device-side check passed, else a code (1 cu_q not monotone, 2 sequence too long,
- * 3 token id out of range, 4 KV capacity, 5 block table entry out of range, 6 a bounded wait gave up);
+ * 3 token id out of range, 4 KV capacity, 5 block table entry out of range, 6 a bounded wait gave up,
+ * 7 a tree's parent pointer does not name an earlier row of its sequence);
  * status[1] = index of the offending sequence or row. */
 HSD_API int hsd_device_status(hsd_ctx *ctx, const void *workspace, void *cuda_stream, int status[4]);
 

@@ -113,6 +113,9 @@ Ws carve(const hsd_ctx* c, void* base, int T, int S) {
   w.rm.seq_len = static_cast<int*>(take(sizeof(int) * S));
   w.rm.seq_slot = static_cast<int*>(take(sizeof(int) * S));
   w.rm.seq_tile0 = static_cast<int*>(take(sizeof(int) * (S + 1)));
+  w.rm.anc = static_cast<uint4*>(take(sizeof(uint4) * T));
+  w.rm.lm_src = static_cast<int*>(take(sizeof(int) * T));        // a tree call carves for 2 x its rows
+  w.rm.lm_next = static_cast<int*>(take(sizeof(int) * T));
   w.sel_rows = static_cast<int*>(take(sizeof(int) * S));
   w.cu_one = static_cast<int*>(take(sizeof(int) * 2));
   w.h_tokens = static_cast<int*>(take(sizeof(int) * T));
@@ -216,6 +219,7 @@ struct StepArgs {
   const void* embeds;
   const int* seq_slots;
   int slot_base;
+  const int* parent;   // candidate trees: parent row within the sequence, or nullptr (chains)
 };
 
 // The decoder forward over one packed batch: rows -> residual stream x after the last layer.
@@ -239,6 +243,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
     sa.pending = a.pending;
     sa.draft = a.draft;
     sa.seq_slots = a.seq_slots;
+    sa.parent = a.parent;
     sa.slot_base = a.slot_base;
     sa.allow_embed_rows = a.prefill && a.embeds != nullptr;
     sa.rope_base = md.rope_base;
@@ -322,7 +327,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         if (c->attn_simt) {
           launch_attn_simt(st, w.q, w.rm, kv, md, l, w.attn, T, w.status);
         } else if (launch_attn_sm100(st, tm_q, tm_k, tm_v, w.plan, kv, md, l, w.attn, c->n_sms, w.status, w.split_ws,
-                                     c->pdl)) {
+                                     a.parent ? w.rm.anc : nullptr, c->pdl)) {
           return fail_cuda(c);
         }
       }
@@ -610,6 +615,68 @@ int hsd_verify_regions(hsd_ctx* c, const hsd_kv* kv, int n_seqs, const int* cu_q
   a.cu_q = cu_q; a.tokens = q_tokens; a.seq_slots = seq_slots; a.slot_base = 0;
   return verify_common(c, kv, a, log_tau, accept_len, emit_tokens, n_emit, row_argmax, row_zmax, row_zdraft, workspace,
                        ws_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int hsd_verify_tree(hsd_ctx* c, const hsd_kv* kv, int n_seqs, const int* cu_q, const int* q_tokens, const int* parent,
+                    const int* seq_slots, int max_q_len, int total_q, float log_tau, int* accept_len, int* emit_tokens,
+                    int* n_emit, int* accept_rows, int* row_argmax, float* row_zmax, float* row_zchild, void* workspace,
+                    size_t ws_bytes, void* cuda_stream) {
+  if (!c || !cu_q || !q_tokens || !parent || !accept_len || !emit_tokens || !n_emit || !accept_rows)
+    return HSD_ERR_INVALID_ARG;
+  if (n_seqs <= 0 || total_q <= 0 || max_q_len <= 0 || max_q_len > total_q) return HSD_ERR_INVALID_ARG;
+  if (!(log_tau <= 0.f)) return HSD_ERR_INVALID_ARG;
+  if (max_q_len > HSD_MAX_TREE_ROWS) return HSD_ERR_TOO_LONG;
+  if (c->simt || c->attn_simt) return HSD_ERR_INVALID_ARG;   // the plain debug kernels know chains only
+  int rc = check_kv(kv);
+  if (rc) return rc;
+  if ((long long)max_q_len > (long long)kv->max_blocks_per_seq * HSD_KV_BLOCK) return HSD_ERR_KV_CAPACITY;
+  // the LM head runs over 2 x total_q rows (every node, and every node's parent for the node's own token)
+  rc = check_ws(c, workspace, ws_bytes, 2 * total_q, n_seqs);
+  if (rc) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const Ws w = carve(c, workspace, 2 * total_q, n_seqs);
+  StepArgs a = {};
+  a.n_seqs = n_seqs; a.total_q = total_q; a.max_q_len = max_q_len; a.prefill = false;
+  a.cu_q = cu_q; a.tokens = q_tokens; a.seq_slots = seq_slots; a.slot_base = 0; a.parent = parent;
+  rc = run_layers(c, kv, a, w, st);
+  if (rc) return rc;
+  {
+    Scope s(c, st, KC_RMSNORM);
+    launch_rmsnorm(st, w.x, c->final_norm, w.h, 2 * total_q, c->md.d, c->md.eps, w.rm.lm_src, c->pdl);
+  }
+  rc = run_lm_head(c, w, 2 * total_q, w.rm.lm_next, st);
+  if (rc) return rc;
+  {
+    Scope s(c, st, KC_ACCEPT);
+    TreeAcceptArgs ta;
+    ta.n_seqs = n_seqs; ta.max_q_len = max_q_len; ta.total_q = total_q; ta.log_tau = log_tau;
+    ta.parent = parent;
+    ta.row_best = w.row_best;
+    ta.zdraft = w.zdraft;
+    ta.accept_len = accept_len; ta.emit_tokens = emit_tokens; ta.n_emit = n_emit; ta.accept_rows = accept_rows;
+    ta.row_argmax = row_argmax; ta.row_zmax = row_zmax; ta.row_zchild = row_zchild;
+    launch_tree_accept(st, ta, w.rm, w.status, c->pdl);
+  }
+  return check_cuda(c);
+}
+
+int hsd_kv_commit_tree(hsd_ctx* c, const hsd_kv* kv, int n_seqs, const int* seq_slots, const int* accept_len,
+                       const int* accept_rows, int max_q_len, int* blocks_in_use, void* cuda_stream) {
+  if (!c || !accept_len || !accept_rows || n_seqs <= 0 || max_q_len <= 0 || max_q_len > HSD_MAX_TREE_ROWS)
+    return HSD_ERR_INVALID_ARG;
+  int rc = check_kv(kv);
+  if (rc) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  {
+    Scope s(c, st, KC_COMMIT);
+    launch_tree_compact(st, kv_view(kv), c->md.n_layers, c->md.Hkv, n_seqs, seq_slots, accept_len, accept_rows, max_q_len,
+                        c->pdl);
+  }
+  {
+    Scope s(c, st, KC_COMMIT);
+    launch_commit(st, kv_view(kv), n_seqs, seq_slots, accept_len, blocks_in_use, c->pdl);
+  }
+  return check_cuda(c);
 }
 
 }  // extern "C"

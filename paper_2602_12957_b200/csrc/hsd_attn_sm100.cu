@@ -37,6 +37,7 @@ struct AttnParams {
   int max_blocks, n_blocks, Hq, Hkv, group, layer;
   bf16* out;            // [T, Hq*64]
   float* split_ws;      // partials of sliced items: [q-tile][kv head][slice][2 + 64][128 rows]
+  const uint4* anc;     // [T] ancestry masks of candidate-tree rows, or nullptr: plain causal order within the call
   int* status;
 };
 
@@ -105,7 +106,7 @@ __global__ void attn_plan_kernel(RowMeta rm, AttnPlan pl, int n_seqs, int tokens
         const int len = base + (k < rem ? 1 : 0);
         pl.items_unsorted[2 * n] = make_int4(rm.seq_q0[s] + tok0, rm.seq_len[s] + tok0,
                                              min(tokens_per_tile, rm.seq_n[s] - tok0), rm.seq_slot[s]);
-        pl.items_unsorted[2 * n + 1] = make_int4(lo | ((lo + len) << 16), k | (ns << 16), t, len);
+        pl.items_unsorted[2 * n + 1] = make_int4(lo | ((lo + len) << 16), k | (ns << 8) | (tok0 << 16), t, len);
         ++n;
         lo += len;
       }
@@ -299,9 +300,14 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       const int kvh = w % p.Hkv;
       const int q_row0 = ia.x, pos0 = ia.y, n_tok = ia.z;
       const int kt_lo = ib.x & 0xffff, kt_hi = ib.x >> 16;
-      const int split = ib.y & 0xffff, n_split = ib.y >> 16;
+      const int split = ib.y & 0xff, n_split = (ib.y >> 8) & 0xff;
       const int pos_row = pos0 + tok;
       const bool row_ok = tok < n_tok;
+      // candidate trees (Sec. 3.2, Fig. 2(c)): a row sees the committed context and, of the rows of this call, only
+      // itself and its ancestors.  len0 = committed length; the mask's bit i stands for cache row len0 + i.
+      const int len0 = pos0 - (ib.y >> 16);
+      uint4 am = make_uint4(0u, 0u, 0u, 0u);
+      if (p.anc && row_ok) am = p.anc[q_row0 + tok];
       // warp-uniform: some row of this warp is a real token.  A ragged last q-tile leaves whole warps without one;
       // they keep step with the barriers but skip the loads, the exps and the P rows (which only feed their own,
       // never stored, output rows)
@@ -351,7 +357,27 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (lane == 0) mbar_arrive(s_empty + b);
 
         const int kbase = j * 64;
-        if (kbase + 63 > pos0) {                          // some row of the tile masks part of this KV tile
+        if (p.anc) {
+          if (kbase + 63 >= len0) {                       // the tile holds rows of this call
+            // 32 bits of the row's visibility string from key position `pos` on: ones below the committed length,
+            // the ancestry mask over the call's rows, zeros beyond them
+            auto word = [&](int i) -> uint32_t {
+              return i < 0 ? 0xffffffffu : i == 0 ? am.x : i == 1 ? am.y : i == 2 ? am.z : i == 3 ? am.w : 0u;
+            };
+            auto vis32 = [&](int pos) -> uint32_t {
+              if (pos <= -32) return 0xffffffffu;
+              if (pos >= 128) return 0u;
+              const int wi = pos >> 5;                    // floor, also for negative positions
+              return __funnelshift_r(word(wi), word(wi + 1), pos & 31);
+            };
+            const uint32_t v0 = vis32(kbase - len0), v1 = vis32(kbase - len0 + 32);
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              if (!((v0 >> e) & 1u)) s0[e] = 0xff800000u;          // -inf
+              if (!((v1 >> e) & 1u)) s1[e] = 0xff800000u;
+            }
+          }
+        } else if (kbase + 63 > pos0) {                   // some row of the tile masks part of this KV tile
 #pragma unroll
           for (int e = 0; e < 32; ++e) {
             if (kbase + e > pos_row) s0[e] = 0xff800000u;          // -inf
@@ -468,7 +494,7 @@ done:
 
 int launch_attn_sm100(cudaStream_t st, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                       const AttnPlan& plan, const KvView& kv, const ModelDims& md, int layer, bf16* out, int n_sms,
-                      int* status, float* split_ws, bool pdl) {
+                      int* status, float* split_ws, const uint4* anc, bool pdl) {
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(attn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_SMEM) != cudaSuccess)
@@ -486,6 +512,7 @@ int launch_attn_sm100(cudaStream_t st, const CUtensorMap& tmQ, const CUtensorMap
   p.layer = layer;
   p.out = out;
   p.split_ws = split_ws;
+  p.anc = anc;
   p.status = status;
   return launch_kernel(attn_sm100_kernel, dim3(2 * n_sms), dim3(kAttnThreads), ATTN_SMEM, st, pdl, tmQ, tmK, tmV, p);
 }

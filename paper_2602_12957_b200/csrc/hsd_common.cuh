@@ -21,6 +21,7 @@ enum DevStatus : int {
   DEV_KV_CAPACITY = 4,
   DEV_BLOCK_RANGE = 5,
   DEV_WAIT_TIMEOUT = 6,
+  DEV_TREE = 7,            // parent pointers of a candidate tree do not point to earlier rows of the sequence
 };
 
 __device__ __forceinline__ void dev_fail(int* status, int code, int where) {
@@ -40,6 +41,10 @@ struct RowMeta {
   int* seq_len;     // [S] committed length before the call
   int* seq_slot;    // [S] KV slot
   int* seq_tile0;   // [S+1] first attention q-tile of the sequence (exclusive scan)
+  // candidate trees (Sec. 3.2, Eq. 7): written only by calls that pass parent pointers
+  uint4* anc;       // [T] ancestry bit mask: bit i set iff row i of the sequence is the row itself or an ancestor
+  int* lm_src;      // [2T] source row of every LM-head row: [0, T) the rows themselves, [T, 2T) each row's parent
+  int* lm_next;     // [2T] token whose logit the LM-head row captures: -1, and in [T, 2T) the row's own token
 };
 
 // ------------------------------------------------------------------------------------------------

@@ -56,6 +56,7 @@ struct SetupArgs {
   const int* pending;       // dev [1] page mode: token of row 0
   const int* draft;         // dev [T-1] page mode: tokens of rows 1..
   const int* seq_slots;     // dev [S] or nullptr
+  const int* parent;        // dev [T] or nullptr: candidate trees, parent row within the sequence (-1 for row 0)
   int slot_base;            // slot of sequence 0 when seq_slots == nullptr
   int allow_embed_rows;     // prefill: token id < 0 means "use the embeds row"
   float rope_base;
@@ -89,6 +90,26 @@ struct AcceptArgs {
   float* row_zdraft;
 };
 void launch_accept(cudaStream_t st, const AcceptArgs& a, const RowMeta& rm, const int* status, bool pdl);
+// Greedy traversal of candidate trees (Eq. 9-12).  LM-head row r < T holds the argmax at node r, row T + r the
+// logit of node r's own token under its parent's distribution.
+struct TreeAcceptArgs {
+  int n_seqs, max_q_len, total_q;
+  float log_tau;
+  const int* parent;
+  const unsigned long long* row_best;   // [2T]
+  const float* zdraft;                  // [2T]
+  int* accept_len;
+  int* emit_tokens;
+  int* n_emit;
+  int* accept_rows;    // [S, max_q_len] rows of the accepted path after the root
+  int* row_argmax;     // optional outputs, [T]
+  float* row_zmax;
+  float* row_zchild;
+};
+void launch_tree_accept(cudaStream_t st, const TreeAcceptArgs& a, const RowMeta& rm, const int* status, bool pdl);
+// Moves the K/V rows of an accepted tree path (cache rows L + accept_rows[d-1]) to rows L + d, every layer and head.
+void launch_tree_compact(cudaStream_t st, const KvView& kv, int n_layers, int n_kv_heads, int n_seqs, const int* seq_slots,
+                         const int* accept_len, const int* accept_rows, int max_q_len, bool pdl);
 void launch_first_token(cudaStream_t st, const unsigned long long* row_best, int n_seqs, int* first_token,
                         const RowMeta& rm, const KvView& kv, const int* status, bool pdl);
 void launch_commit(cudaStream_t st, const KvView& kv, int n_seqs, const int* seq_slots, const int* accept_len,
@@ -101,7 +122,8 @@ void launch_unpack_best(cudaStream_t st, const unsigned long long* row_best, int
 constexpr int kAttnMaxSplits = 8;      // most KV slices one q-tile is cut into
 struct AttnPlan {
   int4* items;      // two int4 per (q-tile, slice) item, longest first: {first packed row, position of the first
-                    // token, tokens, KV slot}, {first | (last + 1) << 16 KV tile, slice | slices << 16, q-tile, KV tiles}
+                    // token, tokens, KV slot}, {first | (last + 1) << 16 KV tile, slice | slices << 8 | first token of the q-tile within its sequence << 16,
+                    // q-tile, KV tiles}
   int4* items_unsorted;   // the same list in creation order (scratch of the plan kernel)
   int* n_items;
   int* tile_seq;    // [max_tiles] sequence of a q-tile
@@ -113,7 +135,7 @@ void launch_attn_plan(cudaStream_t st, const RowMeta& rm, const AttnPlan& pl, in
                       int target_items, int min_chunk, const int* tile_count, const int* status, bool pdl);
 int launch_attn_sm100(cudaStream_t st, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                       const AttnPlan& plan, const KvView& kv, const ModelDims& md, int layer, bf16* out, int n_sms,
-                      int* status, float* split_ws, bool pdl);
+                      int* status, float* split_ws, const uint4* anc, bool pdl);
 
 // ---- plain SIMT GEMM (hsd_gemm_simt.cu): the debug cross-check and hsd_debug_logits --------------
 enum GemmMode { GM_STORE_BF16 = 0, GM_ADD_F32 = 1, GM_SWIGLU = 2, GM_STORE_F32 = 3, GM_ARGMAX = 4 };

@@ -72,6 +72,37 @@ __global__ void setup_rows_kernel(SetupArgs a, KvView kv, RowMeta rm, int* statu
   const int j_lo = blockIdx.y * kSetupRows;
   const int j_hi = min(n, j_lo + kSetupRows);
   const int half = a.head_dim / 2;
+  // Candidate tree: a row's rotary position is its depth below the pending token, not its index in the call
+  // (Sec. 3.2: a node continues the path pi(v), whatever else is packed beside it).
+  __shared__ int s_depth[kSetupRows];
+  if (a.parent) {
+    for (int j = j_lo + tid; j < j_hi; j += blockDim.x) {
+      uint32_t m[4] = {0u, 0u, 0u, 0u};
+      int d = 0, pj = j;
+      bool ok = j < 128;
+      if (ok) m[j >> 5] |= 1u << (j & 31);
+      while (ok && pj > 0) {
+        const int pp = a.parent[q0 + pj];
+        if (pp < 0 || pp >= pj) { ok = false; break; }
+        pj = pp;
+        m[pj >> 5] |= 1u << (pj & 31);
+        ++d;
+      }
+      if (j == 0 && a.parent[q0] != -1) ok = false;
+      if (!ok) {
+        dev_fail(status, DEV_TREE, q0 + j);
+        d = 0;
+      }
+      s_depth[j - j_lo] = d;
+      const int r = q0 + j;
+      rm.anc[r] = make_uint4(m[0], m[1], m[2], m[3]);
+      rm.lm_src[r] = r;
+      rm.lm_next[r] = -1;
+      rm.lm_src[a.total_q + r] = (ok && j > 0) ? q0 + a.parent[r] : r;
+      rm.lm_next[a.total_q + r] = (ok && j > 0) ? a.tokens[r] : -1;
+    }
+    __syncthreads();
+  }
   for (int j = j_lo + tid; j < j_hi; j += blockDim.x) {
     const int r = q0 + j;
     int tok, nxt = -1;
@@ -94,17 +125,17 @@ __global__ void setup_rows_kernel(SetupArgs a, KvView kv, RowMeta rm, int* statu
       phys = 0;
     }
     rm.row_seq[r] = i;
-    rm.row_pos[r] = pos;
+    rm.row_pos[r] = a.parent ? L + s_depth[j - j_lo] : pos;
     rm.row_tok[r] = tok;
     rm.row_kv[r] = phys * HSD_KV_BLOCK + pos % HSD_KV_BLOCK;
-    rm.row_next[r] = a.allow_embed_rows ? -1 : nxt;
+    rm.row_next[r] = (a.allow_embed_rows || a.parent) ? -1 : nxt;
   }
   // rotary table: (cos, sin) of pos * base^(-2i/D), angle formed in double so long contexts keep accuracy
   for (int e = j_lo * half + tid; e < j_hi * half; e += blockDim.x) {
     const int j = e / half, f = e % half;
     const double inv = exp2(-(double)(2 * f) / (double)a.head_dim * log2((double)a.rope_base));
     double sn, cs;
-    sincos((double)(L + j) * inv, &sn, &cs);
+    sincos((double)(L + (a.parent ? s_depth[j - j_lo] : j)) * inv, &sn, &cs);
     rm.rope_cs[(size_t)(q0 + j) * half + f] = make_float2((float)cs, (float)sn);
   }
 }
@@ -380,6 +411,122 @@ __global__ void accept_kernel(AcceptArgs a, RowMeta rm, const int* status) {
 }
 void launch_accept(cudaStream_t st, const AcceptArgs& a, const RowMeta& rm, const int* status, bool pdl) {
   launch_kernel(accept_kernel, dim3((a.n_seqs + 3) / 4), dim3(128), 0, st, pdl, a, rm, status);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Greedy traversal of a candidate tree (Eq. 9-12), one warp per sequence.  At the current node s: u_hat = the
+// full-vocabulary argmax at s; u* = the child of s with the best score (exact mode: the child that carries u_hat);
+// move to it iff z[u*] - z[u_hat] >= log tau; stop when the test fails or s has no child; emit pi(s) + u_hat.
+__global__ void tree_accept_kernel(TreeAcceptArgs a, RowMeta rm, const int* status) {
+  pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
+  pdl_launch_dependents();
+  if (*status) return;
+  const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (i >= a.n_seqs) return;
+  const int lane = threadIdx.x & 31;
+  const int q0 = rm.seq_q0[i], n = rm.seq_n[i], T = a.total_q;
+  if (n <= 0) {
+    if (lane == 0) { a.accept_len[i] = 0; a.n_emit[i] = 0; }
+    return;
+  }
+  int* emit = a.emit_tokens + (size_t)i * a.max_q_len;
+  int* path = a.accept_rows + (size_t)i * a.max_q_len;
+  int s = 0, acc = 0;
+  for (int step = 0; step < n; ++step) {
+    const unsigned long long best = a.row_best[q0 + s];
+    const int uhat = key_col(best);
+    int pick = -1;
+    if (a.log_tau == 0.f) {
+      for (int c0 = 1; c0 < n && pick < 0; c0 += 32) {
+        const int c = c0 + lane;
+        const bool hit = c < n && a.parent[q0 + c] == s && rm.row_tok[q0 + c] == uhat;
+        const unsigned m = __ballot_sync(0xffffffffu, hit);
+        if (m) pick = c0 + __ffs(m) - 1;
+      }
+    } else {
+      // best child by (score, then lower token id), then lower row among equals
+      unsigned long long bk = 0ull;
+      int bc = -1;
+      for (int c = 1 + lane; c < n; c += 32) {
+        if (a.parent[q0 + c] != s) continue;
+        const unsigned long long k = argmax_key(a.zdraft[T + q0 + c], rm.row_tok[q0 + c]);
+        if (bc < 0 || k > bk) { bk = k; bc = c; }
+      }
+      unsigned long long wk = bc >= 0 ? bk : 0ull;
+      for (int o = 16; o; o >>= 1) {
+        const unsigned long long ok2 = __shfl_xor_sync(0xffffffffu, wk, o);
+        wk = ok2 > wk ? ok2 : wk;
+      }
+      const unsigned has = __ballot_sync(0xffffffffu, bc >= 0);
+      if (has) {
+        const int cand = (bc >= 0 && bk == wk) ? bc : 0x7fffffff;
+        int lo = cand;
+        for (int o = 16; o; o >>= 1) lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        pick = lo;
+        if (!(a.zdraft[T + q0 + pick] - key_value(best) >= a.log_tau)) pick = -1;
+      }
+    }
+    if (pick < 0) break;
+    if (lane == 0) {
+      path[acc] = pick;
+      emit[acc] = rm.row_tok[q0 + pick];
+    }
+    ++acc;
+    s = pick;
+  }
+  if (lane == 0) {
+    emit[acc] = key_col(a.row_best[q0 + s]);
+    a.accept_len[i] = acc;
+    a.n_emit[i] = acc + 1;
+  }
+  for (int j = lane; j < n; j += 32) {
+    const unsigned long long best = a.row_best[q0 + j];
+    if (a.row_argmax) a.row_argmax[q0 + j] = key_col(best);
+    if (a.row_zmax) a.row_zmax[q0 + j] = key_value(best);
+    if (a.row_zchild) a.row_zchild[q0 + j] = j > 0 ? a.zdraft[T + q0 + j] : __int_as_float(0x7fc00000);
+  }
+}
+void launch_tree_accept(cudaStream_t st, const TreeAcceptArgs& a, const RowMeta& rm, const int* status, bool pdl) {
+  launch_kernel(tree_accept_kernel, dim3((a.n_seqs + 3) / 4), dim3(128), 0, st, pdl, a, rm, status);
+}
+
+// KV maintenance after a tree step (Sec. 4.2: rollbacks and cache maintenance are part of the decode loop): the
+// accepted path's rows move from their packed places L + r_d to the places L + d their rotary positions stand for.
+// One CTA per (sequence, layer); a path's rows increase strictly, so moving depth by depth never overwrites a row
+// that is still to be read.
+__global__ void tree_compact_kernel(KvView kv, int n_kv_heads, int n_seqs, const int* seq_slots, const int* accept_len,
+                                    const int* accept_rows, int max_q_len) {
+  pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
+  pdl_launch_dependents();
+  const int i = blockIdx.x, layer = blockIdx.y;
+  const int slot = seq_slots ? seq_slots[i] : i;
+  if (slot < 0 || slot >= kv.n_slots) return;
+  const int a = accept_len[i];
+  const int L = kv.seq_lens[slot];
+  const int* bt = kv.block_table + (size_t)slot * kv.max_blocks;
+  const int chunks = n_kv_heads * 2 * 8;                 // 16-byte chunks of one token's K and V rows in a layer
+  for (int d = 1; d <= a && d < max_q_len; ++d) {
+    const int r = accept_rows[(size_t)i * max_q_len + d - 1];
+    if (r != d && r > 0 && (L + r) / HSD_KV_BLOCK < kv.max_blocks) {
+      const int ps = L + r, pd = L + d;
+      const int bs = bt[ps / HSD_KV_BLOCK], bd = bt[pd / HSD_KV_BLOCK];
+      if (bs >= 0 && bs < kv.n_blocks && bd >= 0 && bd < kv.n_blocks) {
+        for (int t = threadIdx.x; t < chunks; t += blockDim.x) {
+          const int c16 = t & 7, pool = (t >> 3) & 1, h = t >> 4;
+          bf16* base = pool ? kv.v_pool : kv.k_pool;
+          const size_t src = ((((size_t)layer * kv.n_blocks + bs) * n_kv_heads + h) * 64 + ps % HSD_KV_BLOCK) * 64;
+          const size_t dst = ((((size_t)layer * kv.n_blocks + bd) * n_kv_heads + h) * 64 + pd % HSD_KV_BLOCK) * 64;
+          reinterpret_cast<uint4*>(base + dst)[c16] = reinterpret_cast<const uint4*>(base + src)[c16];
+        }
+      }
+    }
+    __syncthreads();
+  }
+}
+void launch_tree_compact(cudaStream_t st, const KvView& kv, int n_layers, int n_kv_heads, int n_seqs, const int* seq_slots,
+                         const int* accept_len, const int* accept_rows, int max_q_len, bool pdl) {
+  launch_kernel(tree_compact_kernel, dim3(n_seqs, n_layers), dim3(128), 0, st, pdl, kv, n_kv_heads, n_seqs, seq_slots,
+                accept_len, accept_rows, max_q_len);
 }
 
 // Prefill epilogue: first pending token per sequence, and seq_lens += rows.

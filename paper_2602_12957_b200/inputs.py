@@ -269,6 +269,75 @@ def plant_draft(greedy: Sequence[int], k: int, agree_len: int, rand_tokens: np.n
     return d.astype(np.int32)
 
 
+# --------------------------------------------------------------------------- candidate trees
+def plant_tree(greedy: Sequence[int], n_nodes: int, agree_len: int, vocab: int, seed: int, n_branches: int = 6,
+               shuffle: bool = True):
+    """A packed candidate tree of `n_nodes` nodes below the root (paper Sec. 3.2: suffixes merged on common
+    prefixes).  One root-to-leaf "main" path copies `greedy` (some decoder's own greedy continuation, supplied by
+    the caller) for `agree_len` tokens and then leaves it; `n_branches` side paths of random tokens fork off
+    random nodes of the tree; siblings always carry distinct tokens, and a side branch never carries the greedy
+    token of its depth, so the greedy path through the tree is unique.  Rows are packed parents-first but, with
+    `shuffle`, otherwise in random order, so a row's index and its depth differ.
+
+    Returns (tokens [n_nodes] int32 of rows 1.., parent [n_nodes + 1] int32 with parent[0] = -1, main_rows: the
+    packed rows of the main path in depth order)."""
+    rng = np.random.Generator(np.random.PCG64(seed + 3_000_017))
+    g = [int(t) for t in greedy]
+    n_nodes = int(n_nodes)
+    if n_nodes < 1:
+        return np.zeros(0, np.int32), np.asarray([-1], np.int32), []
+    n_side = min(n_branches, max(0, n_nodes - 1))
+    side_total = int(rng.integers(n_side, max(n_side, n_nodes // 2) + 1)) if n_side else 0
+    main_len = n_nodes - side_total
+    if len(g) < min(agree_len + 1, main_len):
+        raise ValueError("greedy continuation too short for the planted agreement")
+    # logical tree: node ids 1.., 0 = root
+    par, tok, depth = [-1], [-1], [0]
+    kids = {0: set()}
+
+    def add(p, t):
+        par.append(p); tok.append(int(t)); depth.append(depth[p] + 1)
+        kids[p].add(int(t)); kids[len(par) - 1] = set()
+        return len(par) - 1
+
+    def fresh(p, avoid):
+        while True:
+            t = int(rng.integers(0, vocab))
+            if t not in kids[p] and t != avoid:
+                return t
+
+    main, cur = [], 0
+    a = int(min(agree_len, main_len))
+    for d in range(main_len):
+        gt = g[d] if d < len(g) else -1
+        t = gt if d < a else fresh(cur, gt)
+        cur = add(cur, t)
+        main.append(cur)
+    left = side_total
+    for b in range(n_side):
+        length = left if b == n_side - 1 else int(rng.integers(1, max(1, left - (n_side - 1 - b)) + 1))
+        left -= length
+        cur = int(rng.integers(0, len(par)))
+        for _ in range(length):
+            d = depth[cur]
+            cur = add(cur, fresh(cur, g[d] if d < len(g) else -1))
+    n = len(par)
+    # packing order: random topological order (a node becomes available once its parent is placed)
+    order, avail = [0], [j for j in range(1, n) if par[j] == 0]
+    children = {j: [] for j in range(n)}
+    for j in range(1, n):
+        children[par[j]].append(j)
+    while avail:
+        pick = int(rng.integers(0, len(avail))) if shuffle else 0
+        j = avail.pop(pick)
+        order.append(j)
+        avail.extend(children[j])
+    where = {j: r for r, j in enumerate(order)}
+    parent = np.asarray([-1] + [where[par[j]] for j in order[1:]], np.int32)
+    tokens = np.asarray([tok[j] for j in order[1:]], np.int32)
+    return tokens, parent, [where[j] for j in main]
+
+
 # --------------------------------------------------------------------------- paged KV layout
 def blocks_needed(n_tokens: int, kv_block: int = 64) -> int:
     return (int(n_tokens) + kv_block - 1) // kv_block

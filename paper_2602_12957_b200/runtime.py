@@ -139,6 +139,28 @@ class Engine:
         B.check(st, "hsd_verify_regions")
         return out
 
+    def verify_tree(self, q_tokens: torch.Tensor, cu_q: torch.Tensor, parent: torch.Tensor, max_q_len: int,
+                    total_q: int, out: Optional[dict] = None, slots: Optional[torch.Tensor] = None,
+                    log_tau: float = 0.0):
+        """Candidate trees (the workspace must have been sized for 2 * total_q rows)."""
+        n_seqs = cu_q.numel() - 1
+        if out is None:
+            out = self.alloc_outputs(n_seqs, max_q_len, total_q)
+            out["accept_rows"] = torch.zeros(n_seqs, max_q_len, dtype=torch.int32, device=self.dev)
+            out["row_zchild"] = out.pop("row_zdraft")
+        st = B.hsd_verify_tree(self.model.ctx, self.kv.c, n_seqs, cu_q, q_tokens, parent, slots, max_q_len, total_q,
+                               log_tau, out["accept_len"], out["emit_tokens"], out["n_emit"], out["accept_rows"],
+                               out["row_argmax"], out["row_zmax"], out["row_zchild"], self.ws.ptr, self.ws.bytes,
+                               _stream())
+        B.check(st, "hsd_verify_tree")
+        return out
+
+    def commit_tree(self, accept_len: torch.Tensor, accept_rows: torch.Tensor, slots: Optional[torch.Tensor] = None,
+                    blocks_in_use: Optional[torch.Tensor] = None):
+        st = B.hsd_kv_commit_tree(self.model.ctx, self.kv.c, int(accept_len.numel()), slots, accept_len, accept_rows,
+                                  int(accept_rows.shape[1]), blocks_in_use, _stream())
+        B.check(st, "hsd_kv_commit_tree")
+
     def verify_page(self, slot: int, pending: torch.Tensor, chunk: torch.Tensor, out: Optional[dict] = None,
                     log_tau: float = 0.0):
         n = int(chunk.numel())
