@@ -111,9 +111,17 @@ WORKLOADS = {
     "page": "page-level stage, one chunk mid-schedule: batch 1, 6400 committed tokens, chunk of 512 draft tokens",
     "long1024": "long-document page verify, one chunk mid-schedule: batch 1, 10240 committed tokens, chunk of 1024",
     "long2048": "long-document page verify, one chunk mid-schedule: batch 1, 10240 committed tokens, chunk of 2048",
+    "tree": "candidate-tree verification (the paper's packed form): the region batch's 16 prefixes (256-1024), each with a "
+            "prefix tree of 127 nodes packed into 128 rows (one planted main path + 6 side branches), tau 0.75, "
+            "followed by the compaction of the accepted path's K/V rows",
     "mixed": "mixed serving batch: 64 regions (prefix 128-2048, lognormal drafts mean 96, 8-512) + 2 page chunks of 1024 "
              "over 4352-token prefixes, one varlen launch",
 }
+
+
+TREE_NODES = 127     # nodes below the root: 128 packed rows per sequence, the paper's packing limit (Sec. 4.3)
+TREE_MAIN = 64       # about this many of them lie on the main path
+LOG_TAU_TREE = float(np.log(0.75))
 
 
 def make_workload(args, rank):
@@ -123,6 +131,12 @@ def make_workload(args, rank):
     name = getattr(args, "workload", "region")
     if name == "region":
         return I.region_workload(seed=I.BASE_SEED + 1 + 1000 * rank, cfg=cfg)
+    if name == "tree":
+        wl = I.region_workload(seed=I.BASE_SEED + 1 + 1000 * rank, cfg=cfg)
+        for s_ in wl.seqs:          # same prefixes; the draft becomes a 127-node tree whose main path agrees as planted
+            s_.agree_len = int(round(TREE_MAIN * s_.agree_len / max(1, s_.draft_len)))
+            s_.draft_len = TREE_NODES
+        return wl
     args.random_drafts = True
     if name == "mixed":
         return I.mixed_workload(seed=I.BASE_SEED + 4 + 1000 * rank, cfg=cfg)
@@ -147,13 +161,16 @@ def build_gpu_state(args, rank):
     ks = [s.draft_len for s in seqs]
     total_q = sum(ks) + S
     total_prefix = sum(s.prefix_len for s in seqs)
-    eng = R.Engine(model, kv, max(total_prefix, total_q), S)
+    tree = wl is not None and getattr(args, "workload", "region") == "tree"
+    eng = R.Engine(model, kv, max(total_prefix, 2 * total_q if tree else total_q), S)
     first = eng.prefill([s.prefix_embeds for s in seqs], [s.prefix_ids for s in seqs])
     eng.check_device("prefill")
     prefix_lens = kv.seq_lens.clone()
 
     # greedy continuation by plain one-token steps (empty drafts), to plant the agreement lengths
     need = 0 if args.random_drafts else max(min(s.agree_len + 1, s.draft_len) for s in seqs)
+    if tree:
+        need = TREE_NODES
     cu1 = eng._i32(np.arange(S + 1))
     out1 = eng.alloc_outputs(S, 1, S)
     pending = first.clone()
@@ -166,14 +183,21 @@ def build_gpu_state(args, rank):
     eng.check_device("greedy continuation")
     greedy = torch.stack(hist, 1).cpu().numpy() if hist else np.zeros((S, 0), np.int32)
     kv.seq_lens.copy_(prefix_lens)
-    if args.random_drafts:      # profiling runs: kernel time does not depend on token values
+    if tree:
+        drafts = []
+    elif args.random_drafts:    # profiling runs: kernel time does not depend on token values
         drafts = [s.rand_tokens[:s.draft_len] for s in seqs]
     else:
         drafts = [I.plant_draft(greedy[i], s.draft_len, s.agree_len, s.rand_tokens, cfg.vocab, False)
                   for i, s in enumerate(seqs)]
+    parent = None
+    if tree:
+        planted = [I.plant_tree(greedy[i], TREE_NODES, s.agree_len, cfg.vocab, wl.seed + i) for i, s in enumerate(seqs)]
+        drafts = [p[0] for p in planted]
+        parent = np.concatenate([p[1] for p in planted]).astype(np.int32)
     toks, cu = I.pack_queries(first.cpu().numpy(), drafts)
     return dict(cfg=cfg, wl=wl, model=model, kv=kv, eng=eng, toks=toks, cu=cu, total_q=total_q, max_q=max(ks) + 1,
-                prefix_lens=prefix_lens, ks=ks, S=S, drafts=drafts)
+                prefix_lens=prefix_lens, ks=ks, S=S, drafts=drafts, parent=parent)
 
 
 def kernel_work_table(cfg, work: RF.StepWork, T: int):
@@ -185,7 +209,7 @@ def kernel_work_table(cfg, work: RF.StepWork, T: int):
     t["gemm_o"] = RF.gemm_work(T, d, cfg.n_heads * cfg.head_dim, 8.0)          # fp32 read-modify-write
     t["gemm_gate_up"] = (2.0 * T * 2 * f * d, 2.0 * (T * d + 2 * f * d) + 2.0 * T * f)
     t["gemm_down"] = RF.gemm_work(T, d, f, 8.0)
-    t["lm_head_argmax"] = (2.0 * T * V * d, 2.0 * (T * d + V * d) + 12.0 * T)
+    t["lm_head_argmax"] = (2.0 * T * V * d, 2.0 * (T * d + V * d) + 12.0 * T)       # (a tree step runs it over 2T rows)
     t["attention"] = (work.attn_flops / L, work.kv_read_bytes / L + 4.0 * T * cfg.n_heads * cfg.head_dim)
     t["rmsnorm"] = (0.0, 6.0 * T * d)
     return t
@@ -209,10 +233,19 @@ def run_ours(args):
     d_toks, d_cu = eng._i32(st["toks"]), eng._i32(st["cu"])
     out = eng.alloc_outputs(S, max_q, T)
     stream = torch.cuda.Stream(device=dev)
+    tree = st["parent"] is not None
+    if tree:
+        d_parent = eng._i32(st["parent"])
+        out["accept_rows"] = torch.zeros(S, max_q, dtype=torch.int32, device=dev)
+        out["row_zchild"] = out.pop("row_zdraft")
 
     def step():
-        eng.verify_regions(d_toks, d_cu, max_q, T, out=out)
-        eng.commit(out["accept_len"])
+        if tree:
+            eng.verify_tree(d_toks, d_cu, d_parent, max_q, T, out=out, log_tau=LOG_TAU_TREE)
+            eng.commit_tree(out["accept_len"], out["accept_rows"])
+        else:
+            eng.verify_regions(d_toks, d_cu, max_q, T, out=out)
+            eng.commit(out["accept_len"])
         kv.seq_lens.copy_(st["prefix_lens"])          # rewind so every timed step sees the same state
 
     launches0 = B.hsd_launch_count(eng.model.ctx)
@@ -281,10 +314,23 @@ def run_ours(args):
     e2e_steps = max(3, min(args.steps, 200))
     ctx = eng.model.ctx
 
+    h_par = torch.from_numpy(st["parent"]).pin_memory() if tree else None
+
     def e2e_step():
-        rc, _ = B.hsd_verify_regions_host(ctx, kv.c, S, h_cu, h_toks, None, 0.0, 1, h_acc, h_emit, h_nem, eng.ws.ptr,
-                                          eng.ws.bytes, stream.cuda_stream)
-        B.check(rc, "hsd_verify_regions_host")
+        if tree:     # the tree calls take device buffers: the copies are made here, on the same stream
+            d_toks.copy_(h_toks, non_blocking=True)
+            d_cu.copy_(h_cu, non_blocking=True)
+            d_parent.copy_(h_par, non_blocking=True)
+            eng.verify_tree(d_toks, d_cu, d_parent, max_q, T, out=out, log_tau=LOG_TAU_TREE)
+            eng.commit_tree(out["accept_len"], out["accept_rows"])
+            h_acc.copy_(out["accept_len"], non_blocking=True)
+            h_nem.copy_(out["n_emit"], non_blocking=True)
+            h_emit.copy_(out["emit_tokens"], non_blocking=True)
+            stream.synchronize()
+        else:
+            rc, _ = B.hsd_verify_regions_host(ctx, kv.c, S, h_cu, h_toks, None, 0.0, 1, h_acc, h_emit, h_nem, eng.ws.ptr,
+                                              eng.ws.bytes, stream.cuda_stream)
+            B.check(rc, "hsd_verify_regions_host")
         kv.seq_lens.copy_(st["prefix_lens"])          # rewind (bench artefact: every step sees the same state)
 
     with torch.cuda.stream(stream):
@@ -303,10 +349,12 @@ def run_ours(args):
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         e2e_ms = float(tt.item())
     e2e = {"value": draft_tokens * world / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
-           "h2d_bytes_per_step": int(h_toks.numel() * 4 + h_cu.numel() * 4),
+           "h2d_bytes_per_step": int(h_toks.numel() * 4 + h_cu.numel() * 4 + (h_par.numel() * 4 if tree else 0)),
            "d2h_bytes_per_step": int((h_acc.numel() + h_nem.numel() + h_emit.numel()) * 4 + 16),
            "call": "hsd_verify_regions_host (pinned host buffers; the library replays the step as a CUDA graph it captured "
-                   "at the second call of this shape; stream synchronised per step)"}
+                   "at the second call of this shape; stream synchronised per step)" if not tree else
+                   "hsd_verify_tree + hsd_kv_commit_tree (eager launches) with pinned-host copies in and out on the same "
+                   "stream, synchronised per step"}
     accept_mean = float(np.mean([a / k for a, k in zip(h_acc.numpy().tolist(), st["ks"])]))
 
     # ---- per-kernel durations (CUDA events around every launch, eager) for the roofline of the top kernel
