@@ -81,3 +81,36 @@ def test_block_tables_are_disjoint_and_padded():
 def test_pack_queries():
     toks, cu = I.pack_queries([7, 8], [np.array([1, 2, 3]), np.array([], np.int32)])
     assert list(toks) == [7, 1, 2, 3, 8] and list(cu) == [0, 4, 5]
+
+
+def test_plant_tree_is_a_parent_first_prefix_tree_with_one_greedy_path():
+    from collections import defaultdict
+    from oracle import hsd_oracle as O
+    greedy = list(range(500, 700))
+    for seed in range(8):
+        for n, a in ((1, 0), (1, 1), (5, 2), (40, 7), (127, 30)):
+            tok, par, main = I.plant_tree(greedy, n, a, 1000, seed)
+            assert tok.shape == (n,) and par.shape == (n + 1,) and par[0] == -1
+            assert all(0 <= par[j] < j for j in range(1, n + 1))           # parents come first
+            O.tree_depth_and_mask(par)                                     # the oracle accepts it
+            kids = defaultdict(list)
+            for j in range(1, n + 1):
+                kids[int(par[j])].append(int(tok[j - 1]))
+            assert all(len(set(v)) == len(v) for v in kids.values())       # siblings carry distinct tokens
+            # the main path copies the greedy tokens for `a` steps and then leaves them
+            a_eff = min(a, len(main))
+            assert [int(tok[r - 1]) for r in main[:a_eff]] == greedy[:a_eff]
+            assert all(par[main[d]] == (main[d - 1] if d else 0) for d in range(len(main)))
+            if a_eff < len(main):
+                assert int(tok[main[a_eff] - 1]) != greedy[a_eff]
+            # walking the greedy tokens from the root follows the main path for exactly a_eff moves
+            s, moves = 0, 0
+            while True:
+                nxt = [j for j in range(1, n + 1) if par[j] == s and int(tok[j - 1]) == greedy[moves]]
+                if not nxt:
+                    break
+                s, moves = nxt[0], moves + 1
+            assert moves == a_eff and (moves == 0 or s == main[moves - 1])
+    t1, p1, _ = I.plant_tree(greedy, 40, 7, 1000, 3)
+    t2, p2, _ = I.plant_tree(greedy, 40, 7, 1000, 3)
+    assert np.array_equal(t1, t2) and np.array_equal(p1, p2)               # seeded
