@@ -65,6 +65,8 @@ extern "C" {
 
 #define HSD_MAX_Q_LEN 4097         /* most query rows one sequence may have in a verify call          */
 #define HSD_MAX_TREE_ROWS 128      /* most rows (root included) of one sequence in hsd_verify_tree    */
+#define HSD_MAX_WINDOW 8           /* longest reference window hsd_dsv_build takes (the paper uses 3)   */
+#define HSD_DSV_MAX_CANDIDATES 64  /* candidate suffixes per sequence; later matches are ignored        */
 #define HSD_KV_BLOCK 64
 
 /* hsd_model_config.flags */
@@ -168,7 +170,9 @@ HSD_API int hsd_verify_page(hsd_ctx *ctx, const hsd_kv *kv, int seq_slot, const 
 /* One verification step over candidate TREES (Sec. 3.2: prefix tree T of Eq. 7 packed into one sequence, the
  * tree-ancestry mask of Fig. 2(c), greedy traversal of Eq. 9-12).  Per sequence the packed rows are
  * [pending token (the root), node 1, .., node k] in an order that puts every parent before its children;
- *   parent          dev int32 [total_q]: the parent's row index WITHIN the sequence, -1 for row 0
+ *   parent          dev int32 [total_q]: the parent's row index WITHIN the sequence, -1 for row 0; -2 marks a
+ *                   padding row (no parent, no children: it sees the committed context and itself, nothing can
+ *                   move to it; hsd_dsv_build pads with such rows to keep shapes fixed)
  *   max_q_len       at most HSD_MAX_TREE_ROWS rows per sequence (root included; the paper packs <= 128 tokens)
  * A node's rotary position is committed length + depth; it attends to the committed context, itself and its
  * ancestors.  Traversal from the root: at node s, u_hat = argmax over the vocabulary (lowest id on ties), u* = the
@@ -189,6 +193,28 @@ HSD_API int hsd_verify_tree(hsd_ctx *ctx, const hsd_kv *kv, int n_seqs, const in
                     const int *parent, const int *seq_slots, int max_q_len, int total_q, float log_tau,
                     int *accept_len, int *emit_tokens, int *n_emit, int *accept_rows, int *row_argmax, float *row_zmax,
                     float *row_zchild, void *workspace, size_t ws_bytes, void *cuda_stream);
+
+/* Draft-target matching and prefix-tree packing on the device (Sec. 3.2, Eq. 5-7), so that a decode loop of
+ * hsd_dsv_build -> hsd_verify_tree -> hsd_kv_commit_tree has fixed shapes and needs no host decision between steps.
+ *   window          dev int32 [n_seqs, window_n] INOUT: the window_n (<= HSD_MAX_WINDOW) most recent accepted
+ *                   tokens of every sequence, oldest first; a negative entry means "not that many tokens yet" (no
+ *                   match is attempted then); the last entry is the pending token and must be a valid id
+ *   emit_tokens, n_emit   dev int32 [n_seqs, emit_stride], [n_seqs] or both NULL: the tokens the previous step
+ *                   emitted; they are appended to the window before matching (and the window is written back)
+ *   draft_tokens    dev int32, all drafts concatenated;  draft_off dev int32 [n_drafts + 1] their offsets;
+ *   seq_draft_off   dev int32 [n_seqs + 1]: sequence i owns drafts seq_draft_off[i] .. seq_draft_off[i+1] - 1
+ *   max_rows        rows every sequence gets in the packed output (<= HSD_MAX_TREE_ROWS; the paper packs 128)
+ *   q_tokens, parent  dev int32 [n_seqs * max_rows] out: row 0 = the pending token (parent -1), then the tree's
+ *                   nodes with their parent rows, then padding rows (the pending token again, parent -2) which
+ *                   hsd_verify_tree treats as rows without parent or children
+ *   cu_q            dev int32 [n_seqs + 1] out: i * max_rows;   n_rows dev int32 [n_seqs] out: 1 + nodes
+ * Candidates: for every draft of the sequence and every position where the window occurs (Eq. 5), the non-empty
+ * suffix after it (Eq. 6), in draft order then position order, at most HSD_DSV_MAX_CANDIDATES.  Tree (Eq. 7): one
+ * node per distinct prefix, created level by level in candidate order while fewer than max_rows - 1 nodes exist; a
+ * candidate whose next node cannot be created stops growing.  Pure integer work: results are exact. */
+HSD_API int hsd_dsv_build(hsd_ctx *ctx, int n_seqs, int window_n, int *window, const int *emit_tokens, const int *n_emit,
+                  int emit_stride, const int *draft_tokens, const int *draft_off, const int *seq_draft_off,
+                  int max_rows, int *q_tokens, int *parent, int *cu_q, int *n_rows, void *cuda_stream);
 
 /* KV maintenance after hsd_verify_tree (Sec. 4.2 counts it in the decode loop): in every layer the K/V rows of the
  * accepted path move from cache rows L + accept_rows[i][d-1] to rows L + d (d = 1..accept_len[i]; L = committed

@@ -18,6 +18,8 @@ HSD_ERR_INVALID_ARG, HSD_ERR_SHAPE, HSD_ERR_TOO_LONG, HSD_ERR_WORKSPACE = -1, -2
 HSD_ERR_KV_CAPACITY, HSD_ERR_CUDA, HSD_ERR_DEVICE_CHECK, HSD_ERR_NO_DEVICE = -5, -6, -7, -8
 HSD_MAX_Q_LEN = 4097
 HSD_MAX_TREE_ROWS = 128
+HSD_MAX_WINDOW = 8
+HSD_DSV_MAX_CANDIDATES = 64
 HSD_KV_BLOCK = 64
 HSD_FLAG_SIMT_DEBUG = 1
 HSD_FLAG_SIMT_ATTENTION = 2
@@ -32,7 +34,7 @@ EXPORTS = [
     "hsd_verify_page", "hsd_kv_commit", "hsd_verify_regions_host", "hsd_device_status", "hsd_last_cuda_error", "hsd_launch_count",
     "hsd_profile_enable", "hsd_profile_read", "hsd_debug_logits", "hsd_debug_buffer", "hsd_op_linear",
     "hsd_op_lm_head_argmax", "hsd_op_lm_head_argmax_noalloc", "hsd_debug_set_gemm_tile", "hsd_debug_set_attn_plan",
-    "hsd_verify_tree", "hsd_kv_commit_tree",
+    "hsd_verify_tree", "hsd_kv_commit_tree", "hsd_dsv_build",
 ]
 
 
@@ -81,6 +83,7 @@ def _load():
     lib.hsd_verify_tree.argtypes = [vp, C.POINTER(hsd_kv), i, vp, vp, vp, vp, i, i, f, vp, vp, vp, vp, vp, vp, vp, vp, sz,
                                     vp]
     lib.hsd_kv_commit_tree.argtypes = [vp, C.POINTER(hsd_kv), i, vp, vp, vp, i, vp, vp]
+    lib.hsd_dsv_build.argtypes = [vp, i, i, vp, vp, vp, i, vp, vp, vp, i, vp, vp, vp, vp, vp]
     lib.hsd_verify_regions_host.argtypes = [vp, C.POINTER(hsd_kv), i, vp, vp, vp, f, i, vp, vp, vp, C.POINTER(C.c_int), vp, sz, vp]
     lib.hsd_device_status.argtypes = [vp, vp, vp, C.POINTER(C.c_int)]
     lib.hsd_last_cuda_error.argtypes = [vp]
@@ -216,6 +219,13 @@ def hsd_verify_tree(ctx, kv, n_seqs, cu_q, q_tokens, parent, seq_slots, max_q_le
 def hsd_kv_commit_tree(ctx, kv, n_seqs, seq_slots, accept_len, accept_rows, max_q_len, blocks_in_use, stream) -> int:
     return _lib.hsd_kv_commit_tree(ctx, C.byref(kv) if kv is not None else None, n_seqs, _p(seq_slots), _p(accept_len),
                                    _p(accept_rows), max_q_len, _p(blocks_in_use), _p(stream))
+
+
+def hsd_dsv_build(ctx, n_seqs, window_n, window, emit_tokens, n_emit, emit_stride, draft_tokens, draft_off, seq_draft_off,
+                  max_rows, q_tokens, parent, cu_q, n_rows, stream) -> int:
+    return _lib.hsd_dsv_build(ctx, n_seqs, window_n, _p(window), _p(emit_tokens), _p(n_emit), emit_stride,
+                              _p(draft_tokens), _p(draft_off), _p(seq_draft_off), max_rows, _p(q_tokens), _p(parent),
+                              _p(cu_q), _p(n_rows), _p(stream))
 
 
 def hsd_device_status(ctx, workspace, stream):

@@ -110,6 +110,21 @@ void launch_tree_accept(cudaStream_t st, const TreeAcceptArgs& a, const RowMeta&
 // Moves the K/V rows of an accepted tree path (cache rows L + accept_rows[d-1]) to rows L + d, every layer and head.
 void launch_tree_compact(cudaStream_t st, const KvView& kv, int n_layers, int n_kv_heads, int n_seqs, const int* seq_slots,
                          const int* accept_len, const int* accept_rows, int max_q_len, bool pdl);
+// Draft-target matching + prefix-tree packing on the device (Eq. 5-7)
+struct DsvArgs {
+  int n_seqs, window_n, max_rows, emit_stride;
+  int* window;               // [S, n] inout
+  const int* emit_tokens;    // [S, emit_stride] or nullptr
+  const int* n_emit;         // [S] or nullptr
+  const int* draft_tokens;
+  const int* draft_off;      // [n_drafts + 1]
+  const int* seq_draft_off;  // [S + 1]
+  int* q_tokens;             // [S * max_rows]
+  int* parent;               // [S * max_rows]
+  int* cu_q;                 // [S + 1]
+  int* n_rows;               // [S]
+};
+void launch_dsv_build(cudaStream_t st, const DsvArgs& a, bool pdl);
 void launch_first_token(cudaStream_t st, const unsigned long long* row_best, int n_seqs, int* first_token,
                         const RowMeta& rm, const KvView& kv, const int* status, bool pdl);
 void launch_commit(cudaStream_t st, const KvView& kv, int n_seqs, const int* seq_slots, const int* accept_len,

@@ -81,6 +81,7 @@ __global__ void setup_rows_kernel(SetupArgs a, KvView kv, RowMeta rm, int* statu
       int d = 0, pj = j;
       bool ok = j < 128;
       if (ok) m[j >> 5] |= 1u << (j & 31);
+      if (j > 0 && a.parent[q0 + j] == -2) pj = 0;      // padding row: no parent, no children, sees only itself
       while (ok && pj > 0) {
         const int pp = a.parent[q0 + pj];
         if (pp < 0 || pp >= pj) { ok = false; break; }
@@ -98,8 +99,9 @@ __global__ void setup_rows_kernel(SetupArgs a, KvView kv, RowMeta rm, int* statu
       rm.anc[r] = make_uint4(m[0], m[1], m[2], m[3]);
       rm.lm_src[r] = r;
       rm.lm_next[r] = -1;
-      rm.lm_src[a.total_q + r] = (ok && j > 0) ? q0 + a.parent[r] : r;
-      rm.lm_next[a.total_q + r] = (ok && j > 0) ? a.tokens[r] : -1;
+      const bool child = ok && j > 0 && a.parent[r] >= 0;
+      rm.lm_src[a.total_q + r] = child ? q0 + a.parent[r] : r;
+      rm.lm_next[a.total_q + r] = child ? a.tokens[r] : -1;
     }
     __syncthreads();
   }
@@ -527,6 +529,131 @@ void launch_tree_compact(cudaStream_t st, const KvView& kv, int n_layers, int n_
                          const int* accept_len, const int* accept_rows, int max_q_len, bool pdl) {
   launch_kernel(tree_compact_kernel, dim3(n_seqs, n_layers), dim3(128), 0, st, pdl, kv, n_kv_heads, n_seqs, seq_slots,
                 accept_len, accept_rows, max_q_len);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Draft-target matching and prefix-tree packing (Sec. 3.2, Eq. 5-7), one CTA per sequence.
+//  1. the window takes in the tokens the last step emitted (w = the n most recent accepted tokens);
+//  2. every position of the sequence's drafts where w occurs gives a candidate: the non-empty suffix after it
+//     (Eq. 5, 6), in draft order then position order, at most kDsvMaxCands of them;
+//  3. warp 0 grows the prefix tree level by level (Eq. 7): at depth d every live candidate moves to the child
+//     that carries its d-th token, creating it while the node budget lasts; a candidate whose node cannot be
+//     created stops.  Node ids are creation order, so parents precede children and the id is the packed row.
+// Every sequence gets exactly max_rows rows: row 0 = the pending token, then the nodes, then padding rows
+// (parent -2) that no traversal can enter.
+constexpr int kDsvMaxCands = 64;
+constexpr int kDsvMaxWindow = 8;
+__global__ void dsv_build_kernel(DsvArgs a) {
+  pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
+  pdl_launch_dependents();
+  const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  __shared__ int s_w[kDsvMaxWindow];
+  __shared__ int s_cstart[kDsvMaxCands], s_clen[kDsvMaxCands], s_ccur[kDsvMaxCands];
+  __shared__ int s_ntok[HSD_MAX_TREE_ROWS], s_npar[HSD_MAX_TREE_ROWS];
+  __shared__ unsigned s_ballot[4];
+  __shared__ int s_ncand, s_nnodes;
+  const int n = a.window_n;
+  if (tid == 0) {
+    // window <- last n of (window ++ emitted)
+    int tmp[2 * kDsvMaxWindow];
+    int m = 0;
+    for (int i = 0; i < n; ++i) tmp[m++] = a.window[s * n + i];
+    if (a.emit_tokens && a.n_emit) {
+      const int ne = a.n_emit[s];
+      for (int i = max(0, ne - n); i < ne; ++i) {
+        if (m == 2 * kDsvMaxWindow) {
+          for (int k = 1; k < m; ++k) tmp[k - 1] = tmp[k];
+          --m;
+        }
+        tmp[m++] = a.emit_tokens[(size_t)s * a.emit_stride + i];
+      }
+    }
+    for (int i = 0; i < n; ++i) {
+      s_w[i] = tmp[m - n + i];
+      a.window[s * n + i] = s_w[i];
+    }
+    s_ncand = 0;
+    s_nnodes = 0;
+    a.cu_q[s] = s * a.max_rows;
+    if (s == 0) a.cu_q[a.n_seqs] = a.n_seqs * a.max_rows;
+  }
+  __syncthreads();
+  bool have_w = true;
+  for (int i = 0; i < n; ++i) have_w = have_w && s_w[i] >= 0;
+  // ---- candidates
+  if (have_w) {
+    for (int d = a.seq_draft_off[s]; d < a.seq_draft_off[s + 1]; ++d) {
+      const int d0 = a.draft_off[d], len = a.draft_off[d + 1] - d0;
+      for (int j0 = 0; j0 + n < len; j0 += blockDim.x) {      // j + n < len: a non-empty suffix follows the window
+        if (s_ncand >= kDsvMaxCands) break;
+        const int j = j0 + tid;
+        bool hit = j + n < len;
+        for (int i = 0; hit && i < n; ++i) hit = a.draft_tokens[d0 + j + i] == s_w[i];
+        const unsigned b = __ballot_sync(0xffffffffu, hit);
+        if (lane == 0) s_ballot[warp] = b;
+        __syncthreads();
+        int before = s_ncand;
+        for (int w = 0; w < warp; ++w) before += __popc(s_ballot[w]);
+        const int slot = before + __popc(b & ((1u << lane) - 1u));
+        if (hit && slot < kDsvMaxCands) {
+          s_cstart[slot] = d0 + j + n;
+          s_clen[slot] = len - (j + n);
+          s_ccur[slot] = 0;
+        }
+        __syncthreads();
+        if (tid == 0) {
+          int tot = s_ncand;
+          for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += __popc(s_ballot[w]);
+          s_ncand = min(tot, kDsvMaxCands);
+        }
+        __syncthreads();
+      }
+    }
+  }
+  __syncthreads();
+  // ---- prefix tree, level by level (warp 0; node ids 1.. in creation order, id 0 = root)
+  if (warp == 0) {
+    const int ncand = s_ncand, budget = a.max_rows - 1;
+    int nn = 0;
+    unsigned long long alive = ncand >= 64 ? ~0ull : ((1ull << ncand) - 1ull);
+    for (int depth = 0; alive && depth < HSD_MAX_TREE_ROWS; ++depth) {
+      for (int c = 0; c < ncand; ++c) {
+        if (!((alive >> c) & 1ull)) continue;
+        if (depth >= s_clen[c]) { alive &= ~(1ull << c); continue; }
+        const int u = a.draft_tokens[s_cstart[c] + depth];
+        const int cur = s_ccur[c];
+        int found = 0;
+        for (int base = 1; base <= nn && !found; base += 32) {
+          const int id = base + lane;
+          const bool hit = id <= nn && s_npar[id] == cur && s_ntok[id] == u;
+          const unsigned m = __ballot_sync(0xffffffffu, hit);
+          if (m) found = base + __ffs(m) - 1;
+        }
+        if (!found) {
+          if (nn >= budget) { alive &= ~(1ull << c); continue; }
+          ++nn;
+          if (lane == 0) { s_ntok[nn] = u; s_npar[nn] = cur; }
+          found = nn;
+        }
+        if (lane == 0) s_ccur[c] = found;
+        __syncwarp();
+      }
+    }
+    if (lane == 0) s_nnodes = nn;
+  }
+  __syncthreads();
+  // ---- packed rows
+  const int nn = s_nnodes, pending = s_w[n - 1];
+  for (int r = tid; r < a.max_rows; r += blockDim.x) {
+    const size_t o = (size_t)s * a.max_rows + r;
+    if (r == 0) { a.q_tokens[o] = pending; a.parent[o] = -1; }
+    else if (r <= nn) { a.q_tokens[o] = s_ntok[r]; a.parent[o] = s_npar[r]; }
+    else { a.q_tokens[o] = pending; a.parent[o] = -2; }
+  }
+  if (tid == 0) a.n_rows[s] = nn + 1;
+}
+void launch_dsv_build(cudaStream_t st, const DsvArgs& a, bool pdl) {
+  launch_kernel(dsv_build_kernel, dim3(a.n_seqs), dim3(128), 0, st, pdl, a);
 }
 
 // Prefill epilogue: first pending token per sequence, and seq_lens += rows.

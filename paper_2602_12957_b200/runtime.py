@@ -155,6 +155,20 @@ class Engine:
         B.check(st, "hsd_verify_tree")
         return out
 
+    def dsv_build(self, window: torch.Tensor, draft_tokens: torch.Tensor, draft_off: torch.Tensor,
+                  seq_draft_off: torch.Tensor, max_rows: int, emit_tokens: Optional[torch.Tensor] = None,
+                  n_emit: Optional[torch.Tensor] = None, out: Optional[dict] = None):
+        """Matching + prefix-tree packing on the device; `window` [S, n] is updated in place."""
+        S, n = int(window.shape[0]), int(window.shape[1])
+        if out is None:
+            i32 = lambda *s: torch.empty(*s, dtype=torch.int32, device=self.dev)
+            out = {"q_tokens": i32(S * max_rows), "parent": i32(S * max_rows), "cu_q": i32(S + 1), "n_rows": i32(S)}
+        st = B.hsd_dsv_build(self.model.ctx, S, n, window, emit_tokens, n_emit,
+                             int(emit_tokens.shape[1]) if emit_tokens is not None else 0, draft_tokens, draft_off,
+                             seq_draft_off, max_rows, out["q_tokens"], out["parent"], out["cu_q"], out["n_rows"], _stream())
+        B.check(st, "hsd_dsv_build")
+        return out
+
     def commit_tree(self, accept_len: torch.Tensor, accept_rows: torch.Tensor, slots: Optional[torch.Tensor] = None,
                     blocks_in_use: Optional[torch.Tensor] = None):
         st = B.hsd_kv_commit_tree(self.model.ctx, self.kv.c, int(accept_len.numel()), slots, accept_len, accept_rows,

@@ -50,7 +50,7 @@ def test_status_strings(B):
 
 def test_constants_match_the_header(B):
     text = open(HEADER).read()
-    for name in ("HSD_MAX_Q_LEN", "HSD_MAX_TREE_ROWS", "HSD_KV_BLOCK", "HSD_NOALLOC_MAX_ROWS", "HSD_FLAG_SIMT_DEBUG", "HSD_FLAG_SIMT_ATTENTION",
+    for name in ("HSD_MAX_Q_LEN", "HSD_MAX_TREE_ROWS", "HSD_MAX_WINDOW", "HSD_DSV_MAX_CANDIDATES", "HSD_KV_BLOCK", "HSD_NOALLOC_MAX_ROWS", "HSD_FLAG_SIMT_DEBUG", "HSD_FLAG_SIMT_ATTENTION",
                  "HSD_FLAG_DETERMINISTIC", "HSD_FLAG_NO_PDL", "HSD_FLAG_NO_PAIR", "HSD_FLAG_NO_HOST_GRAPH"):
         m = re.search(rf"#define\s+{name}\s+(-?\d+)", text)
         assert m and int(m.group(1)) == getattr(B, name), name
@@ -83,6 +83,8 @@ def test_host_side_argument_checks_need_no_device(B):
     assert B.hsd_verify_tree(None, None, 1, None, None, None, None, 1, 1, 0.0, None, None, None, None, None, None, None,
                              None, 0, None) == B.HSD_ERR_INVALID_ARG
     assert B.hsd_kv_commit_tree(None, None, 1, None, None, None, 1, None, None) == B.HSD_ERR_INVALID_ARG
+    assert B.hsd_dsv_build(None, 1, 3, None, None, None, 0, None, None, None, 128, None, None, None, None,
+                           None) == B.HSD_ERR_INVALID_ARG
 
 
 def test_binding_refuses_to_import_without_the_library(tmp_path, B):
