@@ -111,16 +111,17 @@ WORKLOADS = {
     "page": "page-level stage, one chunk mid-schedule: batch 1, 6400 committed tokens, chunk of 512 draft tokens",
     "long1024": "long-document page verify, one chunk mid-schedule: batch 1, 10240 committed tokens, chunk of 1024",
     "long2048": "long-document page verify, one chunk mid-schedule: batch 1, 10240 committed tokens, chunk of 2048",
-    "tree": "candidate-tree verification (the paper's packed form): the region batch's 16 prefixes (256-1024), each with a "
-            "prefix tree of 127 nodes packed into 128 rows (one planted main path + 6 side branches), tau 0.75, "
-            "followed by the compaction of the accepted path's K/V rows",
+    "tree": "one step of the decoupled-verification loop on the region batch's 16 prefixes (256-1024): window matching "
+            "(n = 3) against two damaged copies of each region's text and prefix-tree packing on the device (128 rows "
+            "per sequence), tree verification at tau 0.75, compaction of the accepted path's K/V rows",
     "mixed": "mixed serving batch: 64 regions (prefix 128-2048, lognormal drafts mean 96, 8-512) + 2 page chunks of 1024 "
              "over 4352-token prefixes, one varlen launch",
 }
 
 
 TREE_NODES = 127     # nodes below the root: 128 packed rows per sequence, the paper's packing limit (Sec. 4.3)
-TREE_MAIN = 64       # about this many of them lie on the main path
+TREE_MAIN = 64       # the planted agreement lengths of the region workload are scaled to this many tokens
+WINDOW_N = 3         # reference window (Sec. 4.3)
 LOG_TAU_TREE = float(np.log(0.75))
 
 
@@ -157,11 +158,11 @@ def build_gpu_state(args, rank):
     del weights
     seqs = wl.seqs
     S = len(seqs)
-    kv = R.KvCache(model, [s.prefix_len + s.draft_len + 2 for s in seqs], seed=wl.seed)
+    tree = getattr(args, "workload", "region") == "tree"
+    kv = R.KvCache(model, [s.prefix_len + s.draft_len + 2 + (2 * WINDOW_N if tree else 0) for s in seqs], seed=wl.seed)
     ks = [s.draft_len for s in seqs]
     total_q = sum(ks) + S
     total_prefix = sum(s.prefix_len for s in seqs)
-    tree = wl is not None and getattr(args, "workload", "region") == "tree"
     eng = R.Engine(model, kv, max(total_prefix, 2 * total_q if tree else total_q), S)
     first = eng.prefill([s.prefix_embeds for s in seqs], [s.prefix_ids for s in seqs])
     eng.check_device("prefill")
@@ -170,7 +171,7 @@ def build_gpu_state(args, rank):
     # greedy continuation by plain one-token steps (empty drafts), to plant the agreement lengths
     need = 0 if args.random_drafts else max(min(s.agree_len + 1, s.draft_len) for s in seqs)
     if tree:
-        need = TREE_NODES
+        need = TREE_NODES + WINDOW_N
     cu1 = eng._i32(np.arange(S + 1))
     out1 = eng.alloc_outputs(S, 1, S)
     pending = first.clone()
@@ -190,14 +191,33 @@ def build_gpu_state(args, rank):
     else:
         drafts = [I.plant_draft(greedy[i], s.draft_len, s.agree_len, s.rand_tokens, cfg.vocab, False)
                   for i, s in enumerate(seqs)]
-    parent = None
+    dsv = None
     if tree:
-        planted = [I.plant_tree(greedy[i], TREE_NODES, s.agree_len, cfg.vocab, wl.seed + i) for i, s in enumerate(seqs)]
-        drafts = [p[0] for p in planted]
-        parent = np.concatenate([p[1] for p in planted]).astype(np.int32)
+        # The region's text = the library's own greedy continuation; its first WINDOW_N tokens count as accepted (their
+        # K/V rows were written by the one-token steps above), the rest is what the two "pipeline drafts" try to
+        # predict: copies of the text with substitution errors, the first one where the workload plants its
+        # disagreement.  Matching the window against them gives two candidates that share a prefix.
+        f = first.cpu().numpy()
+        texts = [np.concatenate([[f[i]], greedy[i]]).astype(np.int32) for i in range(S)]
+        d_list, off, soff = [], [0], [0]
+        for i, s in enumerate(seqs):
+            a_, b_ = texts[i].copy(), texts[i].copy()
+            e1 = min(WINDOW_N + s.agree_len, len(a_) - 1)
+            a_[e1] = (a_[e1] + 1) % cfg.vocab
+            e2 = min(WINDOW_N + max(1, s.agree_len // 2), len(b_) - 1)
+            b_[e2] = (b_[e2] + 2) % cfg.vocab
+            for d_ in (a_, b_):
+                d_list.append(d_)
+                off.append(off[-1] + len(d_))
+            soff.append(len(off) - 1)
+        prefix_lens = prefix_lens + (WINDOW_N - 1)
+        kv.seq_lens.copy_(prefix_lens)
+        dsv = dict(window=np.stack([t[:WINDOW_N] for t in texts]).astype(np.int32), tokens=np.concatenate(d_list),
+                   off=np.asarray(off, np.int32), soff=np.asarray(soff, np.int32))
+        drafts = [np.zeros(TREE_NODES, np.int32) for _ in seqs]     # shapes only: the device packs the rows
     toks, cu = I.pack_queries(first.cpu().numpy(), drafts)
     return dict(cfg=cfg, wl=wl, model=model, kv=kv, eng=eng, toks=toks, cu=cu, total_q=total_q, max_q=max(ks) + 1,
-                prefix_lens=prefix_lens, ks=ks, S=S, drafts=drafts, parent=parent)
+                prefix_lens=prefix_lens, ks=ks, S=S, drafts=drafts, dsv=dsv)
 
 
 def kernel_work_table(cfg, work: RF.StepWork, T: int):
@@ -233,15 +253,20 @@ def run_ours(args):
     d_toks, d_cu = eng._i32(st["toks"]), eng._i32(st["cu"])
     out = eng.alloc_outputs(S, max_q, T)
     stream = torch.cuda.Stream(device=dev)
-    tree = st["parent"] is not None
+    tree = st["dsv"] is not None
     if tree:
-        d_parent = eng._i32(st["parent"])
+        dsv = st["dsv"]
+        d_window = eng._i32(dsv["window"])
+        d_dtok, d_doff, d_dsoff = eng._i32(dsv["tokens"]), eng._i32(dsv["off"]), eng._i32(dsv["soff"])
+        i32 = lambda *shape: torch.empty(*shape, dtype=torch.int32, device=dev)
+        bout = {"q_tokens": i32(T), "parent": i32(T), "cu_q": i32(S + 1), "n_rows": i32(S)}
         out["accept_rows"] = torch.zeros(S, max_q, dtype=torch.int32, device=dev)
         out["row_zchild"] = out.pop("row_zdraft")
 
     def step():
         if tree:
-            eng.verify_tree(d_toks, d_cu, d_parent, max_q, T, out=out, log_tau=LOG_TAU_TREE)
+            eng.dsv_build(d_window, d_dtok, d_doff, d_dsoff, max_q, out=bout)
+            eng.verify_tree(bout["q_tokens"], bout["cu_q"], bout["parent"], max_q, T, out=out, log_tau=LOG_TAU_TREE)
             eng.commit_tree(out["accept_len"], out["accept_rows"])
         else:
             eng.verify_regions(d_toks, d_cu, max_q, T, out=out)
@@ -302,6 +327,8 @@ def run_ours(args):
         ms_total = float(tt.item())
     ms_step = ms_total / args.steps
     draft_tokens = sum(st["ks"])
+    if tree:          # the nodes the device actually packed
+        draft_tokens = int(bout["n_rows"].sum().item()) - S
     value = draft_tokens * world / (ms_step * 1e-3)
 
     # ---- end to end through the C-ABI call that takes HOST buffers (pinned): every step copies the packed drafts
@@ -314,14 +341,13 @@ def run_ours(args):
     e2e_steps = max(3, min(args.steps, 200))
     ctx = eng.model.ctx
 
-    h_par = torch.from_numpy(st["parent"]).pin_memory() if tree else None
+    h_win = torch.from_numpy(st["dsv"]["window"]).pin_memory() if tree else None
 
     def e2e_step():
-        if tree:     # the tree calls take device buffers: the copies are made here, on the same stream
-            d_toks.copy_(h_toks, non_blocking=True)
-            d_cu.copy_(h_cu, non_blocking=True)
-            d_parent.copy_(h_par, non_blocking=True)
-            eng.verify_tree(d_toks, d_cu, d_parent, max_q, T, out=out, log_tau=LOG_TAU_TREE)
+        if tree:     # the drafts stay resident (they are fixed per page); per step the window goes in, the results out
+            d_window.copy_(h_win, non_blocking=True)
+            eng.dsv_build(d_window, d_dtok, d_doff, d_dsoff, max_q, out=bout)
+            eng.verify_tree(bout["q_tokens"], bout["cu_q"], bout["parent"], max_q, T, out=out, log_tau=LOG_TAU_TREE)
             eng.commit_tree(out["accept_len"], out["accept_rows"])
             h_acc.copy_(out["accept_len"], non_blocking=True)
             h_nem.copy_(out["n_emit"], non_blocking=True)
@@ -349,12 +375,12 @@ def run_ours(args):
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         e2e_ms = float(tt.item())
     e2e = {"value": draft_tokens * world / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
-           "h2d_bytes_per_step": int(h_toks.numel() * 4 + h_cu.numel() * 4 + (h_par.numel() * 4 if tree else 0)),
+           "h2d_bytes_per_step": int(h_win.numel() * 4 if tree else h_toks.numel() * 4 + h_cu.numel() * 4),
            "d2h_bytes_per_step": int((h_acc.numel() + h_nem.numel() + h_emit.numel()) * 4 + 16),
            "call": "hsd_verify_regions_host (pinned host buffers; the library replays the step as a CUDA graph it captured "
                    "at the second call of this shape; stream synchronised per step)" if not tree else
-                   "hsd_verify_tree + hsd_kv_commit_tree (eager launches) with pinned-host copies in and out on the same "
-                   "stream, synchronised per step"}
+                   "hsd_dsv_build + hsd_verify_tree + hsd_kv_commit_tree (eager launches), the window copied in from and "
+                   "the results out to pinned host memory on the same stream, synchronised per step"}
     accept_mean = float(np.mean([a / k for a, k in zip(h_acc.numpy().tolist(), st["ks"])]))
 
     # ---- per-kernel durations (CUDA events around every launch, eager) for the roofline of the top kernel

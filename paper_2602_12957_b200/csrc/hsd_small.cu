@@ -550,6 +550,7 @@ __global__ void dsv_build_kernel(DsvArgs a) {
   __shared__ int s_w[kDsvMaxWindow];
   __shared__ int s_cstart[kDsvMaxCands], s_clen[kDsvMaxCands], s_ccur[kDsvMaxCands];
   __shared__ int s_ntok[HSD_MAX_TREE_ROWS], s_npar[HSD_MAX_TREE_ROWS];
+  __shared__ int s_ctok[kDsvMaxCands][HSD_MAX_TREE_ROWS];   // the part of every candidate a tree of this size can hold
   __shared__ unsigned s_ballot[4];
   __shared__ int s_ncand, s_nnodes;
   const int n = a.window_n;
@@ -611,19 +612,25 @@ __global__ void dsv_build_kernel(DsvArgs a) {
     }
   }
   __syncthreads();
+  for (int idx = tid; idx < s_ncand * HSD_MAX_TREE_ROWS; idx += blockDim.x) {
+    const int c = idx / HSD_MAX_TREE_ROWS, d = idx % HSD_MAX_TREE_ROWS;
+    s_ctok[c][d] = d < s_clen[c] ? a.draft_tokens[s_cstart[c] + d] : -1;
+  }
+  __syncthreads();
   // ---- prefix tree, level by level (warp 0; node ids 1.. in creation order, id 0 = root)
   if (warp == 0) {
     const int ncand = s_ncand, budget = a.max_rows - 1;
     int nn = 0;
     unsigned long long alive = ncand >= 64 ? ~0ull : ((1ull << ncand) - 1ull);
     for (int depth = 0; alive && depth < HSD_MAX_TREE_ROWS; ++depth) {
+      const int level0 = nn + 1;       // a node's children are all created while its level is expanded: search only those
       for (int c = 0; c < ncand; ++c) {
         if (!((alive >> c) & 1ull)) continue;
         if (depth >= s_clen[c]) { alive &= ~(1ull << c); continue; }
-        const int u = a.draft_tokens[s_cstart[c] + depth];
+        const int u = s_ctok[c][depth];
         const int cur = s_ccur[c];
         int found = 0;
-        for (int base = 1; base <= nn && !found; base += 32) {
+        for (int base = level0; base <= nn && !found; base += 32) {
           const int id = base + lane;
           const bool hit = id <= nn && s_npar[id] == cur && s_ntok[id] == u;
           const unsigned m = __ballot_sync(0xffffffffu, hit);
