@@ -37,3 +37,68 @@ def test_region_stage_full_size_sampled_rows_match_oracle():
         assert g["emit"][a] == g["row_argmax"][a] and np.all(np.isfinite(g["row_zmax"]))
     print("full size", sample, stats, [(len(orc[i].draft), orc[i].res.accept_len) for i in sample])
     assert stats["max_dz"] < H.LOGIT_TOL
+
+
+def test_tree_step_full_size_sampled_rows_match_oracle():
+    """The tree workload's shape (24 layers, 16 regions x 128 packed rows in one hsd_verify_tree call, tau = 0.75):
+    the region with the shortest prefix is checked row by row against the float32 oracle, every other region for
+    consistency between its path and its own rows."""
+    import torch
+    from oracle import hsd_oracle as O
+    from paper_2602_12957_b200 import runtime as R
+    from .test_gpu_tree import LOG_TAU_PAPER, oracle_decisive_steps, traverse_rows
+    cfg = I.DECODER
+    wl = I.region_workload(seed=I.BASE_SEED + 1, cfg=cfg)
+    weights = I.make_weights(cfg, I.BASE_SEED + 1)
+    S, NODES = len(wl.seqs), 127
+    pick = min(range(S), key=lambda i: wl.seqs[i].prefix_len)
+    model_o = O.Decoder(cfg, weights, np.float32)
+    cache = O.CachedSequence(model_o)
+    sp = wl.seqs[pick]
+    pending_o = cache.prefill(sp.prefix_embeds if np.any(sp.prefix_ids < 0) else None, sp.prefix_ids)
+    greedy = O.greedy_continuation(cache, pending_o, 25)
+    rng = np.random.default_rng(3)
+    toks_l, par_l, pend = [], [], []
+    for i in range(S):
+        if i == pick:
+            t, p, _ = I.plant_tree(greedy, NODES, 24, cfg.vocab, 1000 + i, n_branches=8)
+            pend.append(pending_o)
+        else:
+            t, p, _ = I.plant_tree(rng.integers(0, cfg.vocab, size=NODES).tolist(), NODES, 0, cfg.vocab, 1000 + i)
+            pend.append(int(rng.integers(0, cfg.vocab)))
+        toks_l.append(t); par_l.append(p)
+    res = O.verify_cached(cache, pending_o, toks_l[pick], par_l[pick], LOG_TAU_PAPER, keep_logits=True)
+    model = R.DeviceModel(cfg, weights, 0)
+    kv = R.KvCache(model, [s.prefix_len + 2 * (NODES + 1) + 16 for s in wl.seqs], seed=5, poison=True)
+    T = S * (NODES + 1)
+    eng = R.Engine(model, kv, max(sum(s.prefix_len for s in wl.seqs), 2 * T), S)
+    first = eng.prefill([s.prefix_embeds if np.any(s.prefix_ids < 0) else None for s in wl.seqs],
+                        [s.prefix_ids for s in wl.seqs])
+    eng.check_device("prefill")
+    toks, cu = I.pack_queries(pend, toks_l)
+    parent = np.concatenate(par_l).astype(np.int32)
+    out = eng.verify_tree(eng._i32(toks), eng._i32(cu), eng._i32(parent), NODES + 1, T, log_tau=LOG_TAU_PAPER)
+    eng.check_device("verify_tree")
+    torch.cuda.synchronize()
+    host = {n: t.cpu().numpy() for n, t in out.items()}
+    for i in range(S):
+        a, b = int(cu[i]), int(cu[i + 1])
+        tokens = np.concatenate([[-1], toks_l[i]])
+        am, zm, zc = host["row_argmax"][a:b], host["row_zmax"][a:b], host["row_zchild"][a:b]
+        assert np.all(np.isfinite(zm)) and np.all(np.isfinite(zc[1:]))
+        g_acc = int(host["accept_len"][i])
+        want_path, want_emit = traverse_rows(par_l[i], tokens, am, zm, zc, LOG_TAU_PAPER)
+        assert host["accept_rows"][i][:g_acc].tolist() == want_path
+        assert host["emit_tokens"][i][:g_acc + 1].tolist() == want_emit
+        if i == pick:
+            dz = np.abs(zm - res.row_zmax)
+            dc = max(abs(zc[j] - res.logits[par_l[i][j], int(tokens[j])]) for j in range(1, b - a))
+            assert dz.max() <= H.LOGIT_TOL and dc <= H.LOGIT_TOL, (dz.max(), dc)
+            for j in range(b - a):
+                if res.row_gap[j] > H.GAP_EXACT:
+                    assert am[j] == res.row_argmax[j]
+            clear = oracle_decisive_steps(res, par_l[i], tokens, LOG_TAU_PAPER)
+            m = min(clear, len(res.path))
+            assert want_path[:m] == list(res.path)[:m]
+            print("full-size tree", pick, "max dz", float(dz.max()), "max dzchild", float(dc), "oracle path", len(res.path),
+                  "clear decisions", clear, "library path", g_acc)
