@@ -433,45 +433,70 @@ __global__ void tree_accept_kernel(TreeAcceptArgs a, RowMeta rm, const int* stat
   }
   int* emit = a.emit_tokens + (size_t)i * a.max_q_len;
   int* path = a.accept_rows + (size_t)i * a.max_q_len;
+  // every lane keeps four nodes (lane, lane + 32, ..) in registers: the walk itself then only fetches the row it
+  // stands on
+  constexpr int kPer = HSD_MAX_TREE_ROWS / 32;
+  int npar[kPer], ntok[kPer];
+  float nz[kPer];
+#pragma unroll
+  for (int k = 0; k < kPer; ++k) {
+    const int c = lane + 32 * k;
+    const bool in = c >= 1 && c < n;
+    npar[k] = in ? a.parent[q0 + c] : -3;
+    ntok[k] = in ? rm.row_tok[q0 + c] : -1;
+    nz[k] = in ? a.zdraft[T + q0 + c] : 0.f;
+  }
   int s = 0, acc = 0;
   for (int step = 0; step < n; ++step) {
     const unsigned long long best = a.row_best[q0 + s];
     const int uhat = key_col(best);
-    int pick = -1;
+    int pick = -1, pick_tok = -1;
+    float pick_z = 0.f;
     if (a.log_tau == 0.f) {
-      for (int c0 = 1; c0 < n && pick < 0; c0 += 32) {
-        const int c = c0 + lane;
-        const bool hit = c < n && a.parent[q0 + c] == s && rm.row_tok[q0 + c] == uhat;
-        const unsigned m = __ballot_sync(0xffffffffu, hit);
-        if (m) pick = c0 + __ffs(m) - 1;
-      }
+      // the child that carries u_hat (lowest row if a caller packed the same token twice under one parent)
+      int mine = 0x7fffffff;
+#pragma unroll
+      for (int k = kPer - 1; k >= 0; --k)
+        if (npar[k] == s && ntok[k] == uhat) mine = lane + 32 * k;
+      for (int o = 16; o; o >>= 1) mine = min(mine, __shfl_xor_sync(0xffffffffu, mine, o));
+      if (mine != 0x7fffffff) pick = mine;
     } else {
       // best child by (score, then lower token id), then lower row among equals
       unsigned long long bk = 0ull;
-      int bc = -1;
-      for (int c = 1 + lane; c < n; c += 32) {
-        if (a.parent[q0 + c] != s) continue;
-        const unsigned long long k = argmax_key(a.zdraft[T + q0 + c], rm.row_tok[q0 + c]);
-        if (bc < 0 || k > bk) { bk = k; bc = c; }
+      int bc = 0x7fffffff;
+#pragma unroll
+      for (int k = 0; k < kPer; ++k) {
+        if (npar[k] != s) continue;
+        const unsigned long long key = argmax_key(nz[k], ntok[k]);
+        if (bc == 0x7fffffff || key > bk) { bk = key; bc = lane + 32 * k; }
       }
-      unsigned long long wk = bc >= 0 ? bk : 0ull;
+      unsigned long long wk = bc != 0x7fffffff ? bk : 0ull;
+      const unsigned has = __ballot_sync(0xffffffffu, bc != 0x7fffffff);
       for (int o = 16; o; o >>= 1) {
-        const unsigned long long ok2 = __shfl_xor_sync(0xffffffffu, wk, o);
-        wk = ok2 > wk ? ok2 : wk;
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, wk, o);
+        wk = other > wk ? other : wk;
       }
-      const unsigned has = __ballot_sync(0xffffffffu, bc >= 0);
       if (has) {
-        const int cand = (bc >= 0 && bk == wk) ? bc : 0x7fffffff;
-        int lo = cand;
+        int lo = (bc != 0x7fffffff && bk == wk) ? bc : 0x7fffffff;
         for (int o = 16; o; o >>= 1) lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
         pick = lo;
-        if (!(a.zdraft[T + q0 + pick] - key_value(best) >= a.log_tau)) pick = -1;
       }
+    }
+    if (pick >= 0) {      // the owner lane broadcasts the node's token and score
+      const int owner = pick & 31, k = pick >> 5;
+      int tk = -1;
+      float zk = 0.f;
+#pragma unroll
+      for (int kk = 0; kk < kPer; ++kk)
+        if (kk == k) { tk = ntok[kk]; zk = nz[kk]; }
+      pick_tok = __shfl_sync(0xffffffffu, tk, owner);
+      pick_z = __shfl_sync(0xffffffffu, zk, owner);
+      if (a.log_tau != 0.f && !(pick_z - key_value(best) >= a.log_tau)) pick = -1;
     }
     if (pick < 0) break;
     if (lane == 0) {
       path[acc] = pick;
-      emit[acc] = rm.row_tok[q0 + pick];
+      emit[acc] = pick_tok;
     }
     ++acc;
     s = pick;
