@@ -411,7 +411,8 @@ def run_ours(args):
         roof = {"kernel": top, "bound": "hbm", "achieved": nbytes / dur / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = NCU_TRAFFIC_BYTES.get(top) if args.workload == "region" else None
-    roof["peak_source"] = f"{peak_src} (sustained bf16 figure: kernel timed inside a long step)"
+    roof["peak_source"] = (f"{peak_src} (sustained bf16 figure: kernel timed inside a long step)" if roof["bound"] == "tensor"
+                           else f"{peak_src} (STREAM-style copy bandwidth)")
     roof["us_per_launch"] = dur * 1e6
     t_roof = RF.roofline_time(work.bytes, work.flops, bw, pk)
     step_roof = {"roofline_us": t_roof * 1e6, "frac": t_roof / (ms_step * 1e-3), "bytes": work.bytes, "flops": work.flops,
