@@ -15,7 +15,8 @@ What it computes (paper Sec. 3.2, "Verification and acceptance"):
 
 The decoder itself (pre-norm RMSNorm, rotary positions with rotate-half pairing,
 grouped-query causal attention softmax(QK^T/sqrt(d))V, SwiGLU FFN, untied LM head, no
-biases) is fixed by the benchmark configurations, not by the paper.
+biases) is fixed by the benchmark configurations, not by the paper; `qk_norm` adds the per-head RMSNorm of q and k
+before the rotary embedding that the Qwen3-family decoders the paper evaluates carry.
 
 Readings where the paper is silent:
   * the most recent emitted token has no K/V yet ("pending" token); it is query row 0
@@ -140,6 +141,8 @@ def decoder_forward(model: Decoder, x: np.ndarray, pos: np.ndarray, allowed: np.
         q = qkv[:, :Hq * D].reshape(-1, Hq, D)
         k = qkv[:, Hq * D:(Hq + Hkv) * D].reshape(-1, Hkv, D)
         v = qkv[:, (Hq + Hkv) * D:].reshape(-1, Hkv, D)
+        if c.qk_norm:       # per-head RMSNorm over head_dim, before the rotary embedding
+            q, k = rmsnorm(q, model.w(lw["q_norm"]), c.rms_eps), rmsnorm(k, model.w(lw["k_norm"]), c.rms_eps)
         q, k = rope(q, pos, c.rope_base), rope(k, pos, c.rope_base)
         o = attention(q, k, v, allowed).reshape(-1, Hq * D)
         x = x + o @ model.w(lw["w_o"]).T
@@ -177,8 +180,11 @@ class CachedSequence:
         for li, lw in enumerate(model.weights["layers"]):
             h = rmsnorm(x, model.w(lw["attn_norm"]), c.rms_eps)
             qkv = h @ model.w(lw["w_qkv"]).T
-            q = rope(qkv[:, :Hq * D].reshape(m, Hq, D), pos, c.rope_base)
-            k = rope(qkv[:, Hq * D:(Hq + Hkv) * D].reshape(m, Hkv, D), pos, c.rope_base)
+            q = qkv[:, :Hq * D].reshape(m, Hq, D)
+            k = qkv[:, Hq * D:(Hq + Hkv) * D].reshape(m, Hkv, D)
+            if c.qk_norm:
+                q, k = rmsnorm(q, model.w(lw["q_norm"]), c.rms_eps), rmsnorm(k, model.w(lw["k_norm"]), c.rms_eps)
+            q, k = rope(q, pos, c.rope_base), rope(k, pos, c.rope_base)
             v = qkv[:, (Hq + Hkv) * D:].reshape(m, Hkv, D)
             spec.append((k, v))
             o = attention(q, np.concatenate([self.k[li], k]), np.concatenate([self.v[li], v]), allowed)

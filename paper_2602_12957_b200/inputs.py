@@ -38,6 +38,7 @@ class ModelConfig:
     rope_base: float = 10000.0
     rms_eps: float = 1e-6
     kv_block: int = 64
+    qk_norm: bool = False      # per-head RMSNorm of q and k before the rotary embedding (Qwen3-style decoders)
 
     @property
     def qkv_out(self) -> int:
@@ -111,12 +112,18 @@ def make_weights(cfg: ModelConfig, seed: int) -> Dict[str, object]:
             "w_gate_up": lin(2 * f, d),
             "w_down": lin(d, f),
         })
-    return {
+    out = {
         "layers": layers,
         "embed": lin(cfg.vocab, d),
         "final_norm": gain(),
         "lm_head": lin(cfg.vocab, d),
     }
+    if cfg.qk_norm:     # drawn from a stream of their own, so every other weight is the same with and without them
+        rq = np.random.Generator(np.random.PCG64(seed + 7_000_001))
+        for lw in layers:
+            for name in ("q_norm", "k_norm"):
+                lw[name] = bf16_round(np.float32(1.0) + np.float32(0.1) * rq.standard_normal(hd, dtype=np.float32))
+    return out
 
 
 # --------------------------------------------------------------------------- workloads

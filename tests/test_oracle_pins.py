@@ -533,3 +533,56 @@ def test_float32_mode_tracks_float64():
     emb, ids = mixed_prefix(m64, 12, 4, 19)
     z64, z32 = oracle_full_logits(m64, emb, ids), oracle_full_logits(m32, emb, ids)
     assert z32.dtype == np.float32 and np.max(np.abs(z64 - z32)) < 1e-4
+
+
+# ------------------------------------------------------------------ per-head QK-norm vs a library decoder that has it
+def hf_qwen3(model):
+    """The decoder with per-head q/k RMSNorm as a Hugging Face Qwen3 (library routine)."""
+    from transformers import Qwen3Config, Qwen3ForCausalLM
+    c = model.cfg
+    hc = Qwen3Config(vocab_size=c.vocab, hidden_size=c.d_model, intermediate_size=c.d_ffn,
+                     num_hidden_layers=c.n_layers, num_attention_heads=c.n_heads,
+                     num_key_value_heads=c.n_kv_heads, head_dim=c.head_dim, rms_norm_eps=c.rms_eps,
+                     rope_theta=c.rope_base, attention_bias=False, tie_word_embeddings=False,
+                     max_position_embeddings=4096, use_sliding_window=False, attn_implementation="eager")
+    m = Qwen3ForCausalLM(hc).double().eval()
+    W = model.weights
+    t = lambda a: torch.from_numpy(np.asarray(a, np.float64))
+    sd = {"model.embed_tokens.weight": t(W["embed"]), "model.norm.weight": t(W["final_norm"]),
+          "lm_head.weight": t(W["lm_head"])}
+    Hq, Hkv, D, f = c.n_heads, c.n_kv_heads, c.head_dim, c.d_ffn
+    for i, lw in enumerate(W["layers"]):
+        p = f"model.layers.{i}."
+        sd[p + "input_layernorm.weight"] = t(lw["attn_norm"])
+        sd[p + "post_attention_layernorm.weight"] = t(lw["ffn_norm"])
+        sd[p + "self_attn.q_proj.weight"] = t(lw["w_qkv"][:Hq * D])
+        sd[p + "self_attn.k_proj.weight"] = t(lw["w_qkv"][Hq * D:(Hq + Hkv) * D])
+        sd[p + "self_attn.v_proj.weight"] = t(lw["w_qkv"][(Hq + Hkv) * D:])
+        sd[p + "self_attn.o_proj.weight"] = t(lw["w_o"])
+        sd[p + "self_attn.q_norm.weight"] = t(lw["q_norm"])
+        sd[p + "self_attn.k_norm.weight"] = t(lw["k_norm"])
+        sd[p + "mlp.gate_proj.weight"] = t(lw["w_gate_up"][:f])
+        sd[p + "mlp.up_proj.weight"] = t(lw["w_gate_up"][f:])
+        sd[p + "mlp.down_proj.weight"] = t(lw["w_down"])
+    missing, unexpected = m.load_state_dict(sd, strict=False)
+    assert not unexpected and all("rotary" in k or "inv_freq" in k for k in missing), (missing, unexpected)
+    return m
+
+
+def test_qk_norm_forward_matches_library_qwen3_and_changes_the_result():
+    cfg = I.ModelConfig(n_layers=2, d_model=128, n_heads=4, n_kv_heads=2, head_dim=64, d_ffn=256, vocab=61, qk_norm=True)
+    model = small_model(7, cfg)
+    emb, ids = mixed_prefix(model, 19, 5, 3)
+    z = oracle_full_logits(model, emb, ids)
+    m = hf_qwen3(model)
+    x = torch.from_numpy(model.embed_rows(emb, ids))[None]
+    with torch.no_grad():
+        zr = m(inputs_embeds=x).logits[0].numpy()
+    assert np.max(np.abs(z - zr)) < 2e-7
+    # the cached form agrees with the stateless one, and without the norm the logits differ
+    cache = O.CachedSequence(model)
+    cache.prefill(emb, ids)
+    assert np.max(np.abs(cache.last_prefill_logits - z[-1])) < 1e-9
+    plain = I.ModelConfig(n_layers=2, d_model=128, n_heads=4, n_kv_heads=2, head_dim=64, d_ffn=256, vocab=61)
+    model_p = O.Decoder(plain, model.weights, np.float64)
+    assert np.max(np.abs(oracle_full_logits(model_p, emb, ids) - z)) > 1e-3
