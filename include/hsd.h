@@ -89,6 +89,8 @@ typedef struct {
   float rms_eps;     /* RMSNorm epsilon                                                               */
   int kv_block;      /* must be 64                                                                    */
   int flags;         /* HSD_FLAG_*                                                                    */
+  int qk_norm;       /* 1: per-head RMSNorm (over head_dim, rms_eps) of q and k before the rotary embedding,
+                        with the gains hsd_weights.q_norm / k_norm (Qwen3-style decoders); 0: none     */
 } hsd_model_config;
 
 /* Device pointers to bf16 weights.  The per-layer members are HOST arrays of n_layers device pointers. */
@@ -96,6 +98,7 @@ typedef struct {
   const void *embed, *lm_head, *final_norm;
   const void *const *attn_norm, *const *w_qkv, *const *w_o;
   const void *const *ffn_norm, *const *w_gate_up, *const *w_down;
+  const void *const *q_norm, *const *k_norm;   /* bf16 [head_dim] per layer; read only when qk_norm = 1, else may be NULL */
 } hsd_weights;
 
 /* Caller-owned paged KV cache.  All pointers are device pointers. */

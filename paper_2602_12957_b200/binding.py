@@ -48,14 +48,15 @@ class HsdError(RuntimeError):
 class hsd_model_config(C.Structure):
     _fields_ = [("n_layers", C.c_int), ("d_model", C.c_int), ("n_heads", C.c_int), ("n_kv_heads", C.c_int),
                 ("head_dim", C.c_int), ("d_ffn", C.c_int), ("vocab", C.c_int), ("rope_base", C.c_float),
-                ("rms_eps", C.c_float), ("kv_block", C.c_int), ("flags", C.c_int)]
+                ("rms_eps", C.c_float), ("kv_block", C.c_int), ("flags", C.c_int), ("qk_norm", C.c_int)]
 
 
 class hsd_weights(C.Structure):
     _fields_ = [("embed", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p),
                 ("attn_norm", C.POINTER(C.c_void_p)), ("w_qkv", C.POINTER(C.c_void_p)),
                 ("w_o", C.POINTER(C.c_void_p)), ("ffn_norm", C.POINTER(C.c_void_p)),
-                ("w_gate_up", C.POINTER(C.c_void_p)), ("w_down", C.POINTER(C.c_void_p))]
+                ("w_gate_up", C.POINTER(C.c_void_p)), ("w_down", C.POINTER(C.c_void_p)),
+                ("q_norm", C.POINTER(C.c_void_p)), ("k_norm", C.POINTER(C.c_void_p))]
 
 
 class hsd_kv(C.Structure):
@@ -125,11 +126,13 @@ def check(status: int, what: str = "") -> int:
 
 def make_config(cfg, flags: int = 0) -> hsd_model_config:
     return hsd_model_config(cfg.n_layers, cfg.d_model, cfg.n_heads, cfg.n_kv_heads, cfg.head_dim, cfg.d_ffn,
-                            cfg.vocab, cfg.rope_base, cfg.rms_eps, cfg.kv_block, flags)
+                            cfg.vocab, cfg.rope_base, cfg.rms_eps, cfg.kv_block, flags,
+                            1 if getattr(cfg, "qk_norm", False) else 0)
 
 
 def make_weights(embed, lm_head, final_norm, attn_norm: Sequence, w_qkv: Sequence, w_o: Sequence,
-                 ffn_norm: Sequence, w_gate_up: Sequence, w_down: Sequence) -> hsd_weights:
+                 ffn_norm: Sequence, w_gate_up: Sequence, w_down: Sequence, q_norm: Optional[Sequence] = None,
+                 k_norm: Optional[Sequence] = None) -> hsd_weights:
     def arr(ts):
         a = (C.c_void_p * len(ts))(*[t.data_ptr() if t is not None else None for t in ts])
         return a
@@ -137,7 +140,9 @@ def make_weights(embed, lm_head, final_norm, attn_norm: Sequence, w_qkv: Sequenc
     w.embed, w.lm_head, w.final_norm = embed.data_ptr(), lm_head.data_ptr(), final_norm.data_ptr()
     keep = []
     for name, ts in (("attn_norm", attn_norm), ("w_qkv", w_qkv), ("w_o", w_o), ("ffn_norm", ffn_norm),
-                     ("w_gate_up", w_gate_up), ("w_down", w_down)):
+                     ("w_gate_up", w_gate_up), ("w_down", w_down), ("q_norm", q_norm), ("k_norm", k_norm)):
+        if ts is None:
+            continue
         a = arr(ts)
         keep.append(a)
         setattr(w, name, C.cast(a, C.POINTER(C.c_void_p)))

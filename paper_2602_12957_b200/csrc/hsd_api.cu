@@ -33,6 +33,7 @@ struct hsd_ctx {
   ModelDims md;
   const bf16 *embed, *lm_head, *final_norm;
   std::vector<const bf16*> attn_norm, w_qkv, w_o, ffn_norm, w_gate_up, w_down;
+  std::vector<const bf16*> q_norm, k_norm;    // per layer, nullptr when the model has no per-head q/k norm
   std::vector<WeightMaps> tm_qkv, tm_o, tm_gate_up, tm_down;
   WeightMaps tm_lm_head;
   int max_splits;     // K slices the residual-add projections may use (1 with HSD_FLAG_DETERMINISTIC)
@@ -293,7 +294,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
       }
       {
         Scope s(c, st, KC_ROPE_KV);
-        launch_rope_kvwrite(st, w.qkv_f32, w.rm, kv, md, l, w.q, T, w.status);
+        launch_rope_kvwrite(st, w.qkv_f32, w.rm, kv, md, l, w.q, T, w.status, c->q_norm[l], c->k_norm[l]);
       }
       {
         Scope s(c, st, KC_ATTN);
@@ -318,6 +319,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         g.qkv.k_pool_layer = kv.k_pool + (size_t)l * layer_elems;
         g.qkv.v_pool_layer = kv.v_pool + (size_t)l * layer_elems;
         g.qkv.Hq = md.Hq; g.qkv.Hkv = md.Hkv;
+        g.qkv.q_norm = c->q_norm[l]; g.qkv.k_norm = c->k_norm[l]; g.qkv.eps = md.eps;
         g.status = w.status; g.n_sms = c->n_sms; g.max_splits = 1; g.pdl = c->pdl; g.pair = c->pair;
         g.force_bn = c->force_bn;
         if (launch_gemm_sm100(st, g)) return fail_cuda(c);
@@ -486,6 +488,11 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
   for (int l = 0; l < cfg->n_layers; ++l)
     if (!w->attn_norm[l] || !w->w_qkv[l] || !w->w_o[l] || !w->ffn_norm[l] || !w->w_gate_up[l] || !w->w_down[l])
       return HSD_ERR_INVALID_ARG;
+  if (cfg->qk_norm) {
+    if (!w->q_norm || !w->k_norm) return HSD_ERR_INVALID_ARG;
+    for (int l = 0; l < cfg->n_layers; ++l)
+      if (!w->q_norm[l] || !w->k_norm[l]) return HSD_ERR_INVALID_ARG;
+  }
 
   int dev = 0;
   cudaDeviceProp prop;
@@ -509,6 +516,8 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
     c->ffn_norm.push_back(static_cast<const bf16*>(w->ffn_norm[l]));
     c->w_gate_up.push_back(static_cast<const bf16*>(w->w_gate_up[l]));
     c->w_down.push_back(static_cast<const bf16*>(w->w_down[l]));
+    c->q_norm.push_back(cfg->qk_norm ? static_cast<const bf16*>(w->q_norm[l]) : nullptr);
+    c->k_norm.push_back(cfg->qk_norm ? static_cast<const bf16*>(w->k_norm[l]) : nullptr);
   }
   c->n_sms = prop.multiProcessorCount;
   c->device = dev;

@@ -430,6 +430,27 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           tmem_ld32(t_acc + hh * 64, lo);
           tmem_ld32(t_acc + hh * 64 + 32, hi);
           tmem_ld_wait();
+          if (p.qkv.q_norm && head < p.qkv.Hq + p.qkv.Hkv && row_ok) {
+            // per-head RMSNorm of q and k over the head's 64 dims (all in this thread) before the rotation
+            float ss = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              ss += __uint_as_float(lo[i]) * __uint_as_float(lo[i]) + __uint_as_float(hi[i]) * __uint_as_float(hi[i]);
+            const float rs = rsqrtf(ss * (1.f / 64.f) + p.qkv.eps);
+            const uint4* g4 = reinterpret_cast<const uint4*>(is_q ? p.qkv.q_norm : p.qkv.k_norm);
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              const uint4 gl = __ldg(g4 + v), gh = __ldg(g4 + 4 + v);
+              const uint32_t wl[4] = {gl.x, gl.y, gl.z, gl.w}, wh[4] = {gh.x, gh.y, gh.z, gh.w};
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                lo[8 * v + 2 * k] = __float_as_uint(__uint_as_float(lo[8 * v + 2 * k]) * rs * bf16_lo(wl[k]));
+                lo[8 * v + 2 * k + 1] = __float_as_uint(__uint_as_float(lo[8 * v + 2 * k + 1]) * rs * bf16_hi(wl[k]));
+                hi[8 * v + 2 * k] = __float_as_uint(__uint_as_float(hi[8 * v + 2 * k]) * rs * bf16_lo(wh[k]));
+                hi[8 * v + 2 * k + 1] = __float_as_uint(__uint_as_float(hi[8 * v + 2 * k + 1]) * rs * bf16_hi(wh[k]));
+              }
+            }
+          }
           if (head < p.qkv.Hq + p.qkv.Hkv && row_ok) {
 #pragma unroll
             for (int i = 0; i < 16; ++i) {

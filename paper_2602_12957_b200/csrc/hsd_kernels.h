@@ -73,8 +73,9 @@ void launch_rmsnorm(cudaStream_t st, const float* x, const bf16* gain, bf16* h, 
                     const int* sel_rows, bool pdl);
 // last row of every sequence (prefill's LM-head rows)
 void launch_select_last_rows(cudaStream_t st, const RowMeta& rm, int n_seqs, int* sel_rows, bool pdl);
+// q_norm / k_norm: per-head RMSNorm gains applied before the rotation, or nullptr
 void launch_rope_kvwrite(cudaStream_t st, const float* qkv, const RowMeta& rm, const KvView& kv, const ModelDims& md,
-                         int layer, bf16* q, int T, const int* status);
+                         int layer, bf16* q, int T, const int* status, const bf16* q_norm, const bf16* k_norm);
 void launch_attn_simt(cudaStream_t st, const bf16* q, const RowMeta& rm, const KvView& kv, const ModelDims& md,
                       int layer, bf16* out, int T, const int* status);
 struct AcceptArgs {
@@ -185,6 +186,9 @@ struct QkvEpilogue {      // fused RoPE + paged KV write (QKV projection)
   bf16* k_pool_layer;     // layer base of the K pool
   bf16* v_pool_layer;
   int Hq, Hkv;
+  const bf16* q_norm;     // per-head RMSNorm gains [64] of q and k before the rotation, or nullptr (none)
+  const bf16* k_norm;
+  float eps;
 };
 struct GemmSm100Args {
   CUtensorMap tmA;             // activations, box {64, 128}

@@ -263,7 +263,8 @@ void launch_unpack_best(cudaStream_t st, const unsigned long long* row_best, int
 // RoPE + paged KV write from an fp32 qkv row (SIMT path; the tensor-core path fuses this into the
 // QKV projection's epilogue).  One warp per (row, head); lane i holds dims i and i + 32.
 __global__ void rope_kvwrite_kernel(const float* __restrict__ qkv, RowMeta rm, KvView kv, ModelDims md, int layer,
-                                    bf16* __restrict__ q, int T, const int* status) {
+                                    bf16* __restrict__ q, int T, const int* status, const bf16* __restrict__ q_norm,
+                                    const bf16* __restrict__ k_norm) {
   if (*status) return;
   const int heads = md.Hq + 2 * md.Hkv;
   const int w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -275,6 +276,14 @@ __global__ void rope_kvwrite_kernel(const float* __restrict__ qkv, RowMeta rm, K
   const size_t blk_base = ((size_t)layer * kv.n_blocks + phys / 64) * md.Hkv;
   const int off = phys % 64;
   if (hd < md.Hq + md.Hkv) {
+    if (q_norm) {       // per-head RMSNorm over the 64 dims before the rotation
+      float ss = a * a + b * b;
+      for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      const float rs = rsqrtf(ss * (1.f / 64.f) + md.eps);
+      const bf16* g = hd < md.Hq ? q_norm : k_norm;
+      a *= rs * __bfloat162float(g[lane]);
+      b *= rs * __bfloat162float(g[lane + 32]);
+    }
     const float2 cs = rm.rope_cs[(size_t)r * 32 + lane];
     const float ra = a * cs.x - b * cs.y, rb = b * cs.x + a * cs.y;
     if (hd < md.Hq) {
@@ -293,9 +302,9 @@ __global__ void rope_kvwrite_kernel(const float* __restrict__ qkv, RowMeta rm, K
   }
 }
 void launch_rope_kvwrite(cudaStream_t st, const float* qkv, const RowMeta& rm, const KvView& kv, const ModelDims& md,
-                         int layer, bf16* q, int T, const int* status) {
+                         int layer, bf16* q, int T, const int* status, const bf16* q_norm, const bf16* k_norm) {
   const long long warps = (long long)T * (md.Hq + 2 * md.Hkv);
-  rope_kvwrite_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(qkv, rm, kv, md, layer, q, T, status);
+  rope_kvwrite_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(qkv, rm, kv, md, layer, q, T, status, q_norm, k_norm);
 }
 
 // ------------------------------------------------------------------------------------------------

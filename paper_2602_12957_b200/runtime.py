@@ -34,7 +34,8 @@ class DeviceModel:
         self._cfg_c = B.make_config(cfg, flags)
         col = lambda k: [lw[k] for lw in self.layers]
         self._w_c = B.make_weights(self.embed, self.lm_head, self.final_norm, col("attn_norm"), col("w_qkv"), col("w_o"),
-                                   col("ffn_norm"), col("w_gate_up"), col("w_down"))
+                                   col("ffn_norm"), col("w_gate_up"), col("w_down"),
+                                   col("q_norm") if cfg.qk_norm else None, col("k_norm") if cfg.qk_norm else None)
         st, self.ctx = B.hsd_create(self._cfg_c, self._w_c)
         B.check(st, "hsd_create")
 

@@ -31,6 +31,26 @@ def test_tiny_config_matches_oracle(flags):
     print("tiny", flags, stats)
 
 
+@pytest.mark.parametrize("flags", [1, 0], ids=["simt", "tensor"])
+def test_qk_norm_decoder_matches_oracle(flags):
+    """Per-head RMSNorm of q and k before the rotary embedding (the Qwen3-style decoder variant): the Tiny shape and
+    a GQA shape with several q-tiles, through the fused QKV epilogue and through the plain kernels."""
+    import dataclasses
+    tiny = dataclasses.replace(I.TINY, qk_norm=True)
+    stats, _, _, _ = run_region_parity(I.tiny_workload(cfg=tiny), flags)
+    assert stats["max_dz"] < H.LOGIT_TOL
+    cfg = dataclasses.replace(I.small_decoder(2, 8192), qk_norm=True)
+    wl = I.region_workload(seed=78, n_regions=3, prefix_lo=70, prefix_hi=200, draft_mean=50, draft_lo=8, draft_hi=150,
+                           cfg=cfg, name="small_regions_qk_norm")
+    stats2, _, _, _ = run_region_parity(wl, flags)
+    assert stats2["max_dz"] < H.LOGIT_TOL
+    # the norm is really applied: the same weights without it give other logits
+    plain = run_region_parity(I.tiny_workload(), flags)[2]
+    with_norm = run_region_parity(I.tiny_workload(cfg=tiny), flags)[2]
+    assert np.max(np.abs(plain[0]["row_zmax"] - with_norm[0]["row_zmax"])) > 1e-2
+    print("qk_norm", flags, stats, stats2)
+
+
 @pytest.mark.parametrize("flags", [2, 0], ids=["simt_attention", "tensor"])
 def test_small_decoder_regions_match_oracle(flags):
     """Same layer shape as the 24-layer decoder (GQA 16/8, d 1024, FFN 4096), 2 layers, vocab 8192: several
