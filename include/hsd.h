@@ -204,8 +204,11 @@ HSD_API int hsd_verify_tree(hsd_ctx *ctx, const hsd_kv *kv, int n_seqs, const in
  *                   match is attempted then); the last entry is the pending token and must be a valid id
  *   emit_tokens, n_emit   dev int32 [n_seqs, emit_stride], [n_seqs] or both NULL: the tokens the previous step
  *                   emitted; they are appended to the window before matching (and the window is written back)
- *   draft_tokens    dev int32, all drafts concatenated;  draft_off dev int32 [n_drafts + 1] their offsets;
- *   seq_draft_off   dev int32 [n_seqs + 1]: sequence i owns drafts seq_draft_off[i] .. seq_draft_off[i+1] - 1
+ *   draft_tokens    dev int32 [total_draft_tokens], all drafts concatenated;  draft_off dev int32 [n_drafts + 1]
+ *                   their offsets;  seq_draft_off dev int32 [n_seqs + 1]: sequence i owns drafts
+ *                   seq_draft_off[i] .. seq_draft_off[i+1] - 1.  n_drafts and total_draft_tokens are host copies of
+ *                   the array sizes: the kernel clamps every offset it reads to them, so malformed offsets shorten
+ *                   or drop drafts but never read outside the arrays
  *   max_rows        rows every sequence gets in the packed output (<= HSD_MAX_TREE_ROWS; the paper packs 128)
  *   q_tokens, parent  dev int32 [n_seqs * max_rows] out: row 0 = the pending token (parent -1), then the tree's
  *                   nodes with their parent rows, then padding rows (the pending token again, parent -2) which
@@ -216,8 +219,9 @@ HSD_API int hsd_verify_tree(hsd_ctx *ctx, const hsd_kv *kv, int n_seqs, const in
  * node per distinct prefix, created level by level in candidate order while fewer than max_rows - 1 nodes exist; a
  * candidate whose next node cannot be created stops growing.  Pure integer work: results are exact. */
 HSD_API int hsd_dsv_build(hsd_ctx *ctx, int n_seqs, int window_n, int *window, const int *emit_tokens, const int *n_emit,
-                  int emit_stride, const int *draft_tokens, const int *draft_off, const int *seq_draft_off,
-                  int max_rows, int *q_tokens, int *parent, int *cu_q, int *n_rows, void *cuda_stream);
+                  int emit_stride, const int *draft_tokens, int total_draft_tokens, const int *draft_off,
+                  int n_drafts, const int *seq_draft_off, int max_rows, int *q_tokens, int *parent, int *cu_q,
+                  int *n_rows, void *cuda_stream);
 
 /* KV maintenance after hsd_verify_tree (Sec. 4.2 counts it in the decode loop): in every layer the K/V rows of the
  * accepted path move from cache rows L + accept_rows[i][d-1] to rows L + d (d = 1..accept_len[i]; L = committed

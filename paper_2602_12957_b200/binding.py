@@ -84,7 +84,7 @@ def _load():
     lib.hsd_verify_tree.argtypes = [vp, C.POINTER(hsd_kv), i, vp, vp, vp, vp, i, i, f, vp, vp, vp, vp, vp, vp, vp, vp, sz,
                                     vp]
     lib.hsd_kv_commit_tree.argtypes = [vp, C.POINTER(hsd_kv), i, vp, vp, vp, i, vp, vp]
-    lib.hsd_dsv_build.argtypes = [vp, i, i, vp, vp, vp, i, vp, vp, vp, i, vp, vp, vp, vp, vp]
+    lib.hsd_dsv_build.argtypes = [vp, i, i, vp, vp, vp, i, vp, i, vp, i, vp, i, vp, vp, vp, vp, vp]
     lib.hsd_verify_regions_host.argtypes = [vp, C.POINTER(hsd_kv), i, vp, vp, vp, f, i, vp, vp, vp, C.POINTER(C.c_int), vp, sz, vp]
     lib.hsd_device_status.argtypes = [vp, vp, vp, C.POINTER(C.c_int)]
     lib.hsd_last_cuda_error.argtypes = [vp]
@@ -226,11 +226,11 @@ def hsd_kv_commit_tree(ctx, kv, n_seqs, seq_slots, accept_len, accept_rows, max_
                                    _p(accept_rows), max_q_len, _p(blocks_in_use), _p(stream))
 
 
-def hsd_dsv_build(ctx, n_seqs, window_n, window, emit_tokens, n_emit, emit_stride, draft_tokens, draft_off, seq_draft_off,
-                  max_rows, q_tokens, parent, cu_q, n_rows, stream) -> int:
+def hsd_dsv_build(ctx, n_seqs, window_n, window, emit_tokens, n_emit, emit_stride, draft_tokens, total_draft_tokens,
+                  draft_off, n_drafts, seq_draft_off, max_rows, q_tokens, parent, cu_q, n_rows, stream) -> int:
     return _lib.hsd_dsv_build(ctx, n_seqs, window_n, _p(window), _p(emit_tokens), _p(n_emit), emit_stride,
-                              _p(draft_tokens), _p(draft_off), _p(seq_draft_off), max_rows, _p(q_tokens), _p(parent),
-                              _p(cu_q), _p(n_rows), _p(stream))
+                              _p(draft_tokens), total_draft_tokens, _p(draft_off), n_drafts, _p(seq_draft_off), max_rows,
+                              _p(q_tokens), _p(parent), _p(cu_q), _p(n_rows), _p(stream))
 
 
 def hsd_device_status(ctx, workspace, stream):

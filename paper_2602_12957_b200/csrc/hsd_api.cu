@@ -670,11 +670,13 @@ int hsd_verify_tree(hsd_ctx* c, const hsd_kv* kv, int n_seqs, const int* cu_q, c
 }
 
 int hsd_dsv_build(hsd_ctx* c, int n_seqs, int window_n, int* window, const int* emit_tokens, const int* n_emit,
-                  int emit_stride, const int* draft_tokens, const int* draft_off, const int* seq_draft_off, int max_rows,
-                  int* q_tokens, int* parent, int* cu_q, int* n_rows, void* cuda_stream) {
+                  int emit_stride, const int* draft_tokens, int total_draft_tokens, const int* draft_off, int n_drafts,
+                  const int* seq_draft_off, int max_rows, int* q_tokens, int* parent, int* cu_q, int* n_rows,
+                  void* cuda_stream) {
   if (!c || !window || !draft_tokens || !draft_off || !seq_draft_off || !q_tokens || !parent || !cu_q || !n_rows)
     return HSD_ERR_INVALID_ARG;
   if (n_seqs <= 0 || window_n <= 0 || window_n > HSD_MAX_WINDOW || max_rows <= 0) return HSD_ERR_INVALID_ARG;
+  if (total_draft_tokens < 0 || n_drafts < 0) return HSD_ERR_INVALID_ARG;
   if ((emit_tokens == nullptr) != (n_emit == nullptr) || (emit_tokens && emit_stride <= 0)) return HSD_ERR_INVALID_ARG;
   if (max_rows > HSD_MAX_TREE_ROWS) return HSD_ERR_TOO_LONG;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -683,6 +685,7 @@ int hsd_dsv_build(hsd_ctx* c, int n_seqs, int window_n, int* window, const int* 
   a.n_seqs = n_seqs; a.window_n = window_n; a.max_rows = max_rows; a.emit_stride = emit_stride;
   a.window = window; a.emit_tokens = emit_tokens; a.n_emit = n_emit;
   a.draft_tokens = draft_tokens; a.draft_off = draft_off; a.seq_draft_off = seq_draft_off;
+  a.total_draft_tokens = total_draft_tokens; a.n_drafts = n_drafts;
   a.q_tokens = q_tokens; a.parent = parent; a.cu_q = cu_q; a.n_rows = n_rows;
   launch_dsv_build(st, a, c->pdl);
   return check_cuda(c);

@@ -113,7 +113,7 @@ void launch_tree_compact(cudaStream_t st, const KvView& kv, int n_layers, int n_
                          const int* accept_len, const int* accept_rows, int max_q_len, bool pdl);
 // Draft-target matching + prefix-tree packing on the device (Eq. 5-7)
 struct DsvArgs {
-  int n_seqs, window_n, max_rows, emit_stride;
+  int n_seqs, window_n, max_rows, emit_stride, total_draft_tokens, n_drafts;
   int* window;               // [S, n] inout
   const int* emit_tokens;    // [S, emit_stride] or nullptr
   const int* n_emit;         // [S] or nullptr

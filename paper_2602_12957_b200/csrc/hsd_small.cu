@@ -617,8 +617,11 @@ __global__ void dsv_build_kernel(DsvArgs a) {
   for (int i = 0; i < n; ++i) have_w = have_w && s_w[i] >= 0;
   // ---- candidates
   if (have_w) {
-    for (int d = a.seq_draft_off[s]; d < a.seq_draft_off[s + 1]; ++d) {
-      const int d0 = a.draft_off[d], len = a.draft_off[d + 1] - d0;
+    // every offset is clamped to the array sizes the host passed: a malformed table shortens or drops drafts
+    const int d_lo = min(max(a.seq_draft_off[s], 0), a.n_drafts), d_hi = min(max(a.seq_draft_off[s + 1], 0), a.n_drafts);
+    for (int d = d_lo; d < d_hi; ++d) {
+      const int d0 = min(max(a.draft_off[d], 0), a.total_draft_tokens);
+      const int len = min(max(a.draft_off[d + 1], d0), a.total_draft_tokens) - d0;
       for (int j0 = 0; j0 + n < len; j0 += blockDim.x) {      // j + n < len: a non-empty suffix follows the window
         if (s_ncand >= kDsvMaxCands) break;
         const int j = j0 + tid;

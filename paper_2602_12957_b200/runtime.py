@@ -165,8 +165,9 @@ class Engine:
             i32 = lambda *s: torch.empty(*s, dtype=torch.int32, device=self.dev)
             out = {"q_tokens": i32(S * max_rows), "parent": i32(S * max_rows), "cu_q": i32(S + 1), "n_rows": i32(S)}
         st = B.hsd_dsv_build(self.model.ctx, S, n, window, emit_tokens, n_emit,
-                             int(emit_tokens.shape[1]) if emit_tokens is not None else 0, draft_tokens, draft_off,
-                             seq_draft_off, max_rows, out["q_tokens"], out["parent"], out["cu_q"], out["n_rows"], _stream())
+                             int(emit_tokens.shape[1]) if emit_tokens is not None else 0, draft_tokens,
+                             int(draft_tokens.numel()), draft_off, int(draft_off.numel()) - 1, seq_draft_off, max_rows,
+                             out["q_tokens"], out["parent"], out["cu_q"], out["n_rows"], _stream())
         B.check(st, "hsd_dsv_build")
         return out
 

@@ -83,7 +83,7 @@ def test_host_side_argument_checks_need_no_device(B):
     assert B.hsd_verify_tree(None, None, 1, None, None, None, None, 1, 1, 0.0, None, None, None, None, None, None, None,
                              None, 0, None) == B.HSD_ERR_INVALID_ARG
     assert B.hsd_kv_commit_tree(None, None, 1, None, None, None, 1, None, None) == B.HSD_ERR_INVALID_ARG
-    assert B.hsd_dsv_build(None, 1, 3, None, None, None, 0, None, None, None, 128, None, None, None, None,
+    assert B.hsd_dsv_build(None, 1, 3, None, None, None, 0, None, 0, None, 0, None, 128, None, None, None, None,
                            None) == B.HSD_ERR_INVALID_ARG
 
 

@@ -98,6 +98,22 @@ def test_build_edge_cases():
     check_build(eng, [[1, 2], [1, 2], [3, 4]], [[], [[1, 2, 3, 4, 5]], [[3, 4]]], 16)
 
 
+def test_malformed_draft_offsets_are_clamped_not_followed():
+    """Offsets that point outside the draft arrays shorten or drop drafts (as if the arrays ended there); the call
+    stays inside the arrays and its outputs are well-formed trees."""
+    import torch
+    eng, _, _ = _engine()
+    toks = eng._i32([1, 2, 3, 4, 5, 1, 2, 3, 9, 9])
+    window = eng._i32(np.asarray([[1, 2, 3]], np.int32)).reshape(1, 3)
+    for off, soff in (([0, 5, 1 << 30], [0, 2]), ([-7, 5, 10], [0, 2]), ([0, 5, 10], [0, 1 << 20]),
+                      ([8, 3, 10], [0, 2]), ([0, 5, 10], [-3, 2])):
+        out = eng.dsv_build(window, toks, eng._i32(off), eng._i32(soff), 16)
+        torch.cuda.synchronize()
+        n = int(out["n_rows"][0])
+        par = out["parent"].cpu().numpy()[:16]
+        assert 1 <= n <= 16 and par[0] == -1 and all(0 <= par[r] < r for r in range(1, n)) and all(par[n:] == -2)
+
+
 def test_device_driven_loop_follows_the_oracle_driven_loop():
     """Three decode steps per sequence with no host decision in between on the device side: hsd_dsv_build (fed by the
     previous step's emitted tokens) -> hsd_verify_tree -> hsd_kv_commit_tree.  The oracle side makes the same steps
