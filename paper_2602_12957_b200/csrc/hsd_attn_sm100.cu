@@ -212,7 +212,17 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   // Round r of the walk: CTA i takes item r G + i in even rounds and r G + (G - 1 - i) in odd ones (the list is
   // sorted longest first, so the CTA that drew a long item in one round draws a short one in the next).
   const int n_rounds = (total + (int)gridDim.x - 1) / (int)gridDim.x;
+  // A launch with fewer items than CTAs leaves some SMs with one busy CTA (the grid is two CTAs per SM, and CTA b
+  // shares its SM with CTA b + G/2 under the usual placement); a CTA that has its SM alone walks its tiles faster,
+  // so the longest items go to those SMs and the others pair a long item with a short one.
+  const int half_grid = (int)gridDim.x / 2;
   auto item_of_round = [&](int r) -> int {
+    if (n_rounds == 1 && total > half_grid) {
+      const int n_second = total - half_grid;          // busy CTAs in the second half of the grid
+      const int bx = (int)blockIdx.x;
+      if (bx < half_grid) return bx >= n_second ? bx - n_second : (half_grid - n_second) + bx;
+      return bx - half_grid < n_second ? total - 1 - (bx - half_grid) : -1;
+    }
     const int i = (r & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x;
     const int w = r * (int)gridDim.x + i;
     return w < total ? w : -1;
