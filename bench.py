@@ -414,6 +414,13 @@ def run_ours(args):
     roof["peak_source"] = (f"{peak_src} (sustained bf16 figure: kernel timed inside a long step)" if roof["bound"] == "tensor"
                            else f"{peak_src} (STREAM-style copy bandwidth)")
     roof["us_per_launch"] = dur * 1e6
+    # the same fraction for every kernel class with a work model (the `roofline` object above is the top one)
+    for k, (fl, nb) in table.items():
+        if k in prof and prof[k][1] > 0:
+            d_k = prof[k][0] * 1e-3 / prof[k][1]
+            tensor_k = fl / pk >= nb / bw
+            kernels[k]["bound"] = "tensor" if tensor_k else "hbm"
+            kernels[k]["roofline_frac"] = (fl / d_k / pk) if tensor_k else (nb / d_k / bw)
     t_roof = RF.roofline_time(work.bytes, work.flops, bw, pk)
     step_roof = {"roofline_us": t_roof * 1e6, "frac": t_roof / (ms_step * 1e-3), "bytes": work.bytes, "flops": work.flops,
                  "bound": "tensor" if work.flops / pk > work.bytes / bw else "hbm"}
