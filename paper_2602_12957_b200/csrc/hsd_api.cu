@@ -260,7 +260,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
   if (!c->attn_simt) {
     Scope s(c, st, KC_SETUP);
     // items per launch: a few per CTA slot (two CTAs per SM), at least attn_min_chunk KV tiles each
-    launch_attn_plan(st, w.rm, w.plan, a.n_seqs, tokens_per_tile, c->attn_target_items / md.Hkv + 1, c->attn_min_chunk,
+    launch_attn_plan(st, w.rm, w.plan, a.n_seqs, tokens_per_tile, max(1, c->attn_target_items / md.Hkv), c->attn_min_chunk,
                      w.status + 4, w.status, c->pdl);
   }
   if (!c->simt) {
@@ -534,7 +534,7 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
   c->hg_exec = nullptr;
   c->hg_launches = 0;
   c->attn_target_items = 2 * c->n_sms;   // one item per CTA slot: slicing costs a partial hand-over per slice
-  c->attn_min_chunk = 16;
+  c->attn_min_chunk = 8;
   c->last_cuda_error = 0;
   c->launches = 0;
   c->profiling = false;
@@ -1026,7 +1026,7 @@ int hsd_debug_set_gemm_tile(hsd_ctx* c, int tile_n, int k_slices) {
 int hsd_debug_set_attn_plan(hsd_ctx* c, int target_items, int min_kv_tiles) {
   if (!c || target_items < 0 || min_kv_tiles < 0) return HSD_ERR_INVALID_ARG;
   c->attn_target_items = target_items ? target_items : 2 * c->n_sms;
-  c->attn_min_chunk = min_kv_tiles ? min_kv_tiles : 16;
+  c->attn_min_chunk = min_kv_tiles ? min_kv_tiles : 8;
   return HSD_OK;
 }
 
