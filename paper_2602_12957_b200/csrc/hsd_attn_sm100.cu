@@ -91,23 +91,30 @@ __global__ void attn_plan_kernel(RowMeta rm, AttnPlan pl, int n_seqs, int tokens
   }
   atomicAdd(&s_total, my);
   __syncthreads();
-  __shared__ int s_n;
-  if (threadIdx.x == 0) {
-    // KV tiles per slice: start from an even share.  Rounding up the slice count of every q-tile can leave the
-    // launch with somewhat more items than CTA slots, and then the few CTAs that draw a second item double its
-    // length: in that band (1 to 1.6 items per slot) the share is grown until every slot has at most one item.
-    // Well beyond it a second round is about full and the sorted walk balances it, so the share is kept.
-    int chunk = max(min_chunk, (s_total + target_items - 1) / max(1, target_items));
-    for (int it = 0; it < 256; ++it) {
-      int count = 0, longest = 0;
-      for (int t = 0; t < n_tiles; ++t) {
-        const int n_kv = pl.tile_nkv[t];
-        count += max(1, min(kAttnMaxSplits, (n_kv + chunk - 1) / chunk));
-        longest = max(longest, n_kv);
-      }
-      if (count <= target_items || 5 * count >= 8 * target_items || chunk >= longest) break;
-      chunk += max(1, chunk >> 4);
+  // KV tiles per slice: start from an even share.  Rounding up the slice count of every q-tile can leave the
+  // launch with somewhat more items than CTA slots, and then the few CTAs that draw a second item double its
+  // length: in that band (1 to 1.6 items per slot) the share is grown until every slot has at most one item.
+  // Well beyond it a second round is about full and the sorted walk balances it, so the share is kept.
+  __shared__ int s_n, s_count, s_longest;
+  int chunk = max(min_chunk, (s_total + target_items - 1) / max(1, target_items));
+  for (int it = 0; it < 256; ++it) {                      // every thread runs the same iterations
+    if (threadIdx.x == 0) { s_count = 0; s_longest = 0; }
+    __syncthreads();
+    int count = 0, longest = 0;
+    for (int t = threadIdx.x; t < n_tiles; t += blockDim.x) {
+      const int n_kv = pl.tile_nkv[t];
+      count += max(1, min(kAttnMaxSplits, (n_kv + chunk - 1) / chunk));
+      longest = max(longest, n_kv);
     }
+    atomicAdd(&s_count, count);
+    atomicMax(&s_longest, longest);
+    __syncthreads();
+    const bool done = s_count <= target_items || 5 * s_count >= 8 * target_items || chunk >= s_longest;
+    __syncthreads();
+    if (done) break;
+    chunk += max(1, chunk >> 4);
+  }
+  if (threadIdx.x == 0) {
     int n = 0;
     for (int t = 0; t < n_tiles; ++t) {   // serial: a few hundred tiles at most, once per step
       const int n_kv = pl.tile_nkv[t];
