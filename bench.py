@@ -417,7 +417,8 @@ def run_ours(args):
     # the same fraction for every kernel class with a work model (the `roofline` object above is the top one)
     for k, (fl, nb) in table.items():
         if k in prof and prof[k][1] > 0:
-            d_k = prof[k][0] * 1e-3 / prof[k][1]
+            # the LM-head class has one GEMM per step beside a small clearing kernel: its work model is per step
+            d_k = prof[k][0] * 1e-3 / (prof_steps if k == "lm_head_argmax" else prof[k][1])
             tensor_k = fl / pk >= nb / bw
             kernels[k]["bound"] = "tensor" if tensor_k else "hbm"
             kernels[k]["roofline_frac"] = (fl / d_k / pk) if tensor_k else (nb / d_k / bw)
