@@ -140,6 +140,9 @@ def make_workload(args, rank):
         return wl
     args.random_drafts = True
     if name == "mixed":
+        k = getattr(args, "mixed_k", 0)
+        if k:       # the sweep over a fixed draft length: the 64 regions alone
+            return I.mixed_workload(seed=I.BASE_SEED + 4 + 1000 * rank, fixed_draft_len=k, with_page_chunks=False, cfg=cfg)
         return I.mixed_workload(seed=I.BASE_SEED + 4 + 1000 * rank, cfg=cfg)
     ctx, k = {"page": (6400, 512), "long1024": (10240, 1024), "long2048": (10240, 2048)}[name]
     rng = np.random.Generator(np.random.PCG64(I.BASE_SEED + 2 + 1000 * rank))
@@ -434,7 +437,8 @@ def run_ours(args):
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": WORKLOADS[args.workload],
+                "config": {"workload": WORKLOADS[args.workload] + (f" [64 regions only, every draft {args.mixed_k} tokens]"
+                                                                   if args.workload == "mixed" and args.mixed_k else ""),
                            "regions_per_gpu": S, "query_rows_per_gpu": T, "draft_tokens_per_gpu": draft_tokens,
                            "context_tokens_per_gpu": int(sum(ctx_lens)), "mean_acceptance_rate": accept_mean,
                            "planted_acceptance_rate": float(np.mean([s.agree_len / s.draft_len for s in st["wl"].seqs])),
@@ -508,6 +512,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", default="region", choices=sorted(WORKLOADS),
                     help="region = the benchmark line; the others time one step of the other configurations")
+    ap.add_argument("--mixed-k", type=int, default=0,
+                    help="with --workload mixed: the 64 regions alone, every draft this many tokens long (the k sweep)")
     ap.add_argument("--flags", type=int, default=0, help="HSD_FLAG_* bits for the context (debugging / ablations)")
     ap.add_argument("--random-drafts", action="store_true",
                     help="skip the greedy-continuation pass that plants agreement (for profiler captures)")
