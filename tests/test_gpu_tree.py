@@ -189,6 +189,16 @@ def test_small_decoder_trees_match_oracle(log_tau):
     print("small trees", log_tau, stats)
 
 
+def test_many_short_trees_in_one_call():
+    """Forty sequences with trees of 0 to 59 nodes in one call (more sequences than any grid dimension the other cases
+    reach), then the compacting commit and a chain step on top."""
+    wl = I.tiny_workload(n_regions=40, draft_len=30, prefix_len=96, n_visual=32)
+    rng = np.random.default_rng(1)
+    nodes = [int(x) for x in rng.integers(0, 60, size=40)]
+    stats, _, _ = run_tree_case(wl, nodes, LOG_TAU_PAPER)
+    assert stats["exact"] + stats["tolerated"] == 40 and stats["max_dz"] < H.LOGIT_TOL
+
+
 def test_a_chain_given_as_a_tree_equals_the_chain_call():
     """parent[j] = j - 1 is the linear draft: same integers as hsd_verify_regions, same logits."""
     from paper_2602_12957_b200 import binding as B
