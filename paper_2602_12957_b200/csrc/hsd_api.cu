@@ -13,6 +13,7 @@ using namespace hsd;
 struct ProfEvent {
   int kc;
   cudaEvent_t a, b;
+  bool own_a;      // false: `a` is the end event of the launch before (consecutive launches share one event)
 };
 
 // Everything a call of hsd_verify_regions_host bakes into its launches, by value: two calls with equal keys enqueue
@@ -48,6 +49,8 @@ struct hsd_ctx {
   int last_cuda_error;
   long long launches;
   bool profiling;
+  cudaEvent_t prof_last;          // end event of the last profiled launch of the current call, or nullptr
+  cudaStream_t prof_last_stream;
   // hsd_verify_regions_host: pinned staging and the cached graph of the last repeated call shape
   bool host_graph_ok;
   int* pin;
@@ -152,28 +155,41 @@ struct Scope {   // brackets one launch: counts it and, when profiling, records 
   hsd_ctx* c;
   cudaStream_t st;
   int idx;
+  // Consecutive launches of one call share an event (the end of one is the start of the next), so a profiled
+  // step carries one event record per launch boundary, not two.
   Scope(hsd_ctx* c_, cudaStream_t st_, int kc) : c(c_), st(st_), idx(-1) {
     c->launches++;
     if (!c->profiling) return;
+    auto take = [&](cudaEvent_t* ev) -> bool {
+      if (!c->event_pool.empty()) {
+        *ev = c->event_pool.back();
+        c->event_pool.pop_back();
+        return true;
+      }
+      return cudaEventCreate(ev) == cudaSuccess;
+    };
     ProfEvent e;
     e.kc = kc;
-    cudaEvent_t ev[2];
-    for (int i = 0; i < 2; ++i) {
-      if (!c->event_pool.empty()) {
-        ev[i] = c->event_pool.back();
-        c->event_pool.pop_back();
-      } else if (cudaEventCreate(&ev[i]) != cudaSuccess) {
-        return;
-      }
+    e.own_a = !(c->prof_last && c->prof_last_stream == st);
+    if (e.own_a) {
+      if (!take(&e.a)) return;
+      cudaEventRecord(e.a, st);
+    } else {
+      e.a = c->prof_last;
     }
-    e.a = ev[0];
-    e.b = ev[1];
-    cudaEventRecord(e.a, st);
+    if (!take(&e.b)) {
+      if (e.own_a) c->event_pool.push_back(e.a);
+      return;
+    }
     c->prof_events.push_back(e);
     idx = (int)c->prof_events.size() - 1;
   }
   ~Scope() {
-    if (idx >= 0) cudaEventRecord(c->prof_events[idx].b, st);
+    if (idx >= 0) {
+      cudaEventRecord(c->prof_events[idx].b, st);
+      c->prof_last = c->prof_events[idx].b;
+      c->prof_last_stream = st;
+    }
   }
 };
 
@@ -230,6 +246,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
   const int T = a.total_q;
   const int tokens_per_tile = 128 / md.group;
 
+  c->prof_last = nullptr;      // profiling: what ran between two calls is the caller's, not the first kernel's
   if (cudaMemsetAsync(w.status, 0, 64, st) != cudaSuccess) return check_cuda(c);
   {
     Scope s(c, st, KC_SETUP);
@@ -533,6 +550,8 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
   c->hg_seen_valid = false;
   c->hg_exec = nullptr;
   c->hg_launches = 0;
+  c->prof_last = nullptr;
+  c->prof_last_stream = nullptr;
   c->attn_target_items = 2 * c->n_sms;   // one item per CTA slot: slicing costs a partial hand-over per slice
   c->attn_min_chunk = 8;
   c->last_cuda_error = 0;
@@ -560,7 +579,7 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
 
 int hsd_destroy(hsd_ctx* c) {
   if (!c) return HSD_ERR_INVALID_ARG;
-  for (auto& e : c->prof_events) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
+  for (auto& e : c->prof_events) { if (e.own_a) cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
   for (auto& e : c->event_pool) cudaEventDestroy(e);
   if (c->hg_exec) cudaGraphExecDestroy(c->hg_exec);
   if (c->pin) cudaFreeHost(c->pin);
@@ -890,8 +909,9 @@ long long hsd_launch_count(const hsd_ctx* c) { return c ? c->launches : 0; }
 
 int hsd_profile_enable(hsd_ctx* c, int enable) {
   if (!c) return HSD_ERR_INVALID_ARG;
-  for (auto& e : c->prof_events) { c->event_pool.push_back(e.a); c->event_pool.push_back(e.b); }
+  for (auto& e : c->prof_events) { if (e.own_a) c->event_pool.push_back(e.a); c->event_pool.push_back(e.b); }
   c->prof_events.clear();
+  c->prof_last = nullptr;
   memset(c->prof_ms, 0, sizeof(c->prof_ms));
   memset(c->prof_n, 0, sizeof(c->prof_n));
   c->profiling = enable != 0;
@@ -906,10 +926,13 @@ int hsd_profile_read(hsd_ctx* c, int cap, const char** names, double* total_ms, 
       return fail_cuda(c);
     c->prof_ms[e.kc] += ms;
     c->prof_n[e.kc] += 1;
-    c->event_pool.push_back(e.a);
+  }
+  for (auto& e : c->prof_events) {      // recycle only after every interval has been read (events are shared)
+    if (e.own_a) c->event_pool.push_back(e.a);
     c->event_pool.push_back(e.b);
   }
   c->prof_events.clear();
+  c->prof_last = nullptr;
   int n = 0;
   for (int k = 0; k < KC_COUNT; ++k) {
     if (!c->prof_n[k]) continue;
