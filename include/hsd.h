@@ -101,7 +101,10 @@ typedef struct {
   const void *const *q_norm, *const *k_norm;   /* bf16 [head_dim] per layer; read only when qk_norm = 1, else may be NULL */
 } hsd_weights;
 
-/* Caller-owned paged KV cache.  All pointers are device pointers. */
+/* Caller-owned paged KV cache.  All pointers are device pointers.
+ * k_pool and v_pool must hold FINITE values everywhere before the first call (zero them once at allocation): a key the
+ * mask hides still enters the second attention product as 0 * v, which is 0 only for finite v, so an Inf or NaN bit
+ * pattern left in a row that was never written would turn that tile's outputs into NaN. */
 typedef struct {
   void *k_pool, *v_pool;
   int n_blocks;               /* physical blocks per layer                                            */
@@ -288,6 +291,28 @@ HSD_API int hsd_debug_logits(hsd_ctx *ctx, const void *workspace, int total_q, i
  * "q" bf16 [T,n_heads*head_dim], "attn" bf16 [T,n_heads*head_dim], "act" bf16 [T,d_ffn] of the last layer. */
 HSD_API int hsd_debug_buffer(hsd_ctx *ctx, const void *workspace, int total_q, int n_seqs, const char *name,
                      void **ptr, size_t *bytes);
+
+/* Test-only: arm a tap on an intermediate tensor of ONE decoder layer (Eq. 8 is a stack of such layers; the tap lets a
+ * parity miss be traced to the layer where it starts).  The NEXT forward this context runs (hsd_prefill, hsd_verify_*)
+ * copies, device to device on that call's stream and right after the kernel that produced it, the tensor `which` of
+ * layer `layer` (0-based) into dst, then the tap disarms.  T = that call's packed rows.
+ *   HSD_TAP_X       fp32 [T, d_model]            residual stream after the layer
+ *   HSD_TAP_X_MID   fp32 [T, d_model]            residual stream after the layer's attention block
+ *   HSD_TAP_H_ATTN  bf16 [T, d_model]            RMSNorm output that feeds the QKV projection
+ *   HSD_TAP_H_FFN   bf16 [T, d_model]            RMSNorm output that feeds the gate/up projection
+ *   HSD_TAP_Q       bf16 [T, n_heads*head_dim]   rotated queries
+ *   HSD_TAP_ATTN    bf16 [T, n_heads*head_dim]   attention output
+ *   HSD_TAP_ACT     bf16 [T, d_ffn]              SwiGLU activation
+ *   dst             dev, dst_bytes bytes, caller-owned; a tensor larger than dst_bytes makes that forward return
+ *                   HSD_ERR_WORKSPACE.  layer < 0 disarms.  Errors: INVALID_ARG (layer or which out of range, dst NULL). */
+#define HSD_TAP_X 0
+#define HSD_TAP_H_ATTN 1
+#define HSD_TAP_H_FFN 2
+#define HSD_TAP_Q 3
+#define HSD_TAP_ATTN 4
+#define HSD_TAP_ACT 5
+#define HSD_TAP_X_MID 6
+HSD_API int hsd_debug_tap(hsd_ctx *ctx, int layer, int which, void *dst, size_t dst_bytes);
 
 /* Test/bench-only single operators, asynchronous on the stream.
  * hsd_op_linear: C = A W^T with the epilogue `mode`:

@@ -65,9 +65,10 @@ def rope(x: np.ndarray, pos: np.ndarray, base: float) -> np.ndarray:
 
 
 def softmax_rows(s: np.ndarray) -> np.ndarray:
-    m = np.max(s, axis=-1, keepdims=True)
-    e = np.exp(s - m)
-    return e / np.sum(e, axis=-1, keepdims=True)
+    e = s - np.max(s, axis=-1, keepdims=True)
+    np.exp(e, out=e)
+    e /= np.sum(e, axis=-1, keepdims=True)
+    return e
 
 
 def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, allowed: np.ndarray) -> np.ndarray:
@@ -81,7 +82,9 @@ def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, allowed: np.ndarray) 
     scale = 1.0 / math.sqrt(D)
     for g in range(Hq):
         kh = g // group
-        s = (q[:, g, :] @ k[:, kh, :].T) * scale + neg
+        s = q[:, g, :] @ k[:, kh, :].T
+        s *= scale          # in place: the score matrix of a long context is large
+        s += neg
         out[:, g, :] = softmax_rows(s) @ v[:, kh, :]
     return out
 

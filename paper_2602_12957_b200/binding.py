@@ -34,8 +34,9 @@ EXPORTS = [
     "hsd_verify_page", "hsd_kv_commit", "hsd_verify_regions_host", "hsd_device_status", "hsd_last_cuda_error", "hsd_launch_count",
     "hsd_profile_enable", "hsd_profile_read", "hsd_debug_logits", "hsd_debug_buffer", "hsd_op_linear",
     "hsd_op_lm_head_argmax", "hsd_op_lm_head_argmax_noalloc", "hsd_debug_set_gemm_tile", "hsd_debug_set_attn_plan",
-    "hsd_verify_tree", "hsd_kv_commit_tree", "hsd_dsv_build",
+    "hsd_verify_tree", "hsd_kv_commit_tree", "hsd_dsv_build", "hsd_debug_tap",
 ]
+HSD_TAP_X, HSD_TAP_H_ATTN, HSD_TAP_H_FFN, HSD_TAP_Q, HSD_TAP_ATTN, HSD_TAP_ACT, HSD_TAP_X_MID = range(7)
 
 
 class HsdError(RuntimeError):
@@ -94,6 +95,7 @@ def _load():
     lib.hsd_profile_read.argtypes = [vp, i, C.POINTER(C.c_char_p), C.POINTER(C.c_double), C.POINTER(C.c_longlong)]
     lib.hsd_debug_logits.argtypes = [vp, vp, i, i, vp, vp]
     lib.hsd_debug_buffer.argtypes = [vp, vp, i, i, C.c_char_p, C.POINTER(vp), C.POINTER(sz)]
+    lib.hsd_debug_tap.argtypes = [vp, i, i, vp, sz]
     lib.hsd_debug_set_gemm_tile.argtypes = [vp, i, i]
     lib.hsd_debug_set_attn_plan.argtypes = [vp, i, i]
     lib.hsd_op_linear.argtypes = [vp, vp, vp, vp, i, i, i, i, vp]
@@ -274,6 +276,11 @@ def hsd_debug_buffer(ctx, workspace, total_q, n_seqs, name: str):
     ptr, sz = C.c_void_p(), C.c_size_t()
     st = _lib.hsd_debug_buffer(ctx, _p(workspace), total_q, n_seqs, name.encode(), C.byref(ptr), C.byref(sz))
     return st, ptr.value, sz.value
+
+
+def hsd_debug_tap(ctx, layer: int, which: int, dst, dst_bytes: int) -> int:
+    """Arms a tap: the next forward copies intermediate `which` (HSD_TAP_*) of decoder layer `layer` into dst."""
+    return _lib.hsd_debug_tap(ctx, layer, which, _p(dst), dst_bytes)
 
 
 def hsd_debug_set_gemm_tile(ctx, tile_n: int, k_slices: int) -> int:

@@ -12,8 +12,7 @@ using namespace hsd;
 
 struct ProfEvent {
   int kc;
-  cudaEvent_t a, b;
-  bool own_a;      // false: `a` is the end event of the launch before (consecutive launches share one event)
+  cudaEvent_t a, b;   // recorded right before and right after the launch: every interval owns both its ends
 };
 
 // Everything a call of hsd_verify_regions_host bakes into its launches, by value: two calls with equal keys enqueue
@@ -42,6 +41,9 @@ struct hsd_ctx {
   int force_bn, force_splits;   // hsd_debug_set_gemm_tile
   int pair;                     // GEMMs may run as CTA pairs
   int attn_target_items, attn_min_chunk;   // attention plan: items aimed at per launch, fewest KV tiles per slice
+  int tap_layer, tap_which;                // hsd_debug_tap: armed for the next forward (tap_layer < 0: none)
+  void* tap_dst;
+  size_t tap_bytes;
   int n_sms;
   int device;
   bool simt;
@@ -49,8 +51,6 @@ struct hsd_ctx {
   int last_cuda_error;
   long long launches;
   bool profiling;
-  cudaEvent_t prof_last;          // end event of the last profiled launch of the current call, or nullptr
-  cudaStream_t prof_last_stream;
   // hsd_verify_regions_host: pinned staging and the cached graph of the last repeated call shape
   bool host_graph_ok;
   int* pin;
@@ -155,8 +155,9 @@ struct Scope {   // brackets one launch: counts it and, when profiling, records 
   hsd_ctx* c;
   cudaStream_t st;
   int idx;
-  // Consecutive launches of one call share an event (the end of one is the start of the next), so a profiled
-  // step carries one event record per launch boundary, not two.
+  // Two event records per launch.  An event between two kernels also keeps them from overlapping through
+  // programmatic dependent launch, so a profiled interval is the kernel alone (as a serialising profiler sees it),
+  // not its share of an overlapped step.
   Scope(hsd_ctx* c_, cudaStream_t st_, int kc) : c(c_), st(st_), idx(-1) {
     c->launches++;
     if (!c->profiling) return;
@@ -170,26 +171,17 @@ struct Scope {   // brackets one launch: counts it and, when profiling, records 
     };
     ProfEvent e;
     e.kc = kc;
-    e.own_a = !(c->prof_last && c->prof_last_stream == st);
-    if (e.own_a) {
-      if (!take(&e.a)) return;
-      cudaEventRecord(e.a, st);
-    } else {
-      e.a = c->prof_last;
-    }
+    if (!take(&e.a)) return;
     if (!take(&e.b)) {
-      if (e.own_a) c->event_pool.push_back(e.a);
+      c->event_pool.push_back(e.a);
       return;
     }
+    cudaEventRecord(e.a, st);
     c->prof_events.push_back(e);
     idx = (int)c->prof_events.size() - 1;
   }
   ~Scope() {
-    if (idx >= 0) {
-      cudaEventRecord(c->prof_events[idx].b, st);
-      c->prof_last = c->prof_events[idx].b;
-      c->prof_last_stream = st;
-    }
+    if (idx >= 0) cudaEventRecord(c->prof_events[idx].b, st);
   }
 };
 
@@ -246,8 +238,16 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
   const int T = a.total_q;
   const int tokens_per_tile = 128 / md.group;
 
-  c->prof_last = nullptr;      // profiling: what ran between two calls is the caller's, not the first kernel's
   if (cudaMemsetAsync(w.status, 0, 64, st) != cudaSuccess) return check_cuda(c);
+  // hsd_debug_tap: one armed tap is served by this forward, then disarmed
+  const int tap_layer = c->tap_layer, tap_which = c->tap_which;
+  c->tap_layer = -1;
+  auto tap = [&](int layer, int which, const void* src, size_t bytes) -> int {
+    if (layer != tap_layer || which != tap_which) return HSD_OK;
+    if (bytes > c->tap_bytes) return HSD_ERR_WORKSPACE;
+    return cudaMemcpyAsync(c->tap_dst, src, bytes, cudaMemcpyDeviceToDevice, st) == cudaSuccess ? HSD_OK : fail_cuda(c);
+  };
+  const size_t row_d = (size_t)T * md.d, row_q = (size_t)T * md.Hq * md.D;
   {
     Scope s(c, st, KC_SETUP);
     SetupArgs sa;
@@ -300,8 +300,9 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
   for (int l = 0; l < md.n_layers; ++l) {
     {
       Scope s(c, st, KC_RMSNORM);
-      launch_rmsnorm(st, w.x, c->attn_norm[l], w.h, T, md.d, md.eps, nullptr, c->pdl);
+      launch_rmsnorm(st, w.x, c->attn_norm[l], w.h, T, md.d, md.eps, nullptr, T, w.status, c->pdl);
     }
+    if (int rc = tap(l, HSD_TAP_H_ATTN, w.h, 2 * row_d)) return rc;
     const size_t layer_elems = (size_t)kv.n_blocks * md.Hkv * 64 * 64;
     if (c->simt) {
       {
@@ -331,13 +332,14 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         g.tmC = tm_q_st;
         g.M = T; g.n_out = md.qkv_out; g.K = md.d; g.mode = GS_QKV_ROPE;
         g.qkv.row_kv = w.rm.row_kv;
+        g.qkv.kv_rows = kv.n_blocks * HSD_KV_BLOCK;
         g.qkv.rope_cs = w.rm.rope_cs;
         g.qkv.q_out = w.q;
         g.qkv.k_pool_layer = kv.k_pool + (size_t)l * layer_elems;
         g.qkv.v_pool_layer = kv.v_pool + (size_t)l * layer_elems;
         g.qkv.Hq = md.Hq; g.qkv.Hkv = md.Hkv;
         g.qkv.q_norm = c->q_norm[l]; g.qkv.k_norm = c->k_norm[l]; g.qkv.eps = md.eps;
-        g.status = w.status; g.n_sms = c->n_sms; g.max_splits = 1; g.pdl = c->pdl; g.pair = c->pair;
+        g.status = w.status; g.n_sms = c->n_sms; g.device = c->device; g.max_splits = 1; g.pdl = c->pdl; g.pair = c->pair;
         g.force_bn = c->force_bn;
         if (launch_gemm_sm100(st, g)) return fail_cuda(c);
       }
@@ -345,7 +347,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         Scope s(c, st, KC_ATTN);
         if (c->attn_simt) {
           launch_attn_simt(st, w.q, w.rm, kv, md, l, w.attn, T, w.status);
-        } else if (launch_attn_sm100(st, tm_q, tm_k, tm_v, w.plan, kv, md, l, w.attn, c->n_sms, w.status, w.split_ws,
+        } else if (launch_attn_sm100(st, tm_q, tm_k, tm_v, w.plan, kv, md, l, w.attn, c->n_sms, c->device, w.status, w.split_ws,
                                      a.parent ? w.rm.anc : nullptr, c->pdl)) {
           return fail_cuda(c);
         }
@@ -357,14 +359,18 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         g.tmB = &c->tm_o[l];
         g.tmC = tm_x_add;
         g.M = T; g.n_out = md.d; g.K = md.Hq * md.D; g.mode = GS_ADD_F32;
-        g.status = w.status; g.n_sms = c->n_sms; g.max_splits = c->max_splits; g.pdl = c->pdl; g.pair = c->pair;
+        g.status = w.status; g.n_sms = c->n_sms; g.device = c->device; g.max_splits = c->max_splits; g.pdl = c->pdl; g.pair = c->pair;
         if (launch_gemm_sm100(st, g)) return fail_cuda(c);
       }
     }
+    if (int rc = tap(l, HSD_TAP_Q, w.q, 2 * row_q)) return rc;
+    if (int rc = tap(l, HSD_TAP_ATTN, w.attn, 2 * row_q)) return rc;
+    if (int rc = tap(l, HSD_TAP_X_MID, w.x, 4 * row_d)) return rc;
     {
       Scope s(c, st, KC_RMSNORM);
-      launch_rmsnorm(st, w.x, c->ffn_norm[l], w.h, T, md.d, md.eps, nullptr, c->pdl);
+      launch_rmsnorm(st, w.x, c->ffn_norm[l], w.h, T, md.d, md.eps, nullptr, T, w.status, c->pdl);
     }
+    if (int rc = tap(l, HSD_TAP_H_FFN, w.h, 2 * row_d)) return rc;
     if (c->simt) {
       {
         Scope s(c, st, KC_GEMM_GATEUP);
@@ -384,7 +390,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         g.tmB = &c->tm_gate_up[l];
         g.tmC = tm_act_st;
         g.M = T; g.n_out = 2 * md.ffn; g.K = md.d; g.mode = GS_SWIGLU;
-        g.status = w.status; g.n_sms = c->n_sms; g.max_splits = 1; g.pdl = c->pdl; g.pair = c->pair;
+        g.status = w.status; g.n_sms = c->n_sms; g.device = c->device; g.max_splits = 1; g.pdl = c->pdl; g.pair = c->pair;
         if (launch_gemm_sm100(st, g)) return fail_cuda(c);
       }
       {
@@ -394,10 +400,12 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         g.tmB = &c->tm_down[l];
         g.tmC = tm_x_add;
         g.M = T; g.n_out = md.d; g.K = md.ffn; g.mode = GS_ADD_F32;
-        g.status = w.status; g.n_sms = c->n_sms; g.max_splits = c->max_splits; g.pdl = c->pdl; g.pair = c->pair;
+        g.status = w.status; g.n_sms = c->n_sms; g.device = c->device; g.max_splits = c->max_splits; g.pdl = c->pdl; g.pair = c->pair;
         if (launch_gemm_sm100(st, g)) return fail_cuda(c);
       }
     }
+    if (int rc = tap(l, HSD_TAP_ACT, w.act, 2 * (size_t)T * md.ffn)) return rc;
+    if (int rc = tap(l, HSD_TAP_X, w.x, 4 * row_d)) return rc;
   }
   return check_cuda(c);
 }
@@ -421,7 +429,7 @@ int run_lm_head(hsd_ctx* c, const Ws& w, int rows, const int* row_next, cudaStre
     g.tmB = &c->tm_lm_head;
     g.M = rows; g.n_out = md.V; g.K = md.d; g.mode = GS_ARGMAX;
     g.out = o;
-    g.status = w.status; g.n_sms = c->n_sms; g.max_splits = 1; g.pdl = c->pdl; g.pair = c->pair;
+    g.status = w.status; g.n_sms = c->n_sms; g.device = c->device; g.max_splits = 1; g.pdl = c->pdl; g.pair = c->pair;
     if (launch_gemm_sm100(st, g)) return fail_cuda(c);
   }
   return check_cuda(c);
@@ -443,7 +451,7 @@ int verify_common(hsd_ctx* c, const hsd_kv* kv, const StepArgs& a, float log_tau
   if (rc) return rc;
   {
     Scope s(c, st, KC_RMSNORM);
-    launch_rmsnorm(st, w.x, c->final_norm, w.h, a.total_q, c->md.d, c->md.eps, nullptr, c->pdl);
+    launch_rmsnorm(st, w.x, c->final_norm, w.h, a.total_q, c->md.d, c->md.eps, nullptr, a.total_q, w.status, c->pdl);
   }
   rc = run_lm_head(c, w, a.total_q, w.rm.row_next, st);
   if (rc) return rc;
@@ -550,10 +558,9 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
   c->hg_seen_valid = false;
   c->hg_exec = nullptr;
   c->hg_launches = 0;
-  c->prof_last = nullptr;
-  c->prof_last_stream = nullptr;
   c->attn_target_items = 2 * c->n_sms;   // one item per CTA slot: slicing costs a partial hand-over per slice
   c->attn_min_chunk = 8;
+  c->tap_layer = -1; c->tap_which = 0; c->tap_dst = nullptr; c->tap_bytes = 0;
   c->last_cuda_error = 0;
   c->launches = 0;
   c->profiling = false;
@@ -579,7 +586,7 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
 
 int hsd_destroy(hsd_ctx* c) {
   if (!c) return HSD_ERR_INVALID_ARG;
-  for (auto& e : c->prof_events) { if (e.own_a) cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
+  for (auto& e : c->prof_events) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
   for (auto& e : c->event_pool) cudaEventDestroy(e);
   if (c->hg_exec) cudaGraphExecDestroy(c->hg_exec);
   if (c->pin) cudaFreeHost(c->pin);
@@ -612,11 +619,11 @@ int hsd_prefill(hsd_ctx* c, const hsd_kv* kv, int n_seqs, const int* cu_len, con
   if (rc) return rc;
   {
     Scope s(c, st, KC_RMSNORM);
-    launch_select_last_rows(st, w.rm, n_seqs, w.sel_rows, c->pdl);
+    launch_select_last_rows(st, w.rm, n_seqs, w.sel_rows, w.status, c->pdl);
   }
   {
     Scope s(c, st, KC_RMSNORM);
-    launch_rmsnorm(st, w.x, c->final_norm, w.h, n_seqs, c->md.d, c->md.eps, w.sel_rows, c->pdl);
+    launch_rmsnorm(st, w.x, c->final_norm, w.h, n_seqs, c->md.d, c->md.eps, w.sel_rows, total_rows, w.status, c->pdl);
   }
   rc = run_lm_head(c, w, n_seqs, nullptr, st);
   if (rc) return rc;
@@ -670,7 +677,7 @@ int hsd_verify_tree(hsd_ctx* c, const hsd_kv* kv, int n_seqs, const int* cu_q, c
   if (rc) return rc;
   {
     Scope s(c, st, KC_RMSNORM);
-    launch_rmsnorm(st, w.x, c->final_norm, w.h, 2 * total_q, c->md.d, c->md.eps, w.rm.lm_src, c->pdl);
+    launch_rmsnorm(st, w.x, c->final_norm, w.h, 2 * total_q, c->md.d, c->md.eps, w.rm.lm_src, total_q, w.status, c->pdl);
   }
   rc = run_lm_head(c, w, 2 * total_q, w.rm.lm_next, st);
   if (rc) return rc;
@@ -909,9 +916,8 @@ long long hsd_launch_count(const hsd_ctx* c) { return c ? c->launches : 0; }
 
 int hsd_profile_enable(hsd_ctx* c, int enable) {
   if (!c) return HSD_ERR_INVALID_ARG;
-  for (auto& e : c->prof_events) { if (e.own_a) c->event_pool.push_back(e.a); c->event_pool.push_back(e.b); }
+  for (auto& e : c->prof_events) { c->event_pool.push_back(e.a); c->event_pool.push_back(e.b); }
   c->prof_events.clear();
-  c->prof_last = nullptr;
   memset(c->prof_ms, 0, sizeof(c->prof_ms));
   memset(c->prof_n, 0, sizeof(c->prof_n));
   c->profiling = enable != 0;
@@ -927,12 +933,11 @@ int hsd_profile_read(hsd_ctx* c, int cap, const char** names, double* total_ms, 
     c->prof_ms[e.kc] += ms;
     c->prof_n[e.kc] += 1;
   }
-  for (auto& e : c->prof_events) {      // recycle only after every interval has been read (events are shared)
-    if (e.own_a) c->event_pool.push_back(e.a);
+  for (auto& e : c->prof_events) {
+    c->event_pool.push_back(e.a);
     c->event_pool.push_back(e.b);
   }
   c->prof_events.clear();
-  c->prof_last = nullptr;
   int n = 0;
   for (int k = 0; k < KC_COUNT; ++k) {
     if (!c->prof_n[k]) continue;
@@ -971,6 +976,17 @@ int hsd_debug_buffer(hsd_ctx* c, const void* workspace, int total_q, int n_seqs,
   return HSD_OK;
 }
 
+int hsd_debug_tap(hsd_ctx* c, int layer, int which, void* dst, size_t dst_bytes) {
+  if (!c) return HSD_ERR_INVALID_ARG;
+  if (layer < 0) { c->tap_layer = -1; return HSD_OK; }
+  if (layer >= c->md.n_layers || which < HSD_TAP_X || which > HSD_TAP_X_MID || !dst) return HSD_ERR_INVALID_ARG;
+  c->tap_layer = layer;
+  c->tap_which = which;
+  c->tap_dst = dst;
+  c->tap_bytes = dst_bytes;
+  return HSD_OK;
+}
+
 // Shared body of the LM-head operator: rows of h -> per-row argmax / max logit / next-token logit, with
 // `best` (8 bytes per row) as the only scratch.
 static int lm_head_argmax_impl(hsd_ctx* c, const void* h, int rows, const int* next_tokens, unsigned long long* best,
@@ -991,7 +1007,7 @@ static int lm_head_argmax_impl(hsd_ctx* c, const void* h, int rows, const int* n
       g.tmB = &c->tm_lm_head;
       g.M = rows; g.n_out = md.V; g.K = md.d; g.mode = GS_ARGMAX;
       g.out = o;
-      g.status = nullptr; g.n_sms = c->n_sms; g.max_splits = 1; g.pdl = false; g.pair = c->pair;
+      g.status = nullptr; g.n_sms = c->n_sms; g.device = c->device; g.max_splits = 1; g.pdl = false; g.pair = c->pair;
       if (launch_gemm_sm100(st, g)) return fail_cuda(c);
     }
   }
@@ -1071,7 +1087,7 @@ int hsd_op_linear(hsd_ctx* c, const void* A, const void* W, void* C, int M, int 
   if (mode == 1 ? make_tmap_2d_f32(&g.tmC, C, M, ldc, 32) : make_tmap_2d(&g.tmC, C, M, ldc, 32)) return HSD_ERR_CUDA;
   g.tmB = &wm;
   g.M = M; g.n_out = n_out; g.K = K; g.mode = mode;
-  g.status = nullptr; g.n_sms = c->n_sms; g.max_splits = c->max_splits; g.pdl = false; g.pair = c->pair;
+  g.status = nullptr; g.n_sms = c->n_sms; g.device = c->device; g.max_splits = c->max_splits; g.pdl = false; g.pair = c->pair;
   g.force_bn = c->force_bn; g.force_splits = c->force_splits;
   if (launch_gemm_sm100(st, g)) return fail_cuda(c);
   return check_cuda(c);

@@ -525,12 +525,13 @@ done:
 
 int launch_attn_sm100(cudaStream_t st, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                       const AttnPlan& plan, const KvView& kv, const ModelDims& md, int layer, bf16* out, int n_sms,
-                      int* status, float* split_ws, const uint4* anc, bool pdl) {
-  static bool attr_set = false;
-  if (!attr_set) {
+                      int device, int* status, float* split_ws, const uint4* anc, bool pdl) {
+  static bool attr_set[kMaxDevices] = {};          // the attribute is per device
+  if (device < 0 || device >= kMaxDevices) return -1;
+  if (!attr_set[device]) {
     if (cudaFuncSetAttribute(attn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_SMEM) != cudaSuccess)
       return -1;
-    attr_set = true;
+    attr_set[device] = true;
   }
   AttnParams p;
   p.plan = plan;

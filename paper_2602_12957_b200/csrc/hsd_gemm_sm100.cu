@@ -414,7 +414,12 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           if (nxt >= n0 && nxt < n0 + BN) p.out.zdraft[row] = zd;
         }
       } else if (MODE == GS_QKV_ROPE) {
-        const int phys = row_ok ? p.qkv.row_kv[row] : 0;
+        // row_kv comes from the step's set-up kernel: after a failed device-side check it was not written, so
+        // nothing is stored through it (q included: the step is a no-op), nor through a row outside the pool
+        const bool live = !(p.status && *p.status);
+        int phys = (row_ok && live) ? p.qkv.row_kv[row] : 0;
+        const bool kv_ok = live && phys >= 0 && phys < p.qkv.kv_rows;
+        if (!kv_ok) phys = 0;
         const int blk = phys >> 6, off = phys & 63;
 #pragma unroll 1
         for (int hh = 0; hh < BN / 64; ++hh) {
@@ -471,12 +476,12 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             }
             fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) {
+            if (lane == 0 && live) {
               tma_store_2d(&tmC, buf, head * 64, wrow0);
               bulk_commit();
             }
             ++n_stores;
-          } else if (row_ok) {
+          } else if (row_ok && kv_ok) {
             // K and V rows go to the paged pool: one 128-byte line per (token, kv head)
             const bool is_k = head < p.qkv.Hq + p.qkv.Hkv;
             bf16* pool = is_k ? p.qkv.k_pool_layer : p.qkv.v_pool_layer;
@@ -514,12 +519,13 @@ template <int BN, int MODE, bool PAIR>
 static int launch_one(cudaStream_t st, const GemmSm100Args& a, int splits) {
   using C = Cfg<BN, PAIR>;
   constexpr int OUT_N = (MODE == GS_SWIGLU) ? BN / 2 : BN;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static bool attr_set[kMaxDevices] = {};          // the attribute is per device
+  if (a.device < 0 || a.device >= kMaxDevices) return -1;
+  if (!attr_set[a.device]) {
     if (cudaFuncSetAttribute(gemm_sm100_kernel<BN, MODE, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              C::SMEM_BYTES) != cudaSuccess)
       return -1;
-    attr_set = true;
+    attr_set[a.device] = true;
   }
   GemmDev p;
   p.M = a.M;

@@ -7,6 +7,8 @@ namespace hsd {
 
 typedef __nv_bfloat16 bf16;
 
+constexpr int kMaxDevices = 64;    // device ordinals the per-device launch state is kept for
+
 struct ModelDims {
   int n_layers, d, Hq, Hkv, D, ffn, V, qkv_out, group;
   float rope_base, eps;
@@ -68,11 +70,12 @@ void launch_setup_rows(cudaStream_t st, const SetupArgs& a, const KvView& kv, co
                        int* tile_count, bool pdl);
 void launch_embed(cudaStream_t st, const RowMeta& rm, const bf16* table, const bf16* embeds, float* x, int T, int d,
                   const int* status, bool pdl);
-// h[r] = bf16(rmsnorm(x[src]) * gain), src = sel_rows ? sel_rows[r] : r
+// h[r] = bf16(rmsnorm(x[src]) * gain), src = sel_rows ? sel_rows[r] : r.  The gather form (sel_rows != nullptr) writes
+// nothing when *status is set or src is outside [0, src_rows): the index comes from an earlier kernel of the step.
 void launch_rmsnorm(cudaStream_t st, const float* x, const bf16* gain, bf16* h, int rows, int d, float eps,
-                    const int* sel_rows, bool pdl);
-// last row of every sequence (prefill's LM-head rows)
-void launch_select_last_rows(cudaStream_t st, const RowMeta& rm, int n_seqs, int* sel_rows, bool pdl);
+                    const int* sel_rows, int src_rows, const int* status, bool pdl);
+// last row of every sequence (prefill's LM-head rows); -1 for every sequence when *status is set
+void launch_select_last_rows(cudaStream_t st, const RowMeta& rm, int n_seqs, int* sel_rows, const int* status, bool pdl);
 // q_norm / k_norm: per-head RMSNorm gains applied before the rotation, or nullptr
 void launch_rope_kvwrite(cudaStream_t st, const float* qkv, const RowMeta& rm, const KvView& kv, const ModelDims& md,
                          int layer, bf16* q, int T, const int* status, const bf16* q_norm, const bf16* k_norm);
@@ -151,7 +154,7 @@ void launch_attn_plan(cudaStream_t st, const RowMeta& rm, const AttnPlan& pl, in
                       int target_items, int min_chunk, const int* tile_count, const int* status, bool pdl);
 int launch_attn_sm100(cudaStream_t st, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                       const AttnPlan& plan, const KvView& kv, const ModelDims& md, int layer, bf16* out, int n_sms,
-                      int* status, float* split_ws, const uint4* anc, bool pdl);
+                      int device, int* status, float* split_ws, const uint4* anc, bool pdl);
 
 // ---- plain SIMT GEMM (hsd_gemm_simt.cu): the debug cross-check and hsd_debug_logits --------------
 enum GemmMode { GM_STORE_BF16 = 0, GM_ADD_F32 = 1, GM_SWIGLU = 2, GM_STORE_F32 = 3, GM_ARGMAX = 4 };
@@ -181,6 +184,7 @@ int tma_init();   // resolves cuTensorMapEncodeTiled; 0 on success
 
 struct QkvEpilogue {      // fused RoPE + paged KV write (QKV projection)
   const int* row_kv;
+  int kv_rows;            // rows of one layer of the pool (blocks x 64): a physical row outside it is never written
   const float2* rope_cs;
   bf16* q_out;            // [T, Hq*64]
   bf16* k_pool_layer;     // layer base of the K pool
@@ -200,6 +204,7 @@ struct GemmSm100Args {
   QkvEpilogue qkv;
   int* status;
   int n_sms;
+  int device;                  // CUDA device ordinal of the launch (per-device kernel attributes)
   int max_splits;              // GS_ADD_F32: most K slices per tile (1 = none; slices add in arrival order)
   bool pdl;                    // launch with programmatic stream serialization
   int pair;                    // CTA pairs (clusters of two sharing a 256-row tile) may be used

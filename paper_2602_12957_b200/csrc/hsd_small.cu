@@ -179,13 +179,18 @@ void launch_embed(cudaStream_t st, const RowMeta& rm, const bf16* table, const b
 // between the reduction and the scaling (d <= 2048), so x is read once.
 template <int VEC>   // VEC float4 per lane: d = 128 * VEC
 __global__ void rmsnorm_kernel(const float* __restrict__ x, const bf16* __restrict__ gain, bf16* __restrict__ h,
-                               int rows, int d, float eps, const int* __restrict__ sel_rows) {
+                               int rows, int d, float eps, const int* __restrict__ sel_rows, int src_rows,
+                               const int* __restrict__ status) {
   pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
   pdl_launch_dependents();
   const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (r >= rows) return;
   const int lane = threadIdx.x & 31;
+  // the gather form follows an index an earlier kernel of the step wrote: after a failed device-side check that
+  // index was never written, so nothing is read through it (and an index outside the source is never followed)
+  if (sel_rows && status && *status) return;
   const int src = sel_rows ? sel_rows[r] : r;
+  if (src < 0 || src >= src_rows) return;
   const float4* xp = reinterpret_cast<const float4*>(x + (size_t)src * d);
   float4 v[VEC];
   float ss = 0.f;
@@ -208,27 +213,28 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const bf16* __restri
   }
 }
 void launch_rmsnorm(cudaStream_t st, const float* x, const bf16* gain, bf16* h, int rows, int d, float eps,
-                    const int* sel_rows, bool pdl) {
+                    const int* sel_rows, int src_rows, const int* status, bool pdl) {
   if (rows <= 0) return;
   dim3 grid((rows + 7) / 8), block(256);
+#define HSD_RMS_CASE(V) \
+  case V: launch_kernel(rmsnorm_kernel<V>, grid, block, 0, st, pdl, x, gain, h, rows, d, eps, sel_rows, src_rows, status); break;
   switch (d / 128) {
-    case 1: launch_kernel(rmsnorm_kernel<1>, grid, block, 0, st, pdl, x, gain, h, rows, d, eps, sel_rows); break;
-    case 2: launch_kernel(rmsnorm_kernel<2>, grid, block, 0, st, pdl, x, gain, h, rows, d, eps, sel_rows); break;
-    case 4: launch_kernel(rmsnorm_kernel<4>, grid, block, 0, st, pdl, x, gain, h, rows, d, eps, sel_rows); break;
-    case 8: launch_kernel(rmsnorm_kernel<8>, grid, block, 0, st, pdl, x, gain, h, rows, d, eps, sel_rows); break;
-    case 16: launch_kernel(rmsnorm_kernel<16>, grid, block, 0, st, pdl, x, gain, h, rows, d, eps, sel_rows); break;
+    HSD_RMS_CASE(1) HSD_RMS_CASE(2) HSD_RMS_CASE(4) HSD_RMS_CASE(8) HSD_RMS_CASE(16)
     default: break;   // hsd_create rejects other widths
   }
+#undef HSD_RMS_CASE
 }
 
-__global__ void select_last_rows_kernel(RowMeta rm, int n_seqs, int* sel_rows) {
+__global__ void select_last_rows_kernel(RowMeta rm, int n_seqs, int* sel_rows, const int* status) {
   pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
   pdl_launch_dependents();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n_seqs) sel_rows[i] = rm.seq_q0[i] + max(rm.seq_n[i], 1) - 1;
+  if (i >= n_seqs) return;
+  // after a failed check the per-sequence metadata was not written: name no row at all
+  sel_rows[i] = *status ? -1 : rm.seq_q0[i] + max(rm.seq_n[i], 1) - 1;
 }
-void launch_select_last_rows(cudaStream_t st, const RowMeta& rm, int n_seqs, int* sel_rows, bool pdl) {
-  launch_kernel(select_last_rows_kernel, dim3((n_seqs + 127) / 128), dim3(128), 0, st, pdl, rm, n_seqs, sel_rows);
+void launch_select_last_rows(cudaStream_t st, const RowMeta& rm, int n_seqs, int* sel_rows, const int* status, bool pdl) {
+  launch_kernel(select_last_rows_kernel, dim3((n_seqs + 127) / 128), dim3(128), 0, st, pdl, rm, n_seqs, sel_rows, status);
 }
 
 __global__ void clear_best_kernel(unsigned long long* row_best, float* zdraft, int rows) {
@@ -383,10 +389,13 @@ void launch_attn_simt(cudaStream_t st, const bf16* q, const RowMeta& rm, const K
 __global__ void accept_kernel(AcceptArgs a, RowMeta rm, const int* status) {
   pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
   pdl_launch_dependents();
-  if (*status) return;
   const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (i >= a.n_seqs) return;
   const int lane = threadIdx.x & 31;
+  if (*status) {            // a failed step decides nothing: -1 makes the commit that follows leave the lengths alone
+    if (lane == 0) { a.accept_len[i] = -1; a.n_emit[i] = 0; }
+    return;
+  }
   const int q0 = rm.seq_q0[i], n = rm.seq_n[i];
   if (n <= 0) {
     if (lane == 0) { a.accept_len[i] = 0; a.n_emit[i] = 0; }
@@ -431,10 +440,13 @@ void launch_accept(cudaStream_t st, const AcceptArgs& a, const RowMeta& rm, cons
 __global__ void tree_accept_kernel(TreeAcceptArgs a, RowMeta rm, const int* status) {
   pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
   pdl_launch_dependents();
-  if (*status) return;
   const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (i >= a.n_seqs) return;
   const int lane = threadIdx.x & 31;
+  if (*status) {            // a failed step decides nothing: the compaction and the commit that follow skip -1
+    if (lane == 0) { a.accept_len[i] = -1; a.n_emit[i] = 0; }
+    return;
+  }
   const int q0 = rm.seq_q0[i], n = rm.seq_n[i], T = a.total_q;
   if (n <= 0) {
     if (lane == 0) { a.accept_len[i] = 0; a.n_emit[i] = 0; }
@@ -538,12 +550,14 @@ __global__ void tree_compact_kernel(KvView kv, int n_kv_heads, int n_seqs, const
   const int slot = seq_slots ? seq_slots[i] : i;
   if (slot < 0 || slot >= kv.n_slots) return;
   const int a = accept_len[i];
+  if (a < 0) return;                                     // the step failed a device-side check: nothing to keep
   const int L = kv.seq_lens[slot];
+  if (L < 0 || (long long)L + max_q_len > (long long)kv.max_blocks * HSD_KV_BLOCK) return;
   const int* bt = kv.block_table + (size_t)slot * kv.max_blocks;
   const int chunks = n_kv_heads * 2 * 8;                 // 16-byte chunks of one token's K and V rows in a layer
   for (int d = 1; d <= a && d < max_q_len; ++d) {
     const int r = accept_rows[(size_t)i * max_q_len + d - 1];
-    if (r != d && r > 0 && (L + r) / HSD_KV_BLOCK < kv.max_blocks) {
+    if (r != d && r > 0 && r < max_q_len) {              // a row of this call (L + r is within the table, see above)
       const int ps = L + r, pd = L + d;
       const int bs = bt[ps / HSD_KV_BLOCK], bd = bt[pd / HSD_KV_BLOCK];
       if (bs >= 0 && bs < kv.n_blocks && bd >= 0 && bd < kv.n_blocks) {

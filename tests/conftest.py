@@ -19,6 +19,10 @@ def pytest_collection_modifyitems(config, items):
     except Exception:
         have = False
     if have:
+        # the long-document oracle takes minutes on the CPU: start it now, behind the other tests
+        if any(it.name.startswith("test_long_document_full_size") for it in items) and len(items) > 1:
+            from tests import harness
+            harness.long_document_oracle()
         return
     skip = pytest.mark.skip(reason="no CUDA device")
     for it in items:

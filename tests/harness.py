@@ -129,3 +129,59 @@ def check_first_token(tag, o: OracleSeq, gpu_first: int):
         assert gpu_first == o.pending, f"{tag}: prefill token {gpu_first} != {o.pending}"
     else:
         assert o.pending_logits[gpu_first] >= o.pending_logits.max() - GAP_EXACT
+
+
+# ------------------------------------------------------------------------------------------------ long-document oracle
+LONG_CONTEXT = 16384
+_long_job = {}
+
+
+def long_document_oracle():
+    """The oracle side of the full-size long-document case, computed once per session on a background thread (numpy
+    releases the interpreter lock in its kernels, so it overlaps with the tests that run meanwhile).  Returns a dict:
+    seq (prefix rows), draft (2,048 random tokens), weights, pending() -> the oracle's first token after the prefix
+    (waits for the prefill), results() -> {1024: VerifyResult, 2048: VerifyResult} (waits for everything)."""
+    import threading
+    if _long_job:
+        return _long_job
+    cfg = I.DECODER
+    rng = np.random.Generator(np.random.PCG64(I.BASE_SEED + 3 + 1_000_003))
+    L = LONG_CONTEXT
+    emb = np.zeros((L, cfg.d_model), np.float32)
+    emb[:2048] = I.bf16_round(rng.standard_normal((2048, cfg.d_model), dtype=np.float32))
+    ids = np.full(L, -1, np.int32)
+    ids[2048:] = rng.integers(0, cfg.vocab, size=L - 2048, dtype=np.int32)       # committed text
+    draft = rng.integers(0, cfg.vocab, size=2048, dtype=np.int32)
+    weights = I.make_weights(cfg, I.BASE_SEED + 1)
+    state = {"error": None}
+    prefilled = threading.Event()
+
+    def work():
+        try:
+            model = O.Decoder(cfg, weights, np.float32)
+            cache = O.CachedSequence(model)
+            state["pending"] = cache.prefill(emb, ids)
+            prefilled.set()
+            state["res"] = {k: O.verify_cached(cache, state["pending"], draft[:k], keep_logits=True) for k in (1024, 2048)}
+        except BaseException as e:          # surfaces in the test that asks for the result
+            state["error"] = e
+            prefilled.set()
+
+    t = threading.Thread(target=work, name="long-document-oracle", daemon=True)
+    t.start()
+
+    def pending():
+        prefilled.wait()
+        if state["error"] is not None:
+            raise state["error"]
+        return state["pending"]
+
+    def results():
+        t.join()
+        if state["error"] is not None:
+            raise state["error"]
+        return state["res"]
+
+    _long_job.update(seq=I.SeqInput(emb, ids, 2048, 0, draft, True), draft=draft, weights=weights, pending=pending,
+                     results=results)
+    return _long_job

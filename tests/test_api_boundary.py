@@ -54,6 +54,9 @@ def test_constants_match_the_header(B):
                  "HSD_FLAG_DETERMINISTIC", "HSD_FLAG_NO_PDL", "HSD_FLAG_NO_PAIR", "HSD_FLAG_NO_HOST_GRAPH"):
         m = re.search(rf"#define\s+{name}\s+(-?\d+)", text)
         assert m and int(m.group(1)) == getattr(B, name), name
+    for k, name in enumerate(("X", "H_ATTN", "H_FFN", "Q", "ATTN", "ACT", "X_MID")):
+        m = re.search(rf"#define\s+HSD_TAP_{name}\s+(\d+)", text)
+        assert m and int(m.group(1)) == k == getattr(B, "HSD_TAP_" + name), name
     for name in ("INVALID_ARG", "SHAPE", "TOO_LONG", "WORKSPACE", "KV_CAPACITY", "CUDA", "DEVICE_CHECK", "NO_DEVICE"):
         m = re.search(rf"#define\s+HSD_ERR_{name}\s+\((-\d+)\)", text)
         assert m and int(m.group(1)) == getattr(B, "HSD_ERR_" + name), name
@@ -83,6 +86,7 @@ def test_host_side_argument_checks_need_no_device(B):
     assert B.hsd_verify_tree(None, None, 1, None, None, None, None, 1, 1, 0.0, None, None, None, None, None, None, None,
                              None, 0, None) == B.HSD_ERR_INVALID_ARG
     assert B.hsd_kv_commit_tree(None, None, 1, None, None, None, 1, None, None) == B.HSD_ERR_INVALID_ARG
+    assert B.hsd_debug_tap(None, 0, 0, None, 0) == B.HSD_ERR_INVALID_ARG
     assert B.hsd_dsv_build(None, 1, 3, None, None, None, 0, None, 0, None, 0, None, 128, None, None, None, None,
                            None) == B.HSD_ERR_INVALID_ARG
 

@@ -101,3 +101,87 @@ def test_device_side_checks_report_instead_of_faulting():
     assert B.hsd_verify_regions(*args, 3, 6, 0.5, *tail, eng.ws.ptr, eng.ws.bytes, st_) == B.HSD_ERR_INVALID_ARG
     assert B.hsd_verify_regions(*args, 3, 6, 0.0, None, *tail[1:], eng.ws.ptr, eng.ws.bytes, st_) == B.HSD_ERR_INVALID_ARG
     assert B.hsd_launch_count(dm.ctx) == n0
+
+
+def test_failed_device_check_leaves_cache_and_lengths_untouched():
+    """A step that trips a device-side check is a no-op: no K/V row is written, no length advances, and the decision
+    outputs say so (accept_len -1, n_emit 0) — also on a workspace no valid call has ever filled (zeroed here, so that
+    a store through a never-written row index would land in bounds, on physical row 0, and show up in the comparison)."""
+    import torch
+    from paper_2602_12957_b200 import binding as B
+    from paper_2602_12957_b200 import runtime as R
+    cfg = I.TINY
+    wl = I.tiny_workload()
+    weights = I.make_weights(cfg, wl.seed)
+    dm = R.DeviceModel(cfg, weights, 0)
+    S = 2
+    kv = R.KvCache(dm, [320, 320], seed=0)
+    eng = R.Engine(dm, kv, 512, S)
+    eng.prefill([s.prefix_embeds for s in wl.seqs[:S]], [s.prefix_ids for s in wl.seqs[:S]])
+    eng.check_device("prefill")
+    torch.cuda.synchronize()
+    k0, v0, lens0 = kv.k_pool.clone(), kv.v_pool.clone(), kv.seq_lens.clone()
+    toks = np.array([1, 2, 3, 4, 5, 6], np.int32)
+    cu = np.array([0, 3, 6], np.int32)
+    bad_tok = toks.copy(); bad_tok[4] = cfg.vocab + 5
+    cases = [("token", bad_tok, cu, 3, 3), ("offsets", toks, np.array([0, 4, 3], np.int32), 4, 1),
+             ("too_long", toks, np.array([0, 5, 6], np.int32), 3, 2)]
+
+    def fresh_engine():
+        e = R.Engine(dm, kv, 512, S)
+        e.ws._raw.zero_()
+        return e
+
+    def unchanged():
+        torch.cuda.synchronize()
+        return (torch.equal(kv.k_pool, k0) and torch.equal(kv.v_pool, v0) and torch.equal(kv.seq_lens, lens0))
+
+    for name, t, c, max_q, code in cases:
+        e2 = fresh_engine()
+        out = e2.alloc_outputs(S, max_q, 6)
+        for v in out.values():
+            v.fill_(7)
+        out = e2.verify_regions(e2._i32(t), e2._i32(c), max_q, 6, out=out)
+        e2.commit(out["accept_len"])
+        st, words = e2.device_status()
+        assert st == B.HSD_ERR_DEVICE_CHECK and words[0] == code, (name, st, words)
+        assert out["accept_len"].cpu().tolist() == [-1, -1] and out["n_emit"].cpu().tolist() == [0, 0], name
+        assert unchanged(), name
+    # capacity: one free row left, three needed (lengths are the caller's; restored afterwards)
+    e2 = fresh_engine()
+    kv.seq_lens[1] = kv.max_blocks * 64 - 1
+    lens_cap = kv.seq_lens.clone()
+    out = e2.verify_regions(e2._i32(toks), e2._i32(cu), 3, 6)
+    e2.commit(out["accept_len"])
+    st, words = e2.device_status()
+    assert st == B.HSD_ERR_DEVICE_CHECK and words[0] == 4
+    assert torch.equal(kv.seq_lens, lens_cap) and torch.equal(kv.k_pool, k0) and torch.equal(kv.v_pool, v0)
+    kv.seq_lens.copy_(lens0)
+    # the host-buffer entry with commit folded in: the error comes back and nothing moved
+    e2 = fresh_engine()
+    h_t, h_c = torch.from_numpy(bad_tok).pin_memory(), torch.from_numpy(cu).pin_memory()
+    h_acc = torch.full((S,), 7, dtype=torch.int32).pin_memory()
+    h_nem = torch.full((S,), 7, dtype=torch.int32).pin_memory()
+    h_emit = torch.full((S, 3), 7, dtype=torch.int32).pin_memory()
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for _ in range(3):          # eager, capturing and replayed calls of the library's own graph
+        rc, _ = B.hsd_verify_regions_host(dm.ctx, kv.c, S, h_c, h_t, None, 0.0, 1, h_acc, h_emit, h_nem, e2.ws.ptr,
+                                          e2.ws.bytes, side.cuda_stream)
+        assert rc == B.HSD_ERR_DEVICE_CHECK
+        assert h_acc.tolist() == [-1, -1] and h_nem.tolist() == [0, 0]
+        assert unchanged()
+    # candidate trees: a parent pointer that names a later row
+    e2 = R.Engine(dm, kv, 512, S)
+    e2.ws._raw.zero_()
+    parent = np.array([-1, 0, 1, -1, 2, 0], np.int32)          # row 1 of the second tree points at row 2
+    out = e2.verify_tree(e2._i32(toks), e2._i32(cu), e2._i32(parent), 3, 6)
+    e2.commit_tree(out["accept_len"], out["accept_rows"])
+    st, words = e2.device_status()
+    assert st == B.HSD_ERR_DEVICE_CHECK and words[0] == 7
+    assert out["accept_len"].cpu().tolist() == [-1, -1]
+    assert unchanged()
+    # and the context still works
+    out = eng.verify_regions(eng._i32(toks), eng._i32(cu), 3, 6)
+    st, _ = eng.device_status()
+    assert st == B.HSD_OK and min(out["accept_len"].cpu().tolist()) >= 0

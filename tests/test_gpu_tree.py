@@ -245,7 +245,7 @@ def test_tree_argument_and_device_checks():
                            out["emit_tokens"], out["n_emit"], out["accept_rows"], None, None, None, small.ptr,
                            small.bytes, torch.cuda.current_stream().cuda_stream)
     assert st == B.HSD_ERR_WORKSPACE
-    # a parent that is not an earlier row: device status 7 with the packed row, outputs untouched, context usable
+    # a parent that is not an earlier row: device status 7 with the packed row, no decision (-1, nothing emitted), context usable
     for bad_row, bad_val in ((3, 3), (7, 9), (5, 0), (2, -1)):
         bad = good.copy()
         bad[bad_row] = bad_val
@@ -253,7 +253,7 @@ def test_tree_argument_and_device_checks():
         eng.verify_tree(toks, cu, eng._i32(bad), 5, 10, out=out)
         st, words = eng.device_status()
         assert st == B.HSD_ERR_DEVICE_CHECK and words[0] == 7, (bad_row, words)
-        assert out["accept_len"].cpu().tolist() == [-5, -5]
+        assert out["accept_len"].cpu().tolist() == [-1, -1] and out["n_emit"].cpu().tolist() == [0, 0]
     eng.verify_tree(toks, cu, eng._i32(good), 5, 10, out=out)
     eng.check_device("after the bad trees")
     assert all(0 <= a <= 4 for a in out["accept_len"].cpu().tolist())

@@ -76,11 +76,26 @@ def oracle_full_logits(model, emb, ids):
     return model.logits(O.decoder_forward(model, x, np.arange(n), O.causal_allowed(n)))
 
 
+def library_input_rows(m, emb, ids):
+    """Input rows built WITHOUT the oracle's `embed_rows`: token rows come from the library decoder's own embedding
+    module fed with the id, visual rows (id < 0) are copied in by position."""
+    ids = np.asarray(ids)
+    x = torch.zeros(len(ids), m.config.hidden_size, dtype=torch.float64)
+    with torch.no_grad():
+        for r, t in enumerate(ids.tolist()):
+            if t >= 0:
+                x[r] = m.model.embed_tokens(torch.tensor(t))
+            else:
+                x[r] = torch.from_numpy(np.asarray(emb[r], np.float64))
+    return x
+
+
 def hf_logits(model, emb, ids):
     m = hf_llama(model)
-    x = torch.from_numpy(model.embed_rows(emb, ids))[None]
     with torch.no_grad():
-        return m(inputs_embeds=x).logits[0].numpy()
+        if not np.any(np.asarray(ids) < 0):          # text only: the library gathers its own rows from the ids
+            return m(input_ids=torch.from_numpy(np.asarray(ids, np.int64))[None]).logits[0].numpy()
+        return m(inputs_embeds=library_input_rows(m, emb, ids)[None]).logits[0].numpy()
 
 
 def test_forward_matches_library_llama():
@@ -98,12 +113,43 @@ def test_forward_matches_library_llama_head_dim_64_mha():
     assert np.max(np.abs(oracle_full_logits(model, emb, ids) - hf_logits(model, emb, ids))) < 2e-7
 
 
+def interleaved_prefix(model, seed):
+    """Visual and text rows interleaved, token id 0 and the largest id among the text rows, and an embedding row
+    supplied (and to be ignored) at every text position."""
+    rng = np.random.default_rng(seed)
+    V = model.cfg.vocab
+    ids = np.array([-1, -1, 0, 5, -1, V - 1, 0, 3, -1, -1, 11, 0], np.int64)
+    emb = rng.standard_normal((len(ids), model.cfg.d_model)).astype(np.float32)
+    return emb, ids
+
+
+def test_input_rows_match_library_embedding_module():
+    """`Decoder.embed_rows` against the library decoder's own embedding lookup: a text-only prefix goes in as
+    input ids, a mixed one has its visual rows spliced in by the test; neither side of the comparison calls
+    `embed_rows` except the oracle's."""
+    model = small_model()
+    m = hf_llama(model)
+    emb, ids = interleaved_prefix(model, 21)
+    x = model.embed_rows(emb, ids)
+    assert np.array_equal(x, library_input_rows(m, emb, ids).numpy())
+    assert np.array_equal(x[2], model.weights["embed"][0].astype(np.float64))          # id 0 is a token, not a visual row
+    assert np.array_equal(x[0], emb[0].astype(np.float64)) and not np.array_equal(x[3], emb[3].astype(np.float64))
+    z, zr = oracle_full_logits(model, emb, ids), hf_logits(model, emb, ids)
+    assert np.max(np.abs(z - zr)) < 2e-7
+    text = np.array([0, 7, 96, 0, 1, 50], np.int64)                                     # library fed with input_ids
+    assert np.max(np.abs(oracle_full_logits(model, None, text) - hf_logits(model, None, text))) < 2e-7
+    with pytest.raises(ValueError):
+        model.embed_rows(None, np.array([3, -1]))
+
+
 @pytest.mark.parametrize("mistake", ["rope_sign", "rope_pairing", "no_scale", "gqa_map", "mask_strict",
-                                     "silu_on_up", "eps_outside", "no_residual_gain"])
+                                     "silu_on_up", "eps_outside", "no_residual_gain", "id_zero_is_visual",
+                                     "embed_row_off_by_one", "visual_rows_from_table"])
 def test_library_pin_catches_planted_mistakes(mistake, monkeypatch):
     """A plausible slip planted in the oracle (CPU only) must break the library pin."""
     model = small_model()
-    emb, ids = mixed_prefix(model, 19, 6, 3)
+    emb, ids = interleaved_prefix(model, 3) if "id_zero" in mistake or "embed_row" in mistake or "visual_rows" in mistake \
+        else mixed_prefix(model, 19, 6, 3)
     zr = hf_logits(model, emb, ids)
     if mistake == "rope_sign":
         def bad(x, pos, base):
@@ -146,6 +192,22 @@ def test_library_pin_catches_planted_mistakes(mistake, monkeypatch):
         monkeypatch.setattr(O, "rmsnorm", lambda x, g, eps: x / (np.sqrt(np.mean(x * x, -1, keepdims=True)) + 1e-2) * g)
     elif mistake == "no_residual_gain":
         monkeypatch.setattr(O, "rmsnorm", lambda x, g, eps: x / np.sqrt(np.mean(x * x, -1, keepdims=True) + eps))
+    elif mistake == "id_zero_is_visual":      # `ids <= 0` instead of `ids < 0` selects the visual row
+        def bad(self, embeds, ids_):
+            ids_ = np.asarray(ids_)
+            x = self.w(self.weights["embed"][np.maximum(ids_, 0)])
+            return np.ascontiguousarray(np.where((ids_ <= 0)[:, None], self.w(np.asarray(embeds)), x))
+        monkeypatch.setattr(O.Decoder, "embed_rows", bad)
+    elif mistake == "embed_row_off_by_one":   # table row id + 1
+        def bad(self, embeds, ids_):
+            ids_ = np.asarray(ids_)
+            x = self.w(self.weights["embed"][np.minimum(np.maximum(ids_, 0) + 1, self.cfg.vocab - 1)])
+            return np.ascontiguousarray(np.where((ids_ < 0)[:, None], self.w(np.asarray(embeds)), x))
+        monkeypatch.setattr(O.Decoder, "embed_rows", bad)
+    elif mistake == "visual_rows_from_table": # the given rows are ignored
+        def bad(self, embeds, ids_):
+            return np.ascontiguousarray(self.w(self.weights["embed"][np.maximum(np.asarray(ids_), 0)]))
+        monkeypatch.setattr(O.Decoder, "embed_rows", bad)
     z = oracle_full_logits(model, emb, ids)
     assert np.max(np.abs(z - zr)) > 1e-4
 
