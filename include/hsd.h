@@ -220,11 +220,59 @@ HSD_API int hsd_verify_tree(hsd_ctx *ctx, const hsd_kv *kv, int n_seqs, const in
  * Candidates: for every draft of the sequence and every position where the window occurs (Eq. 5), the non-empty
  * suffix after it (Eq. 6), in draft order then position order, at most HSD_DSV_MAX_CANDIDATES.  Tree (Eq. 7): one
  * node per distinct prefix, created level by level in candidate order while fewer than max_rows - 1 nodes exist; a
- * candidate whose next node cannot be created stops growing.  Pure integer work: results are exact. */
+ * candidate whose next node cannot be created stops growing.  Pure integer work: results are exact.
+ *   seq_map         dev int32 [n_seqs] or NULL: with a map, sequence i matches against the drafts of OWNER seq_map[i], i.e.
+ *                   drafts seq_draft_off[seq_map[i]] .. seq_draft_off[seq_map[i] + 1] - 1 (lane batches: a lane serves
+ *                   different sequences over time); an entry < 0 or >= n_owners means "no drafts".  n_owners = entries of
+ *                   seq_draft_off minus one (host copy; ignored without a map, where it is n_seqs). */
 HSD_API int hsd_dsv_build(hsd_ctx *ctx, int n_seqs, int window_n, int *window, const int *emit_tokens, const int *n_emit,
                   int emit_stride, const int *draft_tokens, int total_draft_tokens, const int *draft_off,
                   int n_drafts, const int *seq_draft_off, int max_rows, int *q_tokens, int *parent, int *cu_q,
-                  int *n_rows, void *cuda_stream);
+                  int *n_rows, const int *seq_map, int n_owners, void *cuda_stream);
+
+/* Decode loop over a LANE BATCH (Sec. 3.1): Stage 1 runs SpecDecode (Eq. 2) on all regions of a page "in parallel" until
+ * every region's output is complete; Stage 2 (Eq. 4) is the same loop with one lane.  n_lanes lanes step together
+ * (hsd_dsv_build -> hsd_verify_tree -> hsd_kv_commit_tree over the lanes, with seq_slots = lane_slot and seq_map =
+ * lane_seq); a lane serves one sequence until its output has max_new tokens, then takes the next waiting sequence, so the
+ * batch shape stays fixed while regions of different lengths come and go.  All decisions are taken on the device: the
+ * host only polls counters[1] (sequences not finished) now and then.
+ * All pointers are device pointers owned by the caller.
+ *   lane_seq      [n_lanes]            sequence a lane serves, -1 = none (the lane then idles on KV slot idle_slot, whose
+ *                                      length is reset to 0 after every step; give it room for one step's rows)
+ *   lane_slot     [n_lanes]            KV slot of every lane for the next step (pass as seq_slots)
+ *   window        [n_lanes, window_n]  reference window of every lane (pass to hsd_dsv_build WITHOUT emit_tokens: the
+ *                                      advance call below has already taken the emitted tokens in)
+ *   first_token   [n_seqs]             first token of every sequence (hsd_prefill's output): token 0 of its output and
+ *                                      its first pending token
+ *   seq_slot      [n_seqs] or NULL     KV slot of every sequence (NULL: slot = sequence index)
+ *   max_new       [n_seqs]             output length of every sequence (the paper's parsers stop at their end token; the
+ *                                      synthetic decoders have none, so lengths are given)
+ *   out_tokens    [n_seqs, out_stride] outputs; out_len [n_seqs] tokens so far; seq_steps [n_seqs] verification steps
+ *                                      spent; seq_accepted [n_seqs] accepted draft tokens (AAL = accepted / steps, Sec. 4.2)
+ *   counters      [4]                  [0] next waiting sequence, [1] sequences not finished, [2] steps taken */
+typedef struct {
+  int n_lanes, n_seqs, window_n, out_stride, idle_slot;
+  int *lane_seq, *lane_slot, *window;
+  const int *first_token, *seq_slot, *max_new;
+  int *out_tokens, *out_len, *seq_steps, *seq_accepted, *counters;
+} hsd_stage;
+
+/* Start a lane batch: every output gets its first token, lanes take the first sequences of the queue (in order), the
+ * others wait.  Errors: INVALID_ARG (null pointers, n_lanes / n_seqs / out_stride < 1, window_n outside 1..HSD_MAX_WINDOW). */
+HSD_API int hsd_stage_begin(hsd_ctx *ctx, const hsd_stage *stage, const hsd_kv *kv, void *cuda_stream);
+
+/* Between two steps: append every lane's emitted tokens (emit_tokens [n_lanes, emit_stride], n_emit, accept_len: the
+ * outputs of the step's hsd_verify_tree) to its sequence's output up to max_new, count the step and its accepted tokens,
+ * rebuild the lane's window from the output's last tokens, retire finished sequences and give their lanes to the next
+ * waiting ones (lanes in index order, queue order: deterministic).  A lane whose accept_len is -1 (the step failed a
+ * device-side check) is left as it was. */
+HSD_API int hsd_stage_advance(hsd_ctx *ctx, const hsd_stage *stage, const hsd_kv *kv, const int *accept_len,
+                      const int *emit_tokens, const int *n_emit, int emit_stride, void *cuda_stream);
+
+/* The page draft (Eq. 3): all outputs concatenated into draft_tokens (dev int32 [capacity]) with draft_off (dev int32
+ * [n_seqs + 1]) their offsets, in the layout hsd_dsv_build takes; outputs beyond `capacity` are cut. */
+HSD_API int hsd_stage_aggregate(hsd_ctx *ctx, const hsd_stage *stage, int *draft_tokens, int capacity, int *draft_off,
+                        void *cuda_stream);
 
 /* KV maintenance after hsd_verify_tree (Sec. 4.2 counts it in the decode loop): in every layer the K/V rows of the
  * accepted path move from cache rows L + accept_rows[i][d-1] to rows L + d (d = 1..accept_len[i]; L = committed

@@ -34,7 +34,8 @@ EXPORTS = [
     "hsd_verify_page", "hsd_kv_commit", "hsd_verify_regions_host", "hsd_device_status", "hsd_last_cuda_error", "hsd_launch_count",
     "hsd_profile_enable", "hsd_profile_read", "hsd_debug_logits", "hsd_debug_buffer", "hsd_op_linear",
     "hsd_op_lm_head_argmax", "hsd_op_lm_head_argmax_noalloc", "hsd_debug_set_gemm_tile", "hsd_debug_set_attn_plan",
-    "hsd_verify_tree", "hsd_kv_commit_tree", "hsd_dsv_build", "hsd_debug_tap",
+    "hsd_verify_tree", "hsd_kv_commit_tree", "hsd_dsv_build", "hsd_debug_tap", "hsd_stage_begin", "hsd_stage_advance",
+    "hsd_stage_aggregate",
 ]
 HSD_TAP_X, HSD_TAP_H_ATTN, HSD_TAP_H_FFN, HSD_TAP_Q, HSD_TAP_ATTN, HSD_TAP_ACT, HSD_TAP_X_MID = range(7)
 
@@ -66,6 +67,14 @@ class hsd_kv(C.Structure):
                 ("n_slots", C.c_int)]
 
 
+class hsd_stage(C.Structure):
+    _fields_ = [("n_lanes", C.c_int), ("n_seqs", C.c_int), ("window_n", C.c_int), ("out_stride", C.c_int),
+                ("idle_slot", C.c_int), ("lane_seq", C.c_void_p), ("lane_slot", C.c_void_p), ("window", C.c_void_p),
+                ("first_token", C.c_void_p), ("seq_slot", C.c_void_p), ("max_new", C.c_void_p),
+                ("out_tokens", C.c_void_p), ("out_len", C.c_void_p), ("seq_steps", C.c_void_p),
+                ("seq_accepted", C.c_void_p), ("counters", C.c_void_p)]
+
+
 def _load():
     if not os.path.exists(LIB_PATH):
         raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2602_12957_b200.build` "
@@ -85,7 +94,10 @@ def _load():
     lib.hsd_verify_tree.argtypes = [vp, C.POINTER(hsd_kv), i, vp, vp, vp, vp, i, i, f, vp, vp, vp, vp, vp, vp, vp, vp, sz,
                                     vp]
     lib.hsd_kv_commit_tree.argtypes = [vp, C.POINTER(hsd_kv), i, vp, vp, vp, i, vp, vp]
-    lib.hsd_dsv_build.argtypes = [vp, i, i, vp, vp, vp, i, vp, i, vp, i, vp, i, vp, vp, vp, vp, vp]
+    lib.hsd_dsv_build.argtypes = [vp, i, i, vp, vp, vp, i, vp, i, vp, i, vp, i, vp, vp, vp, vp, vp, i, vp]
+    lib.hsd_stage_begin.argtypes = [vp, C.POINTER(hsd_stage), C.POINTER(hsd_kv), vp]
+    lib.hsd_stage_advance.argtypes = [vp, C.POINTER(hsd_stage), C.POINTER(hsd_kv), vp, vp, vp, i, vp]
+    lib.hsd_stage_aggregate.argtypes = [vp, C.POINTER(hsd_stage), vp, i, vp, vp]
     lib.hsd_verify_regions_host.argtypes = [vp, C.POINTER(hsd_kv), i, vp, vp, vp, f, i, vp, vp, vp, C.POINTER(C.c_int), vp, sz, vp]
     lib.hsd_device_status.argtypes = [vp, vp, vp, C.POINTER(C.c_int)]
     lib.hsd_last_cuda_error.argtypes = [vp]
@@ -229,10 +241,35 @@ def hsd_kv_commit_tree(ctx, kv, n_seqs, seq_slots, accept_len, accept_rows, max_
 
 
 def hsd_dsv_build(ctx, n_seqs, window_n, window, emit_tokens, n_emit, emit_stride, draft_tokens, total_draft_tokens,
-                  draft_off, n_drafts, seq_draft_off, max_rows, q_tokens, parent, cu_q, n_rows, stream) -> int:
+                  draft_off, n_drafts, seq_draft_off, max_rows, q_tokens, parent, cu_q, n_rows, stream, seq_map=None,
+                  n_owners: int = 0) -> int:
     return _lib.hsd_dsv_build(ctx, n_seqs, window_n, _p(window), _p(emit_tokens), _p(n_emit), emit_stride,
                               _p(draft_tokens), total_draft_tokens, _p(draft_off), n_drafts, _p(seq_draft_off), max_rows,
-                              _p(q_tokens), _p(parent), _p(cu_q), _p(n_rows), _p(stream))
+                              _p(q_tokens), _p(parent), _p(cu_q), _p(n_rows), _p(seq_map), n_owners, _p(stream))
+
+
+def make_stage(n_lanes, n_seqs, window_n, out_stride, idle_slot, lane_seq, lane_slot, window, first_token, seq_slot,
+               max_new, out_tokens, out_len, seq_steps, seq_accepted, counters) -> hsd_stage:
+    ptr = lambda t: None if t is None else t.data_ptr()
+    return hsd_stage(n_lanes, n_seqs, window_n, out_stride, idle_slot, ptr(lane_seq), ptr(lane_slot), ptr(window),
+                     ptr(first_token), ptr(seq_slot), ptr(max_new), ptr(out_tokens), ptr(out_len), ptr(seq_steps),
+                     ptr(seq_accepted), ptr(counters))
+
+
+def hsd_stage_begin(ctx, stage, kv, stream) -> int:
+    return _lib.hsd_stage_begin(ctx, C.byref(stage) if stage is not None else None,
+                                C.byref(kv) if kv is not None else None, _p(stream))
+
+
+def hsd_stage_advance(ctx, stage, kv, accept_len, emit_tokens, n_emit, emit_stride, stream) -> int:
+    return _lib.hsd_stage_advance(ctx, C.byref(stage) if stage is not None else None,
+                                  C.byref(kv) if kv is not None else None, _p(accept_len), _p(emit_tokens), _p(n_emit),
+                                  emit_stride, _p(stream))
+
+
+def hsd_stage_aggregate(ctx, stage, draft_tokens, capacity, draft_off, stream) -> int:
+    return _lib.hsd_stage_aggregate(ctx, C.byref(stage) if stage is not None else None, _p(draft_tokens), capacity,
+                                    _p(draft_off), _p(stream))
 
 
 def hsd_device_status(ctx, workspace, stream):

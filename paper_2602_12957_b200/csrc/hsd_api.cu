@@ -698,22 +698,80 @@ int hsd_verify_tree(hsd_ctx* c, const hsd_kv* kv, int n_seqs, const int* cu_q, c
 int hsd_dsv_build(hsd_ctx* c, int n_seqs, int window_n, int* window, const int* emit_tokens, const int* n_emit,
                   int emit_stride, const int* draft_tokens, int total_draft_tokens, const int* draft_off, int n_drafts,
                   const int* seq_draft_off, int max_rows, int* q_tokens, int* parent, int* cu_q, int* n_rows,
-                  void* cuda_stream) {
+                  const int* seq_map, int n_owners, void* cuda_stream) {
   if (!c || !window || !draft_tokens || !draft_off || !seq_draft_off || !q_tokens || !parent || !cu_q || !n_rows)
     return HSD_ERR_INVALID_ARG;
   if (n_seqs <= 0 || window_n <= 0 || window_n > HSD_MAX_WINDOW || max_rows <= 0) return HSD_ERR_INVALID_ARG;
   if (total_draft_tokens < 0 || n_drafts < 0) return HSD_ERR_INVALID_ARG;
   if ((emit_tokens == nullptr) != (n_emit == nullptr) || (emit_tokens && emit_stride <= 0)) return HSD_ERR_INVALID_ARG;
   if (max_rows > HSD_MAX_TREE_ROWS) return HSD_ERR_TOO_LONG;
+  if (seq_map && n_owners < 0) return HSD_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   Scope s(c, st, KC_SETUP);
   DsvArgs a;
+  a.seq_map = seq_map; a.n_owners = seq_map ? n_owners : n_seqs;
   a.n_seqs = n_seqs; a.window_n = window_n; a.max_rows = max_rows; a.emit_stride = emit_stride;
   a.window = window; a.emit_tokens = emit_tokens; a.n_emit = n_emit;
   a.draft_tokens = draft_tokens; a.draft_off = draft_off; a.seq_draft_off = seq_draft_off;
   a.total_draft_tokens = total_draft_tokens; a.n_drafts = n_drafts;
   a.q_tokens = q_tokens; a.parent = parent; a.cu_q = cu_q; a.n_rows = n_rows;
   launch_dsv_build(st, a, c->pdl);
+  return check_cuda(c);
+}
+
+namespace {
+int stage_dev(const hsd_stage* s, StageDev* d) {
+  if (!s || !s->lane_seq || !s->lane_slot || !s->window || !s->first_token || !s->max_new || !s->out_tokens ||
+      !s->out_len || !s->seq_steps || !s->seq_accepted || !s->counters)
+    return HSD_ERR_INVALID_ARG;
+  if (s->n_lanes < 1 || s->n_seqs < 1 || s->out_stride < 1 || s->window_n < 1 || s->window_n > HSD_MAX_WINDOW)
+    return HSD_ERR_INVALID_ARG;
+  d->n_lanes = s->n_lanes; d->n_seqs = s->n_seqs; d->window_n = s->window_n; d->out_stride = s->out_stride;
+  d->idle_slot = s->idle_slot;
+  d->lane_seq = s->lane_seq; d->lane_slot = s->lane_slot; d->window = s->window;
+  d->first_token = s->first_token; d->seq_slot = s->seq_slot; d->max_new = s->max_new;
+  d->out_tokens = s->out_tokens; d->out_len = s->out_len; d->seq_steps = s->seq_steps;
+  d->seq_accepted = s->seq_accepted; d->counters = s->counters;
+  return HSD_OK;
+}
+}  // namespace
+
+int hsd_stage_begin(hsd_ctx* c, const hsd_stage* stage, const hsd_kv* kv, void* cuda_stream) {
+  if (!c) return HSD_ERR_INVALID_ARG;
+  StageDev d;
+  int rc = stage_dev(stage, &d);
+  if (rc) return rc;
+  rc = check_kv(kv);
+  if (rc) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  Scope s(c, st, KC_SETUP);
+  launch_stage_begin(st, d, kv_view(kv), c->pdl);
+  return check_cuda(c);
+}
+
+int hsd_stage_advance(hsd_ctx* c, const hsd_stage* stage, const hsd_kv* kv, const int* accept_len, const int* emit_tokens,
+                      const int* n_emit, int emit_stride, void* cuda_stream) {
+  if (!c || !accept_len || !emit_tokens || !n_emit || emit_stride < 1) return HSD_ERR_INVALID_ARG;
+  StageDev d;
+  int rc = stage_dev(stage, &d);
+  if (rc) return rc;
+  rc = check_kv(kv);
+  if (rc) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  Scope s(c, st, KC_COMMIT);
+  launch_stage_advance(st, d, kv_view(kv), accept_len, emit_tokens, n_emit, emit_stride, c->pdl);
+  return check_cuda(c);
+}
+
+int hsd_stage_aggregate(hsd_ctx* c, const hsd_stage* stage, int* draft_tokens, int capacity, int* draft_off,
+                        void* cuda_stream) {
+  if (!c || !draft_tokens || !draft_off || capacity < 1) return HSD_ERR_INVALID_ARG;
+  StageDev d;
+  int rc = stage_dev(stage, &d);
+  if (rc) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  Scope s(c, st, KC_SETUP);
+  launch_stage_aggregate(st, d, draft_tokens, capacity, draft_off, c->pdl);
   return check_cuda(c);
 }
 

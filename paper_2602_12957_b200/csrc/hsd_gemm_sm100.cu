@@ -85,19 +85,33 @@ int make_weight_tmaps(WeightMaps* w, const void* base, uint64_t rows, uint64_t c
 }
 
 // ------------------------------------------------------------------------------------------------
+#ifndef HSD_GEMM_KSTEPS
+#define HSD_GEMM_KSTEPS 1
+#endif
 constexpr int BM = 128;
-constexpr int BK = 64;
-constexpr int A_BYTES = BM * BK * 2;
+constexpr int KSUB = 64;                         // one 128-byte-swizzled sub-tile spans 64 bf16 of K
+constexpr int KSTEPS = HSD_GEMM_KSTEPS;          // sub-tiles per pipeline stage
+constexpr int BK = KSUB * KSTEPS;                // K extent of one stage (one barrier round trip)
+constexpr int A_SUB = BM * KSUB * 2;             // bytes of one A sub-tile
+constexpr int A_BYTES = A_SUB * KSTEPS;
 constexpr int kGemmThreads = 256;
 constexpr int STG_BYTES = 4096;                  // one epilogue staging buffer: 32 rows x 128 bytes
 constexpr int STG_TOTAL = 4 * 2 * STG_BYTES;     // four epilogue warps, two buffers each
 
 // PAIR: two CTAs (a cluster) share one 256 x BN tile: each stages its own 128 rows of A and BN/2 rows of B.
+#ifndef HSD_GEMM_STAGES_PAIR
+#define HSD_GEMM_STAGES_PAIR (6 / KSTEPS)
+#define HSD_GEMM_STAGES_256 (4 / KSTEPS)
+#define HSD_GEMM_STAGES_128 (6 / KSTEPS)
+#define HSD_GEMM_STAGES_64 (8 / KSTEPS)
+#endif
 template <int BN, bool PAIR = false>
 struct Cfg {
-  static constexpr int B_BYTES = (PAIR ? BN / 2 : BN) * BK * 2;     // bytes of B this CTA stages per k-block
+  static constexpr int B_SUB = (PAIR ? BN / 2 : BN) * KSUB * 2;     // bytes of one B sub-tile this CTA stages
+  static constexpr int B_BYTES = B_SUB * KSTEPS;                    // bytes of B per stage
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = PAIR ? 6 : ((BN == 256) ? 4 : (BN == 128 ? 6 : 8));
+  static constexpr int STAGES = PAIR ? HSD_GEMM_STAGES_PAIR
+                                     : ((BN == 256) ? HSD_GEMM_STAGES_256 : (BN == 128 ? HSD_GEMM_STAGES_128 : HSD_GEMM_STAGES_64));
   static constexpr int TMEM_COLS = 2 * BN;
   static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STG_TOTAL + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
@@ -147,7 +161,7 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   const __grid_constant__ CUtensorMap tmC, GemmDev p) {
   using C = Cfg<BN, PAIR>;
   constexpr int OUT_N = (MODE == GS_SWIGLU) ? BN / 2 : BN;   // output columns per tile
-  constexpr int HALF_B = BN / 2 * BK * 2;                    // bytes of one weight half-tile
+  constexpr int HALF_B = BN / 2 * KSUB * 2;                  // bytes of one weight half-tile of one sub-tile
   constexpr int TILE_M = PAIR ? 2 * BM : BM;                 // rows of one work unit (both CTAs of a pair)
   const int rank = PAIR ? (int)cluster_ctarank() : 0;        // 0 = the CTA that issues the MMAs
   const int cta = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // index among the unit walkers
@@ -222,10 +236,14 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           if (!mbar_wait(empty + s, ph ^ 1u, abort_flag, p.status, 100)) goto done;
           if (PAIR) {
             if (rank == 0) mbar_expect_tx(full + s, 2 * C::STAGE_BYTES);   // A and B of both CTAs land on this barrier
-            tma_load_2d_pair(smem + s * C::STAGE_BYTES, &tmA, full + s, kb * BK, m0);
+#pragma unroll
+            for (int u = 0; u < KSTEPS; ++u)
+              tma_load_2d_pair(smem + s * C::STAGE_BYTES + u * A_SUB, &tmA, full + s, kb * BK + u * KSUB, m0);
           } else {
             mbar_expect_tx(full + s, A_BYTES);
-            tma_load_2d(smem + s * C::STAGE_BYTES, &tmA, full + s, kb * BK, m0);
+#pragma unroll
+            for (int u = 0; u < KSTEPS; ++u)
+              tma_load_2d(smem + s * C::STAGE_BYTES + u * A_SUB, &tmA, full + s, kb * BK + u * KSUB, m0);
           }
         }
       }
@@ -247,10 +265,15 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           const uint32_t ph = (kc / C::STAGES) & 1;
           if (!mbar_wait(empty + s, ph ^ 1u, abort_flag, p.status, 110 + half)) goto done;
           if (PAIR) {
-            tma_load_2d_pair(smem + s * C::STAGE_BYTES + A_BYTES, &tmB, full + s, kb * BK, row);
+#pragma unroll
+            for (int u = 0; u < KSTEPS; ++u)
+              tma_load_2d_pair(smem + s * C::STAGE_BYTES + A_BYTES + u * C::B_SUB, &tmB, full + s, kb * BK + u * KSUB, row);
           } else {
-            mbar_expect_tx(full + s, HALF_B);
-            tma_load_2d(smem + s * C::STAGE_BYTES + A_BYTES + half * HALF_B, &tmB, full + s, kb * BK, row);
+            mbar_expect_tx(full + s, HALF_B * KSTEPS);
+#pragma unroll
+            for (int u = 0; u < KSTEPS; ++u)
+              tma_load_2d(smem + s * C::STAGE_BYTES + A_BYTES + u * C::B_SUB + half * HALF_B, &tmB, full + s,
+                          kb * BK + u * KSUB, row);
           }
         }
       }
@@ -275,10 +298,14 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           const uint32_t sa = smem_u32(smem + s * C::STAGE_BYTES);
           const uint32_t sb = sa + A_BYTES;
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k) {
-            const uint32_t acc = (kb != kb0 || k != 0) ? 1u : 0u;
-            if (PAIR) umma_bf16_pair(d_tmem, umma_desc_sw128(sa + k * 32), umma_desc_sw128(sb + k * 32), idesc, acc);
-            else umma_bf16(d_tmem, umma_desc_sw128(sa + k * 32), umma_desc_sw128(sb + k * 32), idesc, acc);
+          for (int u = 0; u < KSTEPS; ++u) {
+#pragma unroll
+            for (int k = 0; k < KSUB / 16; ++k) {
+              const uint32_t acc = (kb != kb0 || u != 0 || k != 0) ? 1u : 0u;
+              const uint64_t da = umma_desc_sw128(sa + u * A_SUB + k * 32), db = umma_desc_sw128(sb + u * C::B_SUB + k * 32);
+              if (PAIR) umma_bf16_pair(d_tmem, da, db, idesc, acc);
+              else umma_bf16(d_tmem, da, db, idesc, acc);
+            }
           }
           // smem stage reusable once these MMAs have read it (in both CTAs of a pair)
           if (PAIR) umma_commit_pair(empty + s); else umma_commit(empty + s);

@@ -122,13 +122,35 @@ struct DsvArgs {
   const int* n_emit;         // [S] or nullptr
   const int* draft_tokens;
   const int* draft_off;      // [n_drafts + 1]
-  const int* seq_draft_off;  // [S + 1]
+  const int* seq_draft_off;  // [owners + 1]
+  const int* seq_map;        // [S] or nullptr: sequence i matches against the drafts of owner seq_map[i] (-1: none)
+  int n_owners;              // entries of seq_draft_off minus one (used with seq_map)
   int* q_tokens;             // [S * max_rows]
   int* parent;               // [S * max_rows]
   int* cu_q;                 // [S + 1]
   int* n_rows;               // [S]
 };
 void launch_dsv_build(cudaStream_t st, const DsvArgs& a, bool pdl);
+// Decode-loop bookkeeping between two steps of a lane batch (Sec. 3.1): append what every lane's sequence emitted,
+// retire finished sequences, hand their lanes to waiting ones.  Mirrors hsd_stage in the public header.
+struct StageDev {
+  int n_lanes, n_seqs, window_n, out_stride, idle_slot;
+  int* lane_seq;
+  int* lane_slot;
+  int* window;
+  const int* first_token;
+  const int* seq_slot;
+  const int* max_new;
+  int* out_tokens;
+  int* out_len;
+  int* seq_steps;
+  int* seq_accepted;
+  int* counters;
+};
+void launch_stage_begin(cudaStream_t st, const StageDev& sd, const KvView& kv, bool pdl);
+void launch_stage_advance(cudaStream_t st, const StageDev& sd, const KvView& kv, const int* accept_len,
+                          const int* emit_tokens, const int* n_emit, int emit_stride, bool pdl);
+void launch_stage_aggregate(cudaStream_t st, const StageDev& sd, int* draft_tokens, int capacity, int* draft_off, bool pdl);
 void launch_first_token(cudaStream_t st, const unsigned long long* row_best, int n_seqs, int* first_token,
                         const RowMeta& rm, const KvView& kv, const int* status, bool pdl);
 void launch_commit(cudaStream_t st, const KvView& kv, int n_seqs, const int* seq_slots, const int* accept_len,

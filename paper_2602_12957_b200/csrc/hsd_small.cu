@@ -632,7 +632,11 @@ __global__ void dsv_build_kernel(DsvArgs a) {
   // ---- candidates
   if (have_w) {
     // every offset is clamped to the array sizes the host passed: a malformed table shortens or drops drafts
-    const int d_lo = min(max(a.seq_draft_off[s], 0), a.n_drafts), d_hi = min(max(a.seq_draft_off[s + 1], 0), a.n_drafts);
+    // whose drafts: the sequence's own, or (lane batches) those of the owner the map names; -1 or out of range = none
+    const int owner = a.seq_map ? a.seq_map[s] : s;
+    const bool owned = a.seq_map ? (owner >= 0 && owner < a.n_owners) : true;
+    const int d_lo = owned ? min(max(a.seq_draft_off[owner], 0), a.n_drafts) : 0;
+    const int d_hi = owned ? min(max(a.seq_draft_off[owner + 1], 0), a.n_drafts) : 0;
     for (int d = d_lo; d < d_hi; ++d) {
       const int d0 = min(max(a.draft_off[d], 0), a.total_draft_tokens);
       const int len = min(max(a.draft_off[d + 1], d0), a.total_draft_tokens) - d0;
@@ -712,6 +716,118 @@ __global__ void dsv_build_kernel(DsvArgs a) {
 }
 void launch_dsv_build(cudaStream_t st, const DsvArgs& a, bool pdl) {
   launch_kernel(dsv_build_kernel, dim3(a.n_seqs), dim3(128), 0, st, pdl, a);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Lane batches (Sec. 3.1, Stage 1: many regions, each decoded to its end by repeated steps).  A lane serves one
+// sequence at a time; between two steps one CTA appends what every lane's sequence emitted, counts the step, retires
+// the sequences that have reached their length and hands free lanes to waiting sequences in queue order.
+// counters: [0] next waiting sequence, [1] sequences not finished, [2] steps taken.
+__device__ void stage_assign_lanes(const StageDev& sd, const KvView& kv) {      // one thread, lanes in order
+  int head = sd.counters[0], left = sd.counters[1];
+  for (int i = 0; i < sd.n_lanes; ++i) {
+    const int r = sd.lane_seq[i];
+    if (r >= 0 && sd.out_len[r] < sd.max_new[r]) continue;                      // still decoding
+    if (r >= 0) --left;                                                         // finished in this step
+    int nxt = -1;
+    while (head < sd.n_seqs && nxt < 0) {
+      if (sd.out_len[head] < sd.max_new[head]) nxt = head; else --left;         // (a sequence of length <= 1 is done at once)
+      ++head;
+    }
+    sd.lane_seq[i] = nxt;
+    const int slot = nxt < 0 ? sd.idle_slot : (sd.seq_slot ? sd.seq_slot[nxt] : nxt);
+    sd.lane_slot[i] = slot;
+    for (int k = 0; k < sd.window_n; ++k) sd.window[i * sd.window_n + k] = -1;
+    sd.window[i * sd.window_n + sd.window_n - 1] = nxt < 0 ? 0 : sd.first_token[nxt];
+  }
+  sd.counters[0] = head;
+  sd.counters[1] = left;
+  if (sd.idle_slot >= 0 && sd.idle_slot < kv.n_slots) kv.seq_lens[sd.idle_slot] = 0;   // idle lanes restart from an empty cache
+}
+
+__global__ void stage_begin_kernel(StageDev sd, KvView kv) {
+  pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
+  pdl_launch_dependents();
+  for (int r = threadIdx.x; r < sd.n_seqs; r += blockDim.x) {
+    sd.out_tokens[(size_t)r * sd.out_stride] = sd.first_token[r];
+    sd.out_len[r] = 1;
+    sd.seq_steps[r] = 0;
+    sd.seq_accepted[r] = 0;
+  }
+  for (int i = threadIdx.x; i < sd.n_lanes; i += blockDim.x) sd.lane_seq[i] = -1;
+  if (threadIdx.x == 0) {
+    sd.counters[0] = 0;
+    sd.counters[1] = sd.n_seqs;
+    sd.counters[2] = 0;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) stage_assign_lanes(sd, kv);
+}
+void launch_stage_begin(cudaStream_t st, const StageDev& sd, const KvView& kv, bool pdl) {
+  launch_kernel(stage_begin_kernel, dim3(1), dim3(128), 0, st, pdl, sd, kv);
+}
+
+__global__ void stage_advance_kernel(StageDev sd, KvView kv, const int* accept_len, const int* emit_tokens,
+                                     const int* n_emit, int emit_stride) {
+  pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
+  pdl_launch_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+  for (int i = warp; i < sd.n_lanes; i += n_warps) {       // one warp per lane
+    const int r = sd.lane_seq[i];
+    if (r < 0 || r >= sd.n_seqs) continue;
+    const int a = accept_len[i];
+    if (a < 0) continue;                                   // the step failed a device-side check: nothing was decided
+    const int have = sd.out_len[r];
+    const int room = max(0, min(sd.max_new[r], sd.out_stride) - have);
+    const int take = min(max(n_emit[i], 0), room);
+    for (int k = lane; k < take; k += 32) sd.out_tokens[(size_t)r * sd.out_stride + have + k] = emit_tokens[(size_t)i * emit_stride + k];
+    __syncwarp();
+    if (lane == 0) {
+      sd.out_len[r] = have + take;
+      sd.seq_steps[r] += 1;
+      sd.seq_accepted[r] += min(a, room);
+      // the window keeps the most recent accepted tokens, the pending one last
+      const int n = sd.window_n;
+      for (int k = 0; k < n; ++k) {
+        const int back = n - 1 - k;                        // token `back` places before the newest
+        const int idx = have + take - 1 - back;
+        sd.window[i * n + k] = idx >= 0 ? sd.out_tokens[(size_t)r * sd.out_stride + idx] : -1;
+      }
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    sd.counters[2] += 1;
+    stage_assign_lanes(sd, kv);
+  }
+}
+void launch_stage_advance(cudaStream_t st, const StageDev& sd, const KvView& kv, const int* accept_len,
+                          const int* emit_tokens, const int* n_emit, int emit_stride, bool pdl) {
+  launch_kernel(stage_advance_kernel, dim3(1), dim3(256), 0, st, pdl, sd, kv, accept_len, emit_tokens, n_emit, emit_stride);
+}
+
+// The page draft of Stage 2 (Eq. 3): the outputs of all sequences, concatenated, with their offsets.
+__global__ void stage_aggregate_kernel(StageDev sd, int* draft_tokens, int capacity, int* draft_off) {
+  pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
+  pdl_launch_dependents();
+  __shared__ int s_off;
+  if (threadIdx.x == 0) {
+    int off = 0;
+    for (int r = 0; r < sd.n_seqs; ++r) {                  // serial scan: a page has tens of regions
+      draft_off[r] = off;
+      off = min(capacity, off + max(0, min(sd.out_len[r], sd.out_stride)));
+    }
+    draft_off[sd.n_seqs] = off;
+    s_off = off;
+  }
+  __syncthreads();
+  for (int r = 0; r < sd.n_seqs; ++r) {
+    const int lo = draft_off[r], n = draft_off[r + 1] - lo;
+    for (int k = threadIdx.x; k < n; k += blockDim.x) draft_tokens[lo + k] = sd.out_tokens[(size_t)r * sd.out_stride + k];
+  }
+}
+void launch_stage_aggregate(cudaStream_t st, const StageDev& sd, int* draft_tokens, int capacity, int* draft_off, bool pdl) {
+  launch_kernel(stage_aggregate_kernel, dim3(1), dim3(256), 0, st, pdl, sd, draft_tokens, capacity, draft_off);
 }
 
 // Prefill epilogue: first pending token per sequence, and seq_lens += rows.

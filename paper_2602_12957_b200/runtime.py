@@ -39,6 +39,17 @@ class DeviceModel:
         st, self.ctx = B.hsd_create(self._cfg_c, self._w_c)
         B.check(st, "hsd_create")
 
+    def sibling(self, flags: int) -> "DeviceModel":
+        """A second library context with other HSD_FLAG_* bits over the SAME device weights (nothing is copied)."""
+        other = object.__new__(DeviceModel)
+        other.cfg, other.device = self.cfg, self.device
+        other.embed, other.lm_head, other.final_norm, other.layers = self.embed, self.lm_head, self.final_norm, self.layers
+        other._cfg_c = B.make_config(self.cfg, flags)
+        other._w_c = self._w_c
+        st, other.ctx = B.hsd_create(other._cfg_c, other._w_c)
+        B.check(st, "hsd_create")
+        return other
+
     def close(self):
         if getattr(self, "ctx", None) is not None:
             B.hsd_destroy(self.ctx)
@@ -158,8 +169,10 @@ class Engine:
 
     def dsv_build(self, window: torch.Tensor, draft_tokens: torch.Tensor, draft_off: torch.Tensor,
                   seq_draft_off: torch.Tensor, max_rows: int, emit_tokens: Optional[torch.Tensor] = None,
-                  n_emit: Optional[torch.Tensor] = None, out: Optional[dict] = None):
-        """Matching + prefix-tree packing on the device; `window` [S, n] is updated in place."""
+                  n_emit: Optional[torch.Tensor] = None, out: Optional[dict] = None,
+                  seq_map: Optional[torch.Tensor] = None):
+        """Matching + prefix-tree packing on the device; `window` [S, n] is updated in place.  With `seq_map` [S]
+        sequence i uses the drafts of owner seq_map[i] of `seq_draft_off` (lane batches)."""
         S, n = int(window.shape[0]), int(window.shape[1])
         if out is None:
             i32 = lambda *s: torch.empty(*s, dtype=torch.int32, device=self.dev)
@@ -167,7 +180,8 @@ class Engine:
         st = B.hsd_dsv_build(self.model.ctx, S, n, window, emit_tokens, n_emit,
                              int(emit_tokens.shape[1]) if emit_tokens is not None else 0, draft_tokens,
                              int(draft_tokens.numel()), draft_off, int(draft_off.numel()) - 1, seq_draft_off, max_rows,
-                             out["q_tokens"], out["parent"], out["cu_q"], out["n_rows"], _stream())
+                             out["q_tokens"], out["parent"], out["cu_q"], out["n_rows"], _stream(), seq_map,
+                             int(seq_draft_off.numel()) - 1)
         B.check(st, "hsd_dsv_build")
         return out
 

@@ -1,0 +1,133 @@
+"""The two-stage decode loop on the device (paper Sec. 3.1, Eq. 1-4): lane batches with retirement and hand-over,
+aggregation of the Stage-1 outputs into the page draft, Stage 2.
+
+Two independent checks.  (1) Against the library itself: with tau = 1 speculation is lossless, so on a context with a
+fixed summation order the loop's outputs must equal, token for token, what plain one-token decoding through the same
+library gives — whatever the drafts, the lane count or the graph batching; this exercises matching, packing, tree
+verification, compaction, commit, bookkeeping and lane hand-over end to end with no tolerance.  (2) Against the oracle
+loop: same inputs, same drafts; outputs must agree up to the first token whose decision was a near tie in the oracle
+(top-1 / top-2 gap <= 0.1), the per-sequence step counts likewise when no decision was a near tie."""
+import numpy as np
+import pytest
+
+from oracle import hsd_oracle as O
+from oracle import two_stage_oracle as T
+from paper_2602_12957_b200 import inputs as I
+
+from . import harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _library_greedy(model, prefixes, lengths, seed):
+    """Plain one-token decoding through the library: the text every lossless loop must reproduce."""
+    import torch
+    from paper_2602_12957_b200 import runtime as R
+    S = len(prefixes)
+    kv = R.KvCache(model, [len(ids) + n + 2 for (_, ids), n in zip(prefixes, lengths)], seed=seed)
+    eng = R.Engine(model, kv, max(sum(len(ids) for _, ids in prefixes), S), S)
+    first = eng.prefill([e for e, _ in prefixes], [i for _, i in prefixes])
+    cu1 = eng._i32(np.arange(S + 1))
+    out1 = eng.alloc_outputs(S, 1, S)
+    pending, hist = first.clone(), [first.clone()]
+    for _ in range(max(lengths) - 1):
+        eng.verify_regions(pending, cu1, 1, S, out=out1)
+        eng.commit(out1["accept_len"])
+        pending = out1["emit_tokens"][:, 0].clone()
+        hist.append(pending)
+    eng.check_device("greedy")
+    text = torch.stack(hist, 1).cpu().numpy()
+    return [text[i, :lengths[i]].copy() for i in range(S)]
+
+
+def _damaged(text, rng, n_err, vocab):
+    d = np.asarray(text, np.int64).copy()
+    for pos in rng.choice(np.arange(3, len(d)), size=min(n_err, len(d) - 3), replace=False):
+        d[pos] = (d[pos] + 1 + int(rng.integers(0, vocab - 1))) % vocab
+    return d.astype(np.int32)
+
+
+def _setup(seed=41, n_regions=5):
+    cfg = I.small_decoder(2, 8192)
+    wl = I.region_workload(seed=seed, n_regions=n_regions + 1, prefix_lo=70, prefix_hi=200, draft_mean=30, draft_lo=8,
+                           draft_hi=60, cfg=cfg)
+    weights = I.make_weights(cfg, seed)
+    prefixes = [(s.prefix_embeds, s.prefix_ids) for s in wl.seqs]
+    rng = np.random.default_rng(seed)
+    lengths = [int(x) for x in rng.integers(24, 70, size=n_regions)] + [90]       # regions, then the page
+    return cfg, weights, prefixes, lengths, rng
+
+
+@pytest.mark.parametrize("n_lanes,steps_per_poll,use_graph", [(2, 3, True), (5, 1, False), (8, 4, True)])
+def test_device_loop_is_lossless_and_hands_lanes_over(n_lanes, steps_per_poll, use_graph):
+    from paper_2602_12957_b200 import binding as B
+    from paper_2602_12957_b200 import driver as DR
+    from paper_2602_12957_b200 import runtime as R
+    cfg, weights, prefixes, lengths, rng = _setup()
+    model = R.DeviceModel(cfg, weights, B.HSD_FLAG_DETERMINISTIC)
+    text = _library_greedy(model, prefixes, lengths, seed=1)
+    regions, page = prefixes[:-1], prefixes[-1]
+    # the pipeline's drafts: two damaged copies of every region's text (one region gets garbage, one gets none)
+    drafts = [[_damaged(t, rng, 3, cfg.vocab), _damaged(t, rng, 5, cfg.vocab)] for t in text[:-1]]
+    drafts[1] = [rng.integers(0, cfg.vocab, 50).astype(np.int32)]
+    drafts[2] = []
+    run = DR.run_page(model, regions, drafts, lengths[:-1], page, lengths[-1], n_lanes=n_lanes, max_rows=32,
+                      steps_per_poll=steps_per_poll, use_graph=use_graph, seed=3, poison=True)
+    for r in range(len(regions)):
+        assert run.stage1.tokens[r].tolist() == text[r].tolist(), f"region {r}"
+        assert run.page_draft[r].tolist() == text[r].tolist()                       # Eq. 3: the outputs, as they are
+    assert run.stage2.tokens[0].tolist() == text[-1].tolist()
+    s1 = run.stage1
+    assert s1.steps[1] == lengths[1] - 1 and s1.steps[2] == lengths[2] - 1          # garbage / no drafts: plain decoding
+    assert s1.accepted[1] == 0 and s1.accepted[2] == 0
+    for r in (0, 3, 4):                                                             # good drafts: several tokens per step
+        assert s1.steps[r] < (lengths[r] - 1) * 0.6
+        assert s1.accepted[r] + s1.steps[r] >= lengths[r] - 1                       # every step emits accepted + 1
+    # lanes fewer than regions: the batch needs more steps than its slowest region, but far fewer than the sum
+    assert s1.batch_steps >= int(s1.steps.max())
+    if n_lanes < len(regions):
+        assert s1.batch_steps < int(s1.steps.sum())
+    print("two-stage", n_lanes, "stage1 steps", s1.steps.tolist(), "AAL", round(s1.aal, 2), "batch steps", s1.batch_steps,
+          "stage2 steps", run.stage2.steps.tolist(), "ms", round(s1.ms, 2), round(run.stage2.ms, 2))
+
+
+@pytest.mark.parametrize("log_tau", [0.0, float(np.log(0.75))], ids=["greedy", "tau0.75"])
+def test_device_loop_follows_the_oracle_loop(log_tau):
+    from paper_2602_12957_b200 import driver as DR
+    from paper_2602_12957_b200 import runtime as R
+    cfg, weights, prefixes, lengths, rng = _setup(seed=43, n_regions=4)
+    model_o = O.Decoder(cfg, weights, np.float64)
+    # drafts from the ORACLE's greedy text, so that the oracle loop accepts long runs
+    regions_o = []
+    for (emb, ids), n in zip(prefixes[:-1], lengths[:-1]):
+        seq = O.CachedSequence(model_o)
+        first = seq.prefill(emb, ids)
+        text = [first] + O.greedy_continuation(seq, first, n - 1)
+        regions_o.append(T.RegionInput(emb, ids, [_damaged(text, rng, 3, cfg.vocab).tolist(),
+                                                  _damaged(text, rng, 4, cfg.vocab).tolist()], n))
+    page_o = T.RegionInput(prefixes[-1][0], prefixes[-1][1], [], lengths[-1])
+    want = T.hierarchical_decode(model_o, regions_o, page_o, n=3, max_rows=32, log_tau=log_tau)
+    model = R.DeviceModel(cfg, weights, 0)
+    run = DR.run_page(model, prefixes[:-1], [[np.asarray(d, np.int32) for d in r.drafts] for r in regions_o],
+                      lengths[:-1], prefixes[-1], lengths[-1], n_lanes=3, max_rows=32, log_tau=log_tau, seed=5,
+                      poison=True)
+    checked = 0
+    for r, tr in enumerate(want.region_traces):
+        gaps = np.asarray(tr.token_gap)
+        clear = int(np.argmax(gaps <= H.GAP_EXACT)) if np.any(gaps <= H.GAP_EXACT) else len(gaps)
+        got = run.stage1.tokens[r].tolist()
+        assert len(got) == lengths[r]
+        if log_tau == 0.0:
+            assert got[:clear] == tr.tokens[:clear], f"region {r}: differs before the first near tie at {clear}"
+            checked += clear
+            if clear == len(gaps):
+                assert run.stage1.steps[r] == tr.steps and run.stage1.accepted[r] == sum(tr.accepted_per_step)
+    if log_tau == 0.0:
+        assert checked > 40, "the case must pin a fair number of tokens"
+    else:
+        # with a threshold the accepted text may leave the greedy path; the loop must still fill every output and
+        # never take more steps than plain decoding
+        assert all(run.stage1.steps[r] <= lengths[r] - 1 for r in range(len(lengths) - 1))
+    assert len(run.stage2.tokens[0]) == lengths[-1]
+    print("oracle loop", log_tau, want.summary(), "device stage1 steps", run.stage1.steps.tolist(), "AAL",
+          round(run.stage1.aal, 2), "checked tokens", checked)
