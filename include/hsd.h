@@ -118,7 +118,8 @@ HSD_API const char *hsd_status_string(int status);
 
 /* Create a context for one model on the current device.  Copies the configuration and the weight POINTERS
  * (not the weights) and builds the TMA tensor maps of the weights.  Errors: INVALID_ARG, SHAPE (requires
- * head_dim == 64, kv_block == 64, n_heads a multiple of n_kv_heads, d_model, d_ffn, vocab multiples of 64),
+ * head_dim == 64, kv_block == 64, n_heads a multiple of n_kv_heads with a ratio that divides 128, d_model one of
+ * 128, 256, 512, 1024, 2048, 4096, d_ffn and vocab multiples of 64),
  * NO_DEVICE, CUDA.  No stream work is issued. */
 HSD_API int hsd_create(const hsd_model_config *cfg, const hsd_weights *w, hsd_ctx **out);
 HSD_API int hsd_destroy(hsd_ctx *ctx);

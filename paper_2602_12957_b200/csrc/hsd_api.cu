@@ -505,7 +505,7 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
   const int group = cfg->n_heads / cfg->n_kv_heads;
   if (128 % group) return HSD_ERR_SHAPE;
   const int dv = cfg->d_model / 128;
-  if (cfg->d_model % 128 || !(dv == 1 || dv == 2 || dv == 4 || dv == 8 || dv == 16)) return HSD_ERR_SHAPE;
+  if (cfg->d_model % 128 || !(dv == 1 || dv == 2 || dv == 4 || dv == 8 || dv == 16 || dv == 32)) return HSD_ERR_SHAPE;
   if (cfg->d_ffn % 64 || cfg->vocab % 64) return HSD_ERR_SHAPE;
   if (!w->embed || !w->lm_head || !w->final_norm || !w->attn_norm || !w->w_qkv || !w->w_o || !w->ffn_norm ||
       !w->w_gate_up || !w->w_down)

@@ -176,7 +176,7 @@ void launch_embed(cudaStream_t st, const RowMeta& rm, const bf16* table, const b
 
 // ------------------------------------------------------------------------------------------------
 // RMSNorm: h = bf16(x * rsqrt(mean(x^2) + eps) * gain).  One warp per row; the row stays in registers
-// between the reduction and the scaling (d <= 2048), so x is read once.
+// between the reduction and the scaling (d <= 4096), so x is read once.
 template <int VEC>   // VEC float4 per lane: d = 128 * VEC
 __global__ void rmsnorm_kernel(const float* __restrict__ x, const bf16* __restrict__ gain, bf16* __restrict__ h,
                                int rows, int d, float eps, const int* __restrict__ sel_rows, int src_rows,
@@ -219,7 +219,7 @@ void launch_rmsnorm(cudaStream_t st, const float* x, const bf16* gain, bf16* h, 
 #define HSD_RMS_CASE(V) \
   case V: launch_kernel(rmsnorm_kernel<V>, grid, block, 0, st, pdl, x, gain, h, rows, d, eps, sel_rows, src_rows, status); break;
   switch (d / 128) {
-    HSD_RMS_CASE(1) HSD_RMS_CASE(2) HSD_RMS_CASE(4) HSD_RMS_CASE(8) HSD_RMS_CASE(16)
+    HSD_RMS_CASE(1) HSD_RMS_CASE(2) HSD_RMS_CASE(4) HSD_RMS_CASE(8) HSD_RMS_CASE(16) HSD_RMS_CASE(32)
     default: break;   // hsd_create rejects other widths
   }
 #undef HSD_RMS_CASE

@@ -123,9 +123,12 @@ class PageRun:
 
 def run_page(model: R.DeviceModel, regions, region_drafts, region_max_new, page, page_max_new, n_lanes: int = 16,
              window_n: int = 3, max_rows: int = 128, log_tau: float = 0.0, steps_per_poll: int = 8,
-             use_graph: bool = True, seed: int = 0, poison: bool = False) -> PageRun:
+             use_graph: bool = True, seed: int = 0, poison: bool = False,
+             stage2_draft: Optional[Sequence[np.ndarray]] = None) -> PageRun:
     """The whole hierarchy for one page.  regions / page: (prefix_embeds [L, d] or None, prefix_ids [L]) pairs;
-    region_drafts[i]: list of int arrays (the pipeline's drafts of region i); *_max_new: output lengths."""
+    region_drafts[i]: list of int arrays (the pipeline's drafts of region i); *_max_new: output lengths.
+    `stage2_draft` (benchmarks with synthetic decoders only): drafts Stage 2 matches against INSTEAD of the aggregated
+    Stage-1 outputs, which are still assembled and returned."""
     dev = model.device
     stream = torch.cuda.current_stream()
     n_reg = len(regions)
@@ -162,7 +165,14 @@ def run_page(model: R.DeviceModel, regions, region_drafts, region_max_new, page,
     ev[2].record(stream)
     B.check(B.hsd_stage_aggregate(model.ctx, lb1.stage, page_draft, cap, page_off, _stream()), "hsd_stage_aggregate")
     ev[3].record(stream)
-    lb2 = LaneBatch(eng2, first2, [page_max_new], page_draft, page_off, i32([0, n_reg]), 1, window_n, max_rows, log_tau)
+    d2_tok, d2_off, d2_n = page_draft, page_off, n_reg
+    if stage2_draft is not None:
+        flat, offs = [], [0]
+        for d in stage2_draft:
+            flat.extend(int(t) for t in d)
+            offs.append(len(flat))
+        d2_tok, d2_off, d2_n = i32(flat if flat else [0]), i32(offs), len(stage2_draft)
+    lb2 = LaneBatch(eng2, first2, [page_max_new], d2_tok, d2_off, i32([0, d2_n]), 1, window_n, max_rows, log_tau)
     lb2.remember_lengths()
     s2 = lb2.run(steps_per_poll, use_graph)
     stream.synchronize()

@@ -5,8 +5,8 @@ Two independent checks.  (1) Against the library itself: with tau = 1 speculatio
 fixed summation order the loop's outputs must equal, token for token, what plain one-token decoding through the same
 library gives — whatever the drafts, the lane count or the graph batching; this exercises matching, packing, tree
 verification, compaction, commit, bookkeeping and lane hand-over end to end with no tolerance.  (2) Against the oracle
-loop: same inputs, same drafts; outputs must agree up to the first token whose decision was a near tie in the oracle
-(top-1 / top-2 gap <= 0.1), the per-sequence step counts likewise when no decision was a near tie."""
+loop: same inputs, same drafts; the two outputs may part only at a token the oracle chose by a near tie (top-1 / top-2
+gap <= 0.1), and where they never part the per-sequence step counts and accepted totals are equal too."""
 import numpy as np
 import pytest
 
@@ -24,7 +24,7 @@ def _library_greedy(model, prefixes, lengths, seed):
     import torch
     from paper_2602_12957_b200 import runtime as R
     S = len(prefixes)
-    kv = R.KvCache(model, [len(ids) + n + 2 for (_, ids), n in zip(prefixes, lengths)], seed=seed)
+    kv = R.KvCache(model, [len(ids) + max(lengths) + 2 for _, ids in prefixes], seed=seed)    # all step together
     eng = R.Engine(model, kv, max(sum(len(ids) for _, ids in prefixes), S), S)
     first = eng.prefill([e for e, _ in prefixes], [i for _, i in prefixes])
     cu1 = eng._i32(np.arange(S + 1))
@@ -114,16 +114,21 @@ def test_device_loop_follows_the_oracle_loop(log_tau):
     checked = 0
     for r, tr in enumerate(want.region_traces):
         gaps = np.asarray(tr.token_gap)
-        clear = int(np.argmax(gaps <= H.GAP_EXACT)) if np.any(gaps <= H.GAP_EXACT) else len(gaps)
         got = run.stage1.tokens[r].tolist()
         assert len(got) == lengths[r]
         if log_tau == 0.0:
-            assert got[:clear] == tr.tokens[:clear], f"region {r}: differs before the first near tie at {clear}"
-            checked += clear
-            if clear == len(gaps):
+            # the two texts may part only at a token the oracle chose by a near tie (gap <= 0.1); after that token they are
+            # different texts and nothing more can be compared
+            same = [a == b for a, b in zip(got, tr.tokens)]
+            first_diff = same.index(False) if False in same else len(same)
+            if first_diff < len(same):
+                assert gaps[first_diff] <= H.GAP_EXACT, (f"region {r}: token {first_diff} differs although the oracle's "
+                                                         f"choice was clear (gap {gaps[first_diff]:.3f})")
+            checked += first_diff
+            if first_diff == len(same):
                 assert run.stage1.steps[r] == tr.steps and run.stage1.accepted[r] == sum(tr.accepted_per_step)
     if log_tau == 0.0:
-        assert checked > 40, "the case must pin a fair number of tokens"
+        assert checked > 60, "the case must pin a fair number of tokens"
     else:
         # with a threshold the accepted text may leave the greedy path; the loop must still fill every output and
         # never take more steps than plain decoding

@@ -258,3 +258,15 @@ def test_layer_tap_returns_each_layers_residual_stream():
             got = taps[n_layers - 1][cu[i]:cu[i + 1]]
             err = np.abs(got - ref).max() / np.abs(ref).max()
             assert err < 2e-2, (n_layers, i, err)
+
+
+def test_wide_decoder_with_four_query_heads_per_kv_head_matches_oracle():
+    """A wider decoder shape than the benchmark's (d_model 4096, 32 query / 8 kv heads x 64, FFN 8192: the width class of
+    the 7-9 B parsers the paper evaluates, Sec. 4.3), one layer: 4096-wide RMSNorm rows, K = 4096 / 8192 projections,
+    q-tiles of 32 tokens x 4 heads."""
+    cfg = I.ModelConfig(n_layers=1, d_model=4096, n_heads=32, n_kv_heads=8, head_dim=64, d_ffn=8192, vocab=4096)
+    wl = I.region_workload(seed=81, n_regions=3, prefix_lo=70, prefix_hi=200, draft_mean=40, draft_lo=8, draft_hi=100,
+                           cfg=cfg, name="wide_regions")
+    stats, orc, per, _ = run_region_parity(wl, 0)
+    print("wide", stats, [(len(o.draft), o.res.accept_len) for o in orc.values()])
+    assert stats["max_dz"] < H.LOGIT_TOL
