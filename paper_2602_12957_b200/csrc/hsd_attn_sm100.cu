@@ -15,10 +15,16 @@
 //
 // Persistent CTAs, two per SM, walk the item list.  Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer +
 // TMEM owner, warps 2..5 = softmax (one TMEM lane quarter each, one thread per q row, no shuffles).
-// Per KV tile: S = Q K^T (TMEM) -> online softmax in registers -> P (bf16, shared memory, 128B-swizzled) ->
-// PV = P V (TMEM) -> accumulated into registers with the running-max rescale.  S, P and PV are double-buffered
-// so the tensor pipe works on tile j+1 while the softmax warps are on tile j; two CTAs per SM interleave
-// further.  Every wait is a bounded mbarrier wait, so one that gives up takes the whole CTA to the common exit.
+// Per KV tile: S = Q K^T (TMEM) -> softmax in registers -> P (bf16, shared memory, 128B-swizzled) -> O += P V,
+// accumulated IN TENSOR MEMORY.  S and P are double-buffered, so the tensor pipe works on tile j+1 while the softmax
+// warps are on tile j, and a softmax warp never waits for a product younger than the one two tiles back: measured with
+// every arithmetic instruction removed, a loop in which each tile waits for the product of the tile before it still
+// took four fifths of the kernel's time (two barrier hand-overs per tile on the critical path); with the accumulator
+// in tensor memory nothing in the steady state waits on a hand-over at all.  The exponent reference of a row is not
+// its running maximum but a value that is raised only when the maximum has grown by more than kRescaleBits binary
+// orders since it was set (P stays below 2^kRescaleBits, far inside bf16 and fp32 range): then, and only then, the
+// row's accumulator is read, scaled and written back.  After the first tiles of a row that is rare.  Two CTAs per SM
+// interleave further.  Every wait is a bounded mbarrier wait, so one that gives up takes the whole CTA to the common exit.
 #include "hsd_kernels.h"
 
 namespace hsd {
@@ -29,7 +35,8 @@ constexpr int Q_BYTES = 128 * 128;
 constexpr int KV_TILE_BYTES = 64 * 128;            // one K tile or one V tile
 constexpr int P_BYTES = 128 * 128;
 constexpr int ATTN_SMEM = Q_BYTES + KV_STAGES * 2 * KV_TILE_BYTES + 2 * P_BYTES + 1024 + 256;
-constexpr int ATTN_TMEM_COLS = 256;                // S0 S1 PV0 PV1, 64 fp32 columns each
+constexpr int ATTN_TMEM_COLS = 256;                // S0 S1 (64 fp32 columns each), O (64), 64 unused (allocations are powers of two)
+constexpr float kRescaleBits = 8.f;
 
 struct AttnParams {
   AttnPlan plan;
@@ -176,7 +183,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   uint64_t* s_full = kv_empty + KV_STAGES;
   uint64_t* s_empty = s_full + 2;
   uint64_t* p_full = s_empty + 2;
-  uint64_t* pv_full = p_full + 2;
+  uint64_t* pv_full = p_full + 2;          // [g & 1] O += P(g) V(g) has completed
   uint64_t* group_bar = pv_full + 2;       // the four softmax warps (slice hand-over)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(group_bar + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -299,16 +306,17 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             if (!issue_s(g + 1)) goto done;
             if (j + 2 == n_it) umma_commit(q_empty);      // last S MMA of the item issued: Q is free once it completes
           }
-          // P(g) is written; the softmax warps have also folded PV(g-2) out of the buffer PV(g) is about to overwrite
+          // P(g) is written, and whatever had to be done to the accumulator before this product is done
           if (!mbar_wait(p_full + (g & 1), (g >> 1) & 1, abort_flag, p.status, 413)) goto done;
           tc_fence_after();
           const int st = g % KV_STAGES;
           const uint32_t p_addr = smem_u32(sP + (g & 1) * P_BYTES);
           const uint32_t v_addr = smem_u32(sKV + st * 2 * KV_TILE_BYTES + KV_TILE_BYTES);
-          const uint32_t d = tmem_base + 128 + (g & 1) * 64;
+          const uint32_t d = tmem_base + 128;      // the item's accumulator: the first product of an item overwrites it
 #pragma unroll
           for (int k = 0; k < 4; ++k)   // V [key][dim] is MN-major: a K step of 16 keys is 16 rows of 128 bytes
-            umma_bf16(d, umma_desc_sw128(p_addr + k * 32), umma_desc_sw128(v_addr + k * 2048), idesc_pv, k != 0);
+            umma_bf16(d, umma_desc_sw128(p_addr + k * 32), umma_desc_sw128(v_addr + k * 2048), idesc_pv,
+                      (j != 0 || k != 0) ? 1u : 0u);
           umma_commit(kv_empty + st);
           umma_commit(pv_full + (g & 1));
         }
@@ -343,29 +351,8 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       // they keep step with the barriers but skip the loads, the exps and the P rows (which only feed their own,
       // never stored, output rows)
       const bool warp_ok = (quarter * 32) / p.group < n_tok;
-      float m = -INFINITY, l = 0.f, alpha_prev = 1.f;
-      float o[64];
-#pragma unroll
-      for (int e = 0; e < 64; ++e) o[e] = 0.f;
-
-      // fold PV(gi) into the row accumulator; the rescale for what was accumulated before it is alpha_prev
-      auto fold_pv = [&](uint32_t gi, int where) -> bool {
-        const int pb = gi & 1;
-        bool ok = mbar_wait(pv_full + pb, (gi >> 1) & 1, abort_flag, p.status, where);
-        if (!__all_sync(0xffffffffu, ok)) return false;
-        tc_fence_after();
-        uint32_t t0[32], t1[32];
-        tmem_ld32(t_lane + 128 + pb * 64, t0);
-        tmem_ld32(t_lane + 128 + pb * 64 + 32, t1);
-        tmem_ld_wait();
-        tc_fence_before();
-#pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          o[e] = o[e] * alpha_prev + __uint_as_float(t0[e]);
-          o[32 + e] = o[32 + e] * alpha_prev + __uint_as_float(t1[e]);
-        }
-        return true;
-      };
+      float m_ref = -INFINITY, l = 0.f;                  // exponent reference (log2 units, scaled) and row sum under it
+      const uint32_t t_o = t_lane + 128;                 // this warp's lanes of the accumulator
 
       for (int j = kt_lo; j < kt_hi; ++j, ++g) {
         const int b = g & 1;
@@ -418,9 +405,21 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         float mx = -INFINITY;
 #pragma unroll
         for (int e = 0; e < 32; ++e) mx = max3(mx, __uint_as_float(s0[e]), __uint_as_float(s1[e]));
-        const float m_new = fmaxf(m, mx * sc);
-        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-        const float alpha = ex2(m - m_use);
+        mx *= sc;
+        // The reference moves only when the maximum has outgrown it by more than kRescaleBits (or nothing has been
+        // accumulated under it yet: then moving it costs nothing).
+        float alpha = 1.f;
+        bool rescale = false;
+        if (mx > m_ref) {
+          if (l == 0.f) {
+            m_ref = mx;                                   // nothing accumulated so far (first tile, or all keys masked)
+          } else if (mx > m_ref + kRescaleBits) {
+            alpha = ex2(m_ref - mx);
+            m_ref = mx;
+            rescale = true;
+          }
+        }
+        const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
         float sum = 0.f;
         uint32_t pk[32];
 #pragma unroll
@@ -438,6 +437,29 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           pk[16 + e] = pack_bf16(a0, a1);
         }
         l = l * alpha + sum;
+        // P's buffer was last read by the product of tile g - 2: the only wait of the steady state, two tiles back
+        if (g >= 2) {
+          ok = mbar_wait(pv_full + b, ((g - 2) >> 1) & 1, abort_flag, p.status, 421);
+          if (!__all_sync(0xffffffffu, ok)) goto done;
+        }
+        if (__any_sync(0xffffffffu, rescale)) {
+          // rare: scale this warp's accumulator rows (alpha = 1 where not needed) once the product before this tile,
+          // which still adds into them, has completed
+          ok = mbar_wait(pv_full + (b ^ 1), ((g - 1) >> 1) & 1, abort_flag, p.status, 423);
+          if (!__all_sync(0xffffffffu, ok)) goto done;
+          tc_fence_after();
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {
+            uint32_t o[32];
+            tmem_ld32(t_o + hf * 32, o);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st32(t_o + hf * 32, o);
+          }
+          tmem_st_wait();
+          tc_fence_before();
+        }
         // P row -> shared memory, K-major 128B-swizzled: 16-byte chunk c of row r sits at chunk c ^ (r & 7)
         uint8_t* prow = sP + b * P_BYTES + row * 128;
 #pragma unroll
@@ -446,34 +468,54 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
               make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
         fence_proxy_async_smem();
         mbar_arrive(p_full + b);
-        m = m_new;
-        // the rescale for everything accumulated so far is applied when PV(g-1) is folded in
-        if (j > kt_lo && !fold_pv(g - 1, 421)) goto done;
-        alpha_prev = alpha;
       }
-      if (warp_ok && !fold_pv(g - 1, 422)) goto done;
+      // the item's last product (products complete in issue order, so all of them)
+      if (warp_ok && kt_hi > kt_lo) {
+        bool ok = mbar_wait(pv_full + ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag, p.status, 422);
+        if (!__all_sync(0xffffffffu, ok)) goto done;
+        tc_fence_after();
+      }
 
       // ---- item epilogue
       const int head = kvh * p.group + row % p.group;
       if (n_split == 1) {
-        if (row_ok) {
+        if (warp_ok) {                                     // (a whole warp reads tensor memory together)
           const float inv = 1.f / l;
           uint4* dst = reinterpret_cast<uint4*>(p.out + (size_t)(q_row0 + tok) * p.Hq * 64 + head * 64);
 #pragma unroll
-          for (int c = 0; c < 8; ++c)
-            dst[c] = make_uint4(pack_bf16(o[8 * c] * inv, o[8 * c + 1] * inv), pack_bf16(o[8 * c + 2] * inv, o[8 * c + 3] * inv),
-                                pack_bf16(o[8 * c + 4] * inv, o[8 * c + 5] * inv), pack_bf16(o[8 * c + 6] * inv, o[8 * c + 7] * inv));
+          for (int hf = 0; hf < 2; ++hf) {
+            uint32_t o[32];
+            tmem_ld32(t_o + hf * 32, o);
+            tmem_ld_wait();
+            if (row_ok) {
+#pragma unroll
+              for (int c = 0; c < 4; ++c)
+                dst[hf * 4 + c] = make_uint4(
+                    pack_bf16(__uint_as_float(o[8 * c]) * inv, __uint_as_float(o[8 * c + 1]) * inv),
+                    pack_bf16(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv),
+                    pack_bf16(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv),
+                    pack_bf16(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv));
+            }
+          }
+          tc_fence_before();
         }
       } else {
-        // partials of this (q-tile, kv head): [slice][66][128 rows] floats, entry 0 the running maximum (log2
-        // units), 1 the row sum, 2.. the 64 unnormalised outputs; a warp's accesses are 128-byte lines
+        // partials of this (q-tile, kv head): [slice][66][128 rows] floats, entry 0 the exponent reference (log2
+        // units), 1 the row sum under it, 2.. the 64 unnormalised outputs; a warp's accesses are 128-byte lines
         float* tile_part = p.split_ws + ((size_t)(ib.z * p.Hkv + kvh) * kAttnMaxSplits) * (66 * 128) + row;
         if (warp_ok) {
           float* part = tile_part + (size_t)split * (66 * 128);
-          part[0] = m;
+          part[0] = m_ref;
           part[128] = l;
 #pragma unroll
-          for (int e = 0; e < 64; ++e) part[(2 + e) * 128] = o[e];
+          for (int hf = 0; hf < 2; ++hf) {
+            uint32_t o[32];
+            tmem_ld32(t_o + hf * 32, o);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) part[(2 + hf * 32 + e) * 128] = __uint_as_float(o[e]);
+          }
+          tc_fence_before();
         }
         __threadfence();
         if (!warps_sync(group_bar, group_ph, lane, abort_flag, p.status, 427)) goto done;
@@ -489,6 +531,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           float M = -INFINITY;
           for (int s = 0; s < n_split; ++s) M = fmaxf(M, __ldcg(tile_part + (size_t)s * (66 * 128)));
           float Lsum = 0.f;
+          float o[64];
 #pragma unroll
           for (int e = 0; e < 64; ++e) o[e] = 0.f;
           for (int s = 0; s < n_split; ++s) {             // fixed slice order: the result does not depend on arrival
