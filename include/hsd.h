@@ -378,7 +378,8 @@ HSD_API int hsd_op_linear(hsd_ctx *ctx, const void *A, const void *W, void *C, i
 HSD_API int hsd_debug_set_gemm_tile(hsd_ctx *ctx, int tile_n, int k_slices);
 
 /* Test-only: the attention launch cuts the KV range of every query tile into slices so that it has about
- * `target_items` work items, none shorter than `min_kv_tiles` 64-token KV tiles (0 = the library's defaults).
+ * `target_items` work items, none shorter than `min_kv_tiles` 128-token KV tiles (two paged blocks; 0 = the
+ * library's defaults).
  * Results do not depend on the setting beyond fp32 summation order; tests use it to force many or no slices. */
 HSD_API int hsd_debug_set_attn_plan(hsd_ctx *ctx, int target_items, int min_kv_tiles);
 

@@ -40,7 +40,7 @@ struct hsd_ctx {
   bool pdl;           // kernels are launched with programmatic stream serialization
   int force_bn, force_splits;   // hsd_debug_set_gemm_tile
   int pair;                     // GEMMs may run as CTA pairs
-  int attn_target_items, attn_min_chunk;   // attention plan: items aimed at per launch, fewest KV tiles per slice
+  int attn_target_items, attn_min_chunk;   // attention plan: items aimed at per launch, fewest 128-key KV tiles per slice
   int tap_layer, tap_which;                // hsd_debug_tap: armed for the next forward (tap_layer < 0: none)
   void* tap_dst;
   size_t tap_bytes;
@@ -559,7 +559,7 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
   c->hg_exec = nullptr;
   c->hg_launches = 0;
   c->attn_target_items = 2 * c->n_sms;   // one item per CTA slot: slicing costs a partial hand-over per slice
-  c->attn_min_chunk = 8;
+  c->attn_min_chunk = 4;
   c->tap_layer = -1; c->tap_which = 0; c->tap_dst = nullptr; c->tap_bytes = 0;
   c->last_cuda_error = 0;
   c->launches = 0;
@@ -1123,7 +1123,7 @@ int hsd_debug_set_gemm_tile(hsd_ctx* c, int tile_n, int k_slices) {
 int hsd_debug_set_attn_plan(hsd_ctx* c, int target_items, int min_kv_tiles) {
   if (!c || target_items < 0 || min_kv_tiles < 0) return HSD_ERR_INVALID_ARG;
   c->attn_target_items = target_items ? target_items : 2 * c->n_sms;
-  c->attn_min_chunk = min_kv_tiles ? min_kv_tiles : 8;
+  c->attn_min_chunk = min_kv_tiles ? min_kv_tiles : 4;
   return HSD_OK;
 }
 

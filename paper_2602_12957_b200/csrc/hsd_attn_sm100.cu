@@ -5,37 +5,49 @@
 //
 // Work item = (q-tile, kv slice, kv head).  A q-tile is 128 MMA rows: 128/group consecutive tokens of one
 // sequence x the `group` query heads that share the kv head (GQA packing, so K/V tiles are read once per
-// group).  K and V tiles [64 keys][64 dims] are exactly one paged block per kv head, fetched by TMA through
-// the block table; K is the K-major B operand of S = Q K^T, V the MN-major B operand of P V.  The KV range a q-tile can see is cut into up to
-// kAttnMaxSplits slices so that a launch has a few items per CTA slot whatever the mix of context lengths
-// (one page chunk over a long context, or many short regions); the plan is made once per step on the
-// device (attn_plan_kernel) and reused by every layer.  Slices leave (unnormalised O, max, sum) partials in
-// the workspace and the last slice to finish combines them in slice order, so the result does not depend
-// on which CTA ran what.
+// group).  The KV range a q-tile can see is cut into up to kAttnMaxSplits slices so that a launch has about one item
+// per CTA slot whatever the mix of context lengths (one page chunk over a long context, or many short regions); the
+// plan is made once per step on the device (attn_plan_kernel) and reused by every layer.  Slices leave (unnormalised
+// O, exponent reference, sum) partials in the workspace and the last slice to finish combines them in slice order, so
+// the result does not depend on which CTA ran what.
 //
-// Persistent CTAs, two per SM, walk the item list.  Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer +
-// TMEM owner, warps 2..5 = softmax (one TMEM lane quarter each, one thread per q row, no shuffles).
-// Per KV tile: S = Q K^T (TMEM) -> softmax in registers -> P (bf16, shared memory, 128B-swizzled) -> O += P V,
-// accumulated IN TENSOR MEMORY.  S and P are double-buffered, so the tensor pipe works on tile j+1 while the softmax
-// warps are on tile j, and a softmax warp never waits for a product younger than the one two tiles back: measured with
-// every arithmetic instruction removed, a loop in which each tile waits for the product of the tile before it still
-// took four fifths of the kernel's time (two barrier hand-overs per tile on the critical path); with the accumulator
-// in tensor memory nothing in the steady state waits on a hand-over at all.  The exponent reference of a row is not
-// its running maximum but a value that is raised only when the maximum has grown by more than kRescaleBits binary
-// orders since it was set (P stays below 2^kRescaleBits, far inside bf16 and fp32 range): then, and only then, the
-// row's accumulator is read, scaled and written back.  After the first tiles of a row that is rare.  Two CTAs per SM
-// interleave further.  Every wait is a bounded mbarrier wait, so one that gives up takes the whole CTA to the common exit.
+// A KV tile is 128 keys = two paged blocks [64 keys][64 dims] per kv head, fetched by TMA through the block table
+// into adjacent halves of a stage; K is the K-major B operand of S = Q K^T (one 128 x 128 x 64 product per tile), V
+// the MN-major B operand of O += P V (128 x 64 x 128).  Persistent CTAs, two per SM, walk the item list.  Warp roles:
+// warp 0 = TMA producers (lane 0: Q and the K ring, lane 1: the V ring; K is free as soon as S has been formed, V
+// only after the second product, so the two rings run at their own pace and two stages each suffice), warp 1 = MMA
+// issuer + TMEM owner, warps 2..9 = softmax: warp w works on TMEM lane quarter w mod 4 (the hardware's rule), warps
+// 2..5 on keys 0..63 of the tile and warps 6..9 on keys 64..127, one thread per (row, half).
+// Per tile: S (TMEM, 128 fp32 columns) -> softmax in registers -> P (bf16, shared memory, 128B-swizzled, two K-major
+// sub-tiles) -> O += P V accumulated IN TENSOR MEMORY.  What the measurements behind this shape said (per 64-key tile
+// and CTA, before): the softmax warps' own instruction stream ~1,950 cycles, half of it the 64 exponentials of a row
+// queueing with the other CTA's on the SM's 16 exp lanes per clock; the issuing thread ~1,300 (140-220 cycles for
+// every probe of an already completed barrier, 70-90 per MMA or commit).  Twice the keys per barrier round and MMA
+// group, and twice the warps on the exponentials, attack both.
+// The exponent reference of a row is not its running maximum but a value that is raised only when the maximum has
+// grown by more than kRescaleBits binary orders since it was set (P stays below 2^kRescaleBits, far inside bf16 and
+// fp32 range): then, and only then, the row's accumulator is read, scaled and written back; after the first tiles of
+// a row that is rare.  The two threads of a row swap their halves' maxima through shared memory once per tile, so they
+// take the same decisions.  Every wait is a bounded mbarrier wait, so one that gives up takes the whole CTA to the
+// common exit.
 #include "hsd_kernels.h"
 
 namespace hsd {
 
-constexpr int kAttnThreads = 192;
-constexpr int KV_STAGES = 3;
+constexpr int kSoftmaxWarps = 8;
+constexpr int kAttnThreads = 32 * (2 + kSoftmaxWarps);
+constexpr int KV_STAGES = 2;                       // per ring
 constexpr int Q_BYTES = 128 * 128;
-constexpr int KV_TILE_BYTES = 64 * 128;            // one K tile or one V tile
-constexpr int P_BYTES = 128 * 128;
-constexpr int ATTN_SMEM = Q_BYTES + KV_STAGES * 2 * KV_TILE_BYTES + 2 * P_BYTES + 1024 + 256;
-constexpr int ATTN_TMEM_COLS = 256;                // S0 S1 (64 fp32 columns each), O (64), 64 unused (allocations are powers of two)
+constexpr int KV_BLOCK_BYTES = 64 * 128;           // one paged block of K or of V for one kv head
+constexpr int KV_TILE_BYTES = 2 * KV_BLOCK_BYTES;  // 128 keys
+constexpr int P_SUB_BYTES = 128 * 128;             // P for 64 keys: 128 rows x 128 bytes
+constexpr int P_BYTES = 2 * P_SUB_BYTES;
+constexpr int ATTN_BAR_BYTES = 256;
+constexpr int ATTN_XCH_BYTES = 2 * 128 * 2;        // half-row maxima of a tile, one bf16 per (half, row)
+// No alignment slack: two CTAs of this size plus the per-CTA reserve just fit an SM, so the kernel relies on the
+// 1024-byte alignment it declares for its dynamic shared memory (the swizzled tiles need it) and checks it.
+constexpr int ATTN_SMEM = Q_BYTES + 2 * KV_STAGES * KV_TILE_BYTES + P_BYTES + ATTN_XCH_BYTES + ATTN_BAR_BYTES;
+constexpr int ATTN_TMEM_COLS = 256;                // S (128 fp32 columns), O (64), 64 unused (allocations are powers of two)
 constexpr float kRescaleBits = 8.f;
 
 struct AttnParams {
@@ -57,6 +69,9 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   float y;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
   return y;
+}
+__device__ __forceinline__ void named_bar_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 // Barrier among whole warps on an mbarrier whose count is the number of warps: every lane's earlier shared-memory
 // writes are visible to every participant afterwards.  `phase` counts this thread's uses of `bar`.
@@ -90,7 +105,7 @@ __global__ void attn_plan_kernel(RowMeta rm, AttnPlan pl, int n_seqs, int tokens
     const int L = rm.seq_len[s], n = rm.seq_n[s];
     for (int t = t0; t < t1; ++t) {
       const int tok_end = min(n, (t - t0 + 1) * tokens_per_tile);
-      const int n_kv = (L + tok_end + 63) >> 6;
+      const int n_kv = (L + tok_end + 127) >> 7;         // 128-key tiles (two paged blocks): the unit slices are cut in
       pl.tile_seq[t] = s;
       pl.tile_nkv[t] = n_kv;
       my += n_kv;
@@ -127,14 +142,16 @@ __global__ void attn_plan_kernel(RowMeta rm, AttnPlan pl, int n_seqs, int tokens
       const int n_kv = pl.tile_nkv[t];
       const int s = pl.tile_seq[t];
       const int tok0 = (t - rm.seq_tile0[s]) * tokens_per_tile;
+      const int n_tok = min(tokens_per_tile, rm.seq_n[s] - tok0);
+      const int blocks = (rm.seq_len[s] + tok0 + n_tok + 63) >> 6;    // 64-key blocks the q-tile can see
       const int ns = max(1, min(kAttnMaxSplits, (n_kv + chunk - 1) / chunk));
       const int base = n_kv / ns, rem = n_kv % ns;
       int lo = 0;
       for (int k = 0; k < ns; ++k) {
         const int len = base + (k < rem ? 1 : 0);
-        pl.items_unsorted[2 * n] = make_int4(rm.seq_q0[s] + tok0, rm.seq_len[s] + tok0,
-                                             min(tokens_per_tile, rm.seq_n[s] - tok0), rm.seq_slot[s]);
-        pl.items_unsorted[2 * n + 1] = make_int4(lo | ((lo + len) << 16), k | (ns << 8) | (tok0 << 16), t, len);
+        // the item's range in 64-key blocks: only the last slice of a q-tile can end on half a tile
+        pl.items_unsorted[2 * n] = make_int4(rm.seq_q0[s] + tok0, rm.seq_len[s] + tok0, n_tok, rm.seq_slot[s]);
+        pl.items_unsorted[2 * n + 1] = make_int4((2 * lo) | (min(blocks, 2 * (lo + len)) << 16), k | (ns << 8) | (tok0 << 16), t, len);
         ++n;
         lo += len;
       }
@@ -170,40 +187,47 @@ void launch_attn_plan(cudaStream_t st, const RowMeta& rm, const AttnPlan& pl, in
 __global__ void __launch_bounds__(kAttnThreads, 2)
 attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, AttnParams p) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  extern __shared__ __align__(1024) uint8_t smem[];
   uint8_t* sQ = smem;
-  uint8_t* sKV = sQ + Q_BYTES;                         // stage s: K at s*2*KV_TILE_BYTES, V right after
-  uint8_t* sP = sKV + KV_STAGES * 2 * KV_TILE_BYTES;   // two P buffers
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sP + 2 * P_BYTES);
+  uint8_t* sK = sQ + Q_BYTES;                          // ring stage s: sK + s * KV_TILE_BYTES, block 0 then block 1
+  uint8_t* sV = sK + KV_STAGES * KV_TILE_BYTES;
+  uint8_t* sP = sV + KV_STAGES * KV_TILE_BYTES;        // sub-tile h (keys 64h .. 64h+63): sP + h * P_SUB_BYTES
+  __nv_bfloat16* xch = reinterpret_cast<__nv_bfloat16*>(sP + P_BYTES);        // [half][row]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sP + P_BYTES + ATTN_XCH_BYTES);
   uint64_t* q_full = bars;                 // Q tile landed                       (one phase per item)
   uint64_t* q_empty = bars + 1;            // every S MMA of the item has read Q   (one phase per item)
-  uint64_t* kv_full = bars + 2;
-  uint64_t* kv_empty = kv_full + KV_STAGES;
-  uint64_t* s_full = kv_empty + KV_STAGES;
-  uint64_t* s_empty = s_full + 2;
-  uint64_t* p_full = s_empty + 2;
-  uint64_t* pv_full = p_full + 2;          // [g & 1] O += P(g) V(g) has completed
-  uint64_t* group_bar = pv_full + 2;       // the four softmax warps (slice hand-over)
+  uint64_t* k_full = bars + 2;             // [stage]
+  uint64_t* k_empty = k_full + KV_STAGES;  // [stage] S of the tile has been formed
+  uint64_t* v_full = k_empty + KV_STAGES;
+  uint64_t* v_empty = v_full + KV_STAGES;  // [stage] O += P V of the tile has completed
+  uint64_t* s_full = v_empty + KV_STAGES;  // S(t) is in tensor memory
+  uint64_t* s_empty = s_full + 1;          // the softmax warps hold S(t) in registers
+  uint64_t* p_full = s_empty + 1;          // P(t) is in shared memory (and the accumulator rescaled, if it had to be)
+  uint64_t* o_full = p_full + 1;           // O += P(t) V(t) has completed
+  uint64_t* group_bar = o_full + 1;        // the eight softmax warps (slice hand-over)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(group_bar + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   volatile int* s_flag = abort_flag + 1;   // combine: "this CTA ran the last slice to finish"
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (smem_u32(smem) & 1023u) {            // uniform over the CTA: nothing has been set up yet
+    if (threadIdx.x == 0) dev_fail(p.status, DEV_WAIT_TIMEOUT, 499);
+    return;
+  }
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
     mbar_init(q_empty, 1);
     for (int s = 0; s < KV_STAGES; ++s) {
-      mbar_init(kv_full + s, 1);
-      mbar_init(kv_empty + s, 1);
+      mbar_init(k_full + s, 1);
+      mbar_init(k_empty + s, 1);
+      mbar_init(v_full + s, 1);
+      mbar_init(v_empty + s, 1);
     }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(s_full + b, 1);
-      mbar_init(s_empty + b, 4);
-      mbar_init(p_full + b, 128);
-      mbar_init(pv_full + b, 1);
-    }
-    mbar_init(group_bar, 4);
+    mbar_init(s_full, 1);
+    mbar_init(s_empty, kSoftmaxWarps);
+    mbar_init(p_full, kSoftmaxWarps);
+    mbar_init(o_full, 1);
+    mbar_init(group_bar, kSoftmaxWarps);
     *abort_flag = 0;
     fence_mbar_init();
     tma_prefetch_desc(&tmQ);
@@ -242,11 +266,17 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     return w < total ? w : -1;
   };
 
-  // Global tile counter g (all items of this CTA): S / P / PV buffer = g & 1, KV stage = g % KV_STAGES, and every
-  // barrier's parity follows from how often g has used it; n counts items (Q hand-over barriers).
+  // Tile counter t (all 128-key tiles of all items of this CTA): ring stage = t % KV_STAGES, and every barrier's
+  // parity follows from how often t has used it; n counts items (Q hand-over barriers).
   if (warp == 0) {
-    if (lane == 0) {
-      uint32_t g = 0;
+    if (lane < 2) {
+      // lane 0: Q and the K ring; lane 1: the V ring
+      const bool is_k = lane == 0;
+      uint64_t* full = is_k ? k_full : v_full;
+      uint64_t* empty = is_k ? k_empty : v_empty;
+      uint8_t* ring = is_k ? sK : sV;
+      const CUtensorMap* tm = is_k ? &tmK : &tmV;
+      uint32_t t = 0;
       int n = 0;
       for (int r = 0; r < n_rounds; ++r) {
         const int w = item_of_round(r);
@@ -255,83 +285,88 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         const int kvh = w % p.Hkv;
         const int kt_lo = ib.x & 0xffff, kt_hi = ib.x >> 16;
         const int* bt = p.block_table + (size_t)ia.w * p.max_blocks;
-        int phys = bt[kt_lo];
-        if (!mbar_wait(q_empty, (n & 1) ^ 1u, abort_flag, p.status, 400)) goto done;
-        mbar_expect_tx(q_full, Q_BYTES);
-        tma_load_3d(sQ, &tmQ, q_full, 0, kvh * p.group, ia.x);
-        for (int j = kt_lo; j < kt_hi; ++j, ++g) {
-          const int phys_next = (j + 1 < kt_hi) ? bt[j + 1] : 0;      // block-table entry of the next tile, ahead of need
-          const int st = g % KV_STAGES;
-          if (!mbar_wait(kv_empty + st, ((g / KV_STAGES) & 1) ^ 1u, abort_flag, p.status, 401)) goto done;
-          const int row = (((p.layer * p.n_blocks) + phys) * p.Hkv + kvh) * 64;
-          uint8_t* k_dst = sKV + st * 2 * KV_TILE_BYTES;
-          mbar_expect_tx(kv_full + st, 2 * KV_TILE_BYTES);
-          tma_load_2d(k_dst, &tmK, kv_full + st, 0, row);
-          tma_load_2d(k_dst + KV_TILE_BYTES, &tmV, kv_full + st, 0, row);
-          phys = phys_next;
+        if (is_k) {
+          if (!mbar_wait(q_empty, (n & 1) ^ 1u, abort_flag, p.status, 400)) goto done;
+          mbar_expect_tx(q_full, Q_BYTES);
+          tma_load_3d(sQ, &tmQ, q_full, 0, kvh * p.group, ia.x);
+        }
+        for (int kt = kt_lo; kt < kt_hi; kt += 2, ++t) {
+          // the tile's two blocks; a slice of odd length ends with half a tile: the last block is staged twice and
+          // the softmax warps mask its second copy
+          const int phys0 = bt[kt], phys1 = bt[kt + 1 < kt_hi ? kt + 1 : kt];
+          const int st = t % KV_STAGES;
+          if (!mbar_wait(empty + st, ((t / KV_STAGES) & 1) ^ 1u, abort_flag, p.status, 401)) goto done;
+          const int row0 = (((p.layer * p.n_blocks) + phys0) * p.Hkv + kvh) * 64;
+          const int row1 = (((p.layer * p.n_blocks) + phys1) * p.Hkv + kvh) * 64;
+          uint8_t* dst = ring + st * KV_TILE_BYTES;
+          mbar_expect_tx(full + st, KV_TILE_BYTES);
+          tma_load_2d(dst, tm, full + st, 0, row0);
+          tma_load_2d(dst + KV_BLOCK_BYTES, tm, full + st, 0, row1);
         }
         ++n;
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(64);
+      constexpr uint32_t idesc_s = umma_idesc_bf16(128);
       constexpr uint32_t idesc_pv = umma_idesc_bf16(64, true);
       const uint32_t q_addr = smem_u32(sQ);
-      uint32_t g = 0;
+      uint32_t t = 0;
       int n = 0;
       for (int r = 0; r < n_rounds; ++r) {
         const int w = item_of_round(r);
         if (w < 0) continue;
         const int4 ib = p.plan.items[2 * (w / p.Hkv) + 1];
-        const int n_it = (ib.x >> 16) - (ib.x & 0xffff);
-        auto issue_s = [&](uint32_t gi) -> bool {
-          const int st = gi % KV_STAGES;
-          if (!mbar_wait(kv_full + st, (gi / KV_STAGES) & 1, abort_flag, p.status, 410)) return false;
-          if (!mbar_wait(s_empty + (gi & 1), ((gi >> 1) & 1) ^ 1u, abort_flag, p.status, 411)) return false;
+        const int n_it = ((ib.x >> 16) - (ib.x & 0xffff) + 1) / 2;      // 128-key tiles of the item
+        // S(ti) = Q K(ti)^T: four K = 16 steps over the 64 dims, N = 128 keys
+        auto issue_s = [&](uint32_t ti, bool last) -> bool {
+          const int st = ti % KV_STAGES;
+          if (!mbar_wait(k_full + st, (ti / KV_STAGES) & 1, abort_flag, p.status, 410)) return false;
+          if (!mbar_wait(s_empty, (ti & 1) ^ 1u, abort_flag, p.status, 411)) return false;   // S(ti - 1) is in registers
           tc_fence_after();
-          const uint32_t k_addr = smem_u32(sKV + st * 2 * KV_TILE_BYTES);
-          const uint32_t d = tmem_base + (gi & 1) * 64;
+          const uint32_t k_addr = smem_u32(sK + st * KV_TILE_BYTES);
 #pragma unroll
           for (int k = 0; k < 4; ++k)
-            umma_bf16(d, umma_desc_sw128(q_addr + k * 32), umma_desc_sw128(k_addr + k * 32), idesc, k != 0);
-          umma_commit(s_full + (gi & 1));
+            umma_bf16(tmem_base, umma_desc_sw128(q_addr + k * 32), umma_desc_sw128(k_addr + k * 32), idesc_s, k != 0);
+          umma_commit(s_full);
+          umma_commit(k_empty + st);              // K is free once S has been formed
+          if (last) umma_commit(q_empty);         // last S MMA of the item: Q is free once it completes
           return true;
         };
         if (!mbar_wait(q_full, n & 1, abort_flag, p.status, 412)) goto done;
-        if (!issue_s(g)) goto done;
-        if (n_it == 1) umma_commit(q_empty);
-        for (int j = 0; j < n_it; ++j, ++g) {
-          if (j + 1 < n_it) {
-            if (!issue_s(g + 1)) goto done;
-            if (j + 2 == n_it) umma_commit(q_empty);      // last S MMA of the item issued: Q is free once it completes
-          }
-          // P(g) is written, and whatever had to be done to the accumulator before this product is done
-          if (!mbar_wait(p_full + (g & 1), (g >> 1) & 1, abort_flag, p.status, 413)) goto done;
+        if (!issue_s(t, n_it == 1)) goto done;
+        for (int j = 0; j < n_it; ++j, ++t) {
+          if (j + 1 < n_it && !issue_s(t + 1, j + 2 == n_it)) goto done;
+          // P(t) is written, and whatever had to be done to the accumulator before this product is done
+          if (!mbar_wait(p_full, t & 1, abort_flag, p.status, 413)) goto done;
+          const int st = t % KV_STAGES;
+          if (!mbar_wait(v_full + st, (t / KV_STAGES) & 1, abort_flag, p.status, 415)) goto done;
           tc_fence_after();
-          const int st = g % KV_STAGES;
-          const uint32_t p_addr = smem_u32(sP + (g & 1) * P_BYTES);
-          const uint32_t v_addr = smem_u32(sKV + st * 2 * KV_TILE_BYTES + KV_TILE_BYTES);
+          const uint32_t p_addr = smem_u32(sP);
+          const uint32_t v_addr = smem_u32(sV + st * KV_TILE_BYTES);
           const uint32_t d = tmem_base + 128;      // the item's accumulator: the first product of an item overwrites it
 #pragma unroll
-          for (int k = 0; k < 4; ++k)   // V [key][dim] is MN-major: a K step of 16 keys is 16 rows of 128 bytes
-            umma_bf16(d, umma_desc_sw128(p_addr + k * 32), umma_desc_sw128(v_addr + k * 2048), idesc_pv,
-                      (j != 0 || k != 0) ? 1u : 0u);
-          umma_commit(kv_empty + st);
-          umma_commit(pv_full + (g & 1));
+          for (int k = 0; k < 8; ++k)   // 16 keys per step: P sub-tile k / 4, 32 bytes along its rows; V [key][dim] is
+                                        // MN-major, a step of 16 keys is 16 rows of 128 bytes
+            umma_bf16(d, umma_desc_sw128(p_addr + (k >> 2) * P_SUB_BYTES + (k & 3) * 32),
+                      umma_desc_sw128(v_addr + k * 2048), idesc_pv, (j != 0 || k != 0) ? 1u : 0u);
+          umma_commit(v_empty + st);
+          umma_commit(o_full);
         }
         ++n;
       }
       // every stage-release arrival must land before the CTA's shared memory can be handed on
-      if (g > 0 && !mbar_wait(pv_full + ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag, p.status, 414)) goto done;
+      if (t > 0 && !mbar_wait(o_full, (t - 1) & 1, abort_flag, p.status, 414)) goto done;
     }
   } else {
-    const int quarter = warp & 3;
+    const int quarter = warp & 3;                      // TMEM lane quarter a warp may touch = warp id mod 4
+    const int half = (warp - 2) >> 2;                  // keys [64 half, 64 half + 64) of every tile
     const int row = quarter * 32 + lane;               // q row of the tile = TMEM lane
     const int tok = row / p.group;
     const uint32_t t_lane = tmem_base + (uint32_t(quarter * 32) << 16);
+    const uint32_t t_o = t_lane + 128 + half * 32;     // this thread's 32 columns of the accumulator row
     const float sc = 0.125f * 1.4426950408889634f;     // 1/sqrt(64) * log2(e)
-    uint32_t g = 0, group_ph = 0;
+    uint32_t t = 0, group_ph = 0;
     for (int r = 0; r < n_rounds; ++r) {
       const int w = item_of_round(r);
       if (w < 0) continue;
@@ -351,67 +386,83 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       // they keep step with the barriers but skip the loads, the exps and the P rows (which only feed their own,
       // never stored, output rows)
       const bool warp_ok = (quarter * 32) / p.group < n_tok;
-      float m_ref = -INFINITY, l = 0.f;                  // exponent reference (log2 units, scaled) and row sum under it
-      const uint32_t t_o = t_lane + 128;                 // this warp's lanes of the accumulator
+      float m_ref = -INFINITY, l = 0.f;                // exponent reference (log2 units, scaled); sum of this thread's P
+      // visibility of the 32 keys from `key0` on for this thread's row, as a bit mask
+      auto visible = [&](int key0, int key_end) -> uint32_t {
+        if (key0 >= key_end) return 0u;                 // the second copy of a slice's last block
+        if (p.anc) {
+          auto word = [&](int i) -> uint32_t {
+            return i < 0 ? 0xffffffffu : i == 0 ? am.x : i == 1 ? am.y : i == 2 ? am.z : i == 3 ? am.w : 0u;
+          };
+          const int pos = key0 - len0;
+          if (pos <= -32) return 0xffffffffu;
+          if (pos >= 128) return 0u;
+          const int wi = pos >> 5;                      // floor, also for negative positions
+          return __funnelshift_r(word(wi), word(wi + 1), pos & 31);
+        }
+        const int nvis = pos_row - key0 + 1;            // keys key0 .. pos_row are visible
+        return nvis >= 32 ? 0xffffffffu : (nvis <= 0 ? 0u : ((1u << nvis) - 1u));
+      };
 
-      for (int j = kt_lo; j < kt_hi; ++j, ++g) {
-        const int b = g & 1;
-        bool ok = mbar_wait(s_full + b, (g >> 1) & 1, abort_flag, p.status, 420);
+      for (int kt = kt_lo; kt < kt_hi; kt += 2, ++t) {
+        bool ok = mbar_wait(s_full, t & 1, abort_flag, p.status, 420);
         if (!__all_sync(0xffffffffu, ok)) goto done;
         tc_fence_after();
         if (!warp_ok) {
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(s_empty + b);
-          mbar_arrive(p_full + b);
+          if (lane == 0) mbar_arrive(s_empty);
+          // S(t + 1) is issued before P(t) is consumed, so this warp could be back here for the next tile while phase
+          // t of p_full is still open, and its arrival would then be counted there: like the warps that do write P,
+          // it arrives for tile t only once the product of tile t - 1 (hence phase t - 1 of p_full) is complete
+          if (t > 0) {
+            ok = mbar_wait(o_full, (t - 1) & 1, abort_flag, p.status, 424);
+            if (!__all_sync(0xffffffffu, ok)) goto done;
+          }
+          if (lane == 0) mbar_arrive(p_full);
           continue;
         }
+        const int key_end = min(kt + 2, kt_hi) * 64;    // keys of this tile that belong to the slice
+        const int kb_own = kt * 64 + half * 64;
+        // does any key of the tile need masking for some row of the q-tile?  (warp-uniform)
+        const bool masked_tile = p.anc ? (kt * 64 + 127 >= len0) : (kt * 64 + 127 > pos0);
+        const bool partial_tile = key_end < kt * 64 + 128;
         uint32_t s0[32], s1[32];
-        tmem_ld32(t_lane + b * 64, s0);
-        tmem_ld32(t_lane + b * 64 + 32, s1);
+        tmem_ld32(t_lane + half * 64, s0);
+        tmem_ld32(t_lane + half * 64 + 32, s1);
         tmem_ld_wait();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(s_empty + b);
-
-        const int kbase = j * 64;
-        if (p.anc) {
-          if (kbase + 63 >= len0) {                       // the tile holds rows of this call
-            // 32 bits of the row's visibility string from key position `pos` on: ones below the committed length,
-            // the ancestry mask over the call's rows, zeros beyond them
-            auto word = [&](int i) -> uint32_t {
-              return i < 0 ? 0xffffffffu : i == 0 ? am.x : i == 1 ? am.y : i == 2 ? am.z : i == 3 ? am.w : 0u;
-            };
-            auto vis32 = [&](int pos) -> uint32_t {
-              if (pos <= -32) return 0xffffffffu;
-              if (pos >= 128) return 0u;
-              const int wi = pos >> 5;                    // floor, also for negative positions
-              return __funnelshift_r(word(wi), word(wi + 1), pos & 31);
-            };
-            const uint32_t v0 = vis32(kbase - len0), v1 = vis32(kbase - len0 + 32);
-#pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              if (!((v0 >> e) & 1u)) s0[e] = 0xff800000u;          // -inf
-              if (!((v1 >> e) & 1u)) s1[e] = 0xff800000u;
-            }
-          }
-        } else if (kbase + 63 > pos0) {                   // some row of the tile masks part of this KV tile
+        if (lane == 0) mbar_arrive(s_empty);
+        if (masked_tile || partial_tile) {
+          const uint32_t v0 = visible(kb_own, key_end), v1 = visible(kb_own + 32, key_end);
 #pragma unroll
           for (int e = 0; e < 32; ++e) {
-            if (kbase + e > pos_row) s0[e] = 0xff800000u;          // -inf
-            if (kbase + 32 + e > pos_row) s1[e] = 0xff800000u;
+            if (!((v0 >> e) & 1u)) s0[e] = 0xff800000u;            // -inf
+            if (!((v1 >> e) & 1u)) s1[e] = 0xff800000u;
           }
         }
         float mx = -INFINITY;
 #pragma unroll
         for (int e = 0; e < 32; ++e) mx = max3(mx, __uint_as_float(s0[e]), __uint_as_float(s1[e]));
+        // The row's maximum over all 128 keys: the two threads of a row swap their halves' maxima through shared memory.
+        // Both use the bf16-rounded values of BOTH halves, so they arrive at the same number (the reference only has to
+        // be near the maximum, and identical for the row's two threads).
+        {
+          const __nv_bfloat16 mine = __float2bfloat16_rn(mx);
+          xch[half * 128 + row] = mine;
+          named_bar_sync(1 + quarter, 64);                 // the two warps of this lane quarter
+          mx = fmaxf(__bfloat162float(mine), __bfloat162float(xch[(half ^ 1) * 128 + row]));
+          named_bar_sync(1 + quarter, 64);                 // both have read before either writes the next tile's
+        }
         mx *= sc;
         // The reference moves only when the maximum has outgrown it by more than kRescaleBits (or nothing has been
-        // accumulated under it yet: then moving it costs nothing).
+        // accumulated under it yet: then moving it costs nothing).  `l` is this thread's half of the row sum; whether
+        // anything has been accumulated is a property of the row, so the test uses the reference itself.
         float alpha = 1.f;
         bool rescale = false;
         if (mx > m_ref) {
-          if (l == 0.f) {
+          if (m_ref == -INFINITY) {
             m_ref = mx;                                   // nothing accumulated so far (first tile, or all keys masked)
           } else if (mx > m_ref + kRescaleBits) {
             alpha = ex2(m_ref - mx);
@@ -437,67 +488,69 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           pk[16 + e] = pack_bf16(a0, a1);
         }
         l = l * alpha + sum;
-        // P's buffer was last read by the product of tile g - 2: the only wait of the steady state, two tiles back
-        if (g >= 2) {
-          ok = mbar_wait(pv_full + b, ((g - 2) >> 1) & 1, abort_flag, p.status, 421);
-          if (!__all_sync(0xffffffffu, ok)) goto done;
-        }
-        if (__any_sync(0xffffffffu, rescale)) {
-          // rare: scale this warp's accumulator rows (alpha = 1 where not needed) once the product before this tile,
-          // which still adds into them, has completed
-          ok = mbar_wait(pv_full + (b ^ 1), ((g - 1) >> 1) & 1, abort_flag, p.status, 423);
+        // P's buffer is read by the product of tile t - 1, which also still adds into the accumulator
+        if (t > 0) {
+          ok = mbar_wait(o_full, (t - 1) & 1, abort_flag, p.status, 421);
           if (!__all_sync(0xffffffffu, ok)) goto done;
           tc_fence_after();
+        }
+        if (__any_sync(0xffffffffu, rescale)) {
+          // rare: scale this thread's half of the accumulator row (alpha = 1 where not needed)
+          uint32_t o[32];
+          tmem_ld32(t_o, o);
+          tmem_ld_wait();
 #pragma unroll
-          for (int hf = 0; hf < 2; ++hf) {
-            uint32_t o[32];
-            tmem_ld32(t_o + hf * 32, o);
-            tmem_ld_wait();
-#pragma unroll
-            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st32(t_o + hf * 32, o);
-          }
+          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+          tmem_st32(t_o, o);
           tmem_st_wait();
           tc_fence_before();
         }
-        // P row -> shared memory, K-major 128B-swizzled: 16-byte chunk c of row r sits at chunk c ^ (r & 7)
-        uint8_t* prow = sP + b * P_BYTES + row * 128;
+        // P row -> shared memory, sub-tile `half`, K-major 128B-swizzled: 16-byte chunk c of row r sits at chunk c ^ (r & 7)
+        uint8_t* prow = sP + half * P_SUB_BYTES + row * 128;
 #pragma unroll
         for (int c = 0; c < 8; ++c)
           *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) =
               make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
         fence_proxy_async_smem();
-        mbar_arrive(p_full + b);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(p_full);
       }
       // the item's last product (products complete in issue order, so all of them)
-      if (warp_ok && kt_hi > kt_lo) {
-        bool ok = mbar_wait(pv_full + ((g - 1) & 1), ((g - 1) >> 1) & 1, abort_flag, p.status, 422);
+      if (kt_hi > kt_lo) {
+        bool ok = mbar_wait(o_full, (t - 1) & 1, abort_flag, p.status, 422);
         if (!__all_sync(0xffffffffu, ok)) goto done;
         tc_fence_after();
       }
+      // the row sum is the sum of its two threads' halves: exchanged through P's buffer, which nothing reads any more
+      float l_row = l;
+      if (warp_ok) {
+        float* lx = reinterpret_cast<float*>(sP);        // [2][128]
+        lx[half * 128 + row] = l;
+        named_bar_sync(1 + quarter, 64);                 // the two warps of this lane quarter
+        l_row += lx[(half ^ 1) * 128 + row];
+        named_bar_sync(1 + quarter, 64);                 // both have read before either writes P again
+      }
 
-      // ---- item epilogue
+      // ---- item epilogue: this thread owns dims [32 half, 32 half + 32) of its row
       const int head = kvh * p.group + row % p.group;
       if (n_split == 1) {
         if (warp_ok) {                                     // (a whole warp reads tensor memory together)
-          const float inv = 1.f / l;
-          uint4* dst = reinterpret_cast<uint4*>(p.out + (size_t)(q_row0 + tok) * p.Hq * 64 + head * 64);
-#pragma unroll
-          for (int hf = 0; hf < 2; ++hf) {
-            uint32_t o[32];
-            tmem_ld32(t_o + hf * 32, o);
-            tmem_ld_wait();
-            if (row_ok) {
-#pragma unroll
-              for (int c = 0; c < 4; ++c)
-                dst[hf * 4 + c] = make_uint4(
-                    pack_bf16(__uint_as_float(o[8 * c]) * inv, __uint_as_float(o[8 * c + 1]) * inv),
-                    pack_bf16(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv),
-                    pack_bf16(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv),
-                    pack_bf16(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv));
-            }
-          }
+          const float inv = 1.f / l_row;
+          uint32_t o[32];
+          tmem_ld32(t_o, o);
+          tmem_ld_wait();
           tc_fence_before();
+          if (row_ok) {
+            uint4* dst = reinterpret_cast<uint4*>(p.out + (size_t)(q_row0 + tok) * p.Hq * 64 + head * 64 + half * 32);
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+              dst[c] = make_uint4(
+                  pack_bf16(__uint_as_float(o[8 * c]) * inv, __uint_as_float(o[8 * c + 1]) * inv),
+                  pack_bf16(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv),
+                  pack_bf16(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv),
+                  pack_bf16(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv));
+          }
         }
       } else {
         // partials of this (q-tile, kv head): [slice][66][128 rows] floats, entry 0 the exponent reference (log2
@@ -505,17 +558,16 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         float* tile_part = p.split_ws + ((size_t)(ib.z * p.Hkv + kvh) * kAttnMaxSplits) * (66 * 128) + row;
         if (warp_ok) {
           float* part = tile_part + (size_t)split * (66 * 128);
-          part[0] = m_ref;
-          part[128] = l;
-#pragma unroll
-          for (int hf = 0; hf < 2; ++hf) {
-            uint32_t o[32];
-            tmem_ld32(t_o + hf * 32, o);
-            tmem_ld_wait();
-#pragma unroll
-            for (int e = 0; e < 32; ++e) part[(2 + hf * 32 + e) * 128] = __uint_as_float(o[e]);
+          if (half == 0) {
+            part[0] = m_ref;
+            part[128] = l_row;
           }
+          uint32_t o[32];
+          tmem_ld32(t_o, o);
+          tmem_ld_wait();
           tc_fence_before();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) part[(2 + half * 32 + e) * 128] = __uint_as_float(o[e]);
         }
         __threadfence();
         if (!warps_sync(group_bar, group_ph, lane, abort_flag, p.status, 427)) goto done;
@@ -531,22 +583,22 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           float M = -INFINITY;
           for (int s = 0; s < n_split; ++s) M = fmaxf(M, __ldcg(tile_part + (size_t)s * (66 * 128)));
           float Lsum = 0.f;
-          float o[64];
+          float o[32];
 #pragma unroll
-          for (int e = 0; e < 64; ++e) o[e] = 0.f;
+          for (int e = 0; e < 32; ++e) o[e] = 0.f;
           for (int s = 0; s < n_split; ++s) {             // fixed slice order: the result does not depend on arrival
             const float* ps = tile_part + (size_t)s * (66 * 128);
-            const float mx = __ldcg(ps);
-            const float wgt = (mx == -INFINITY) ? 0.f : ex2(mx - M);
+            const float mxs = __ldcg(ps);
+            const float wgt = (mxs == -INFINITY) ? 0.f : ex2(mxs - M);
             Lsum += wgt * __ldcg(ps + 128);
 #pragma unroll
-            for (int e = 0; e < 64; ++e) o[e] += wgt * __ldcg(ps + (2 + e) * 128);
+            for (int e = 0; e < 32; ++e) o[e] += wgt * __ldcg(ps + (2 + half * 32 + e) * 128);
           }
           if (row_ok) {
             const float inv = 1.f / Lsum;
-            uint4* dst = reinterpret_cast<uint4*>(p.out + (size_t)(q_row0 + tok) * p.Hq * 64 + head * 64);
+            uint4* dst = reinterpret_cast<uint4*>(p.out + (size_t)(q_row0 + tok) * p.Hq * 64 + head * 64 + half * 32);
 #pragma unroll
-            for (int c = 0; c < 8; ++c)
+            for (int c = 0; c < 4; ++c)
               dst[c] = make_uint4(pack_bf16(o[8 * c] * inv, o[8 * c + 1] * inv), pack_bf16(o[8 * c + 2] * inv, o[8 * c + 3] * inv),
                                   pack_bf16(o[8 * c + 4] * inv, o[8 * c + 5] * inv), pack_bf16(o[8 * c + 6] * inv, o[8 * c + 7] * inv));
           }
