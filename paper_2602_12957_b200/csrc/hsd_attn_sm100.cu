@@ -18,8 +18,8 @@
 // only after the second product, so the two rings run at their own pace and two stages each suffice), warp 1 = MMA
 // issuer + TMEM owner, warps 2..9 = softmax: warp w works on TMEM lane quarter w mod 4 (the hardware's rule), warps
 // 2..5 on keys 0..63 of the tile and warps 6..9 on keys 64..127, one thread per (row, half).
-// Per tile: S (TMEM, 128 fp32 columns) -> softmax in registers -> P (bf16, shared memory, 128B-swizzled, two K-major
-// sub-tiles) -> O += P V accumulated IN TENSOR MEMORY.  What the measurements behind this shape said (per 64-key tile
+// Per tile: S (TMEM, 128 fp32 columns) -> softmax in registers -> P (bf16, back into TMEM: 64 columns, the A operand
+// of the second product, so P never passes through shared memory) -> O += P V accumulated IN TENSOR MEMORY.  What the measurements behind this shape said (per 64-key tile
 // and CTA, before): the softmax warps' own instruction stream ~1,950 cycles, half of it the 64 exponentials of a row
 // queueing with the other CTA's on the SM's 16 exp lanes per clock; the issuing thread ~1,300 (140-220 cycles for
 // every probe of an already completed barrier, 70-90 per MMA or commit).  Twice the keys per barrier round and MMA
@@ -40,14 +40,13 @@ constexpr int KV_STAGES = 2;                       // per ring
 constexpr int Q_BYTES = 128 * 128;
 constexpr int KV_BLOCK_BYTES = 64 * 128;           // one paged block of K or of V for one kv head
 constexpr int KV_TILE_BYTES = 2 * KV_BLOCK_BYTES;  // 128 keys
-constexpr int P_SUB_BYTES = 128 * 128;             // P for 64 keys: 128 rows x 128 bytes
-constexpr int P_BYTES = 2 * P_SUB_BYTES;
 constexpr int ATTN_BAR_BYTES = 256;
-constexpr int ATTN_XCH_BYTES = 2 * 128 * 2;        // half-row maxima of a tile, one bf16 per (half, row)
+constexpr int ATTN_XCH_BYTES = 2 * 128 * 2 + 2 * 128 * 4;   // per (half, row): the tile's half-row maximum (bf16); the item's half-row sum (fp32)
 // No alignment slack: two CTAs of this size plus the per-CTA reserve just fit an SM, so the kernel relies on the
 // 1024-byte alignment it declares for its dynamic shared memory (the swizzled tiles need it) and checks it.
-constexpr int ATTN_SMEM = Q_BYTES + 2 * KV_STAGES * KV_TILE_BYTES + P_BYTES + ATTN_XCH_BYTES + ATTN_BAR_BYTES;
-constexpr int ATTN_TMEM_COLS = 256;                // S (128 fp32 columns), O (64), 64 unused (allocations are powers of two)
+constexpr int ATTN_SMEM = Q_BYTES + 2 * KV_STAGES * KV_TILE_BYTES + ATTN_XCH_BYTES + ATTN_BAR_BYTES;
+constexpr int ATTN_TMEM_COLS = 256;                // S: 128 fp32 columns, O: 64, P: 64 (128 keys, two bf16 per column)
+constexpr int TMEM_COL_O = 128, TMEM_COL_P = 192;
 constexpr float kRescaleBits = 8.f;
 
 struct AttnParams {
@@ -191,9 +190,9 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   uint8_t* sQ = smem;
   uint8_t* sK = sQ + Q_BYTES;                          // ring stage s: sK + s * KV_TILE_BYTES, block 0 then block 1
   uint8_t* sV = sK + KV_STAGES * KV_TILE_BYTES;
-  uint8_t* sP = sV + KV_STAGES * KV_TILE_BYTES;        // sub-tile h (keys 64h .. 64h+63): sP + h * P_SUB_BYTES
-  __nv_bfloat16* xch = reinterpret_cast<__nv_bfloat16*>(sP + P_BYTES);        // [half][row]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sP + P_BYTES + ATTN_XCH_BYTES);
+  __nv_bfloat16* xch = reinterpret_cast<__nv_bfloat16*>(sV + KV_STAGES * KV_TILE_BYTES);   // [half][row] maxima
+  float* lx = reinterpret_cast<float*>(xch + 2 * 128);                                         // [half][row] sums
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sV + KV_STAGES * KV_TILE_BYTES + ATTN_XCH_BYTES);
   uint64_t* q_full = bars;                 // Q tile landed                       (one phase per item)
   uint64_t* q_empty = bars + 1;            // every S MMA of the item has read Q   (one phase per item)
   uint64_t* k_full = bars + 2;             // [stage]
@@ -202,7 +201,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   uint64_t* v_empty = v_full + KV_STAGES;  // [stage] O += P V of the tile has completed
   uint64_t* s_full = v_empty + KV_STAGES;  // S(t) is in tensor memory
   uint64_t* s_empty = s_full + 1;          // the softmax warps hold S(t) in registers
-  uint64_t* p_full = s_empty + 1;          // P(t) is in shared memory (and the accumulator rescaled, if it had to be)
+  uint64_t* p_full = s_empty + 1;          // P(t) is in tensor memory (and the accumulator rescaled, if it had to be)
   uint64_t* o_full = p_full + 1;           // O += P(t) V(t) has completed
   uint64_t* group_bar = o_full + 1;        // the eight softmax warps (slice hand-over)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(group_bar + 1);
@@ -342,14 +341,13 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           const int st = t % KV_STAGES;
           if (!mbar_wait(v_full + st, (t / KV_STAGES) & 1, abort_flag, p.status, 415)) goto done;
           tc_fence_after();
-          const uint32_t p_addr = smem_u32(sP);
           const uint32_t v_addr = smem_u32(sV + st * KV_TILE_BYTES);
-          const uint32_t d = tmem_base + 128;      // the item's accumulator: the first product of an item overwrites it
+          const uint32_t d = tmem_base + TMEM_COL_O;   // the item's accumulator: the first product of an item overwrites it
 #pragma unroll
-          for (int k = 0; k < 8; ++k)   // 16 keys per step: P sub-tile k / 4, 32 bytes along its rows; V [key][dim] is
-                                        // MN-major, a step of 16 keys is 16 rows of 128 bytes
-            umma_bf16(d, umma_desc_sw128(p_addr + (k >> 2) * P_SUB_BYTES + (k & 3) * 32),
-                      umma_desc_sw128(v_addr + k * 2048), idesc_pv, (j != 0 || k != 0) ? 1u : 0u);
+          for (int k = 0; k < 8; ++k)   // 16 keys per step: 8 columns of P in tensor memory; V [key][dim] is MN-major,
+                                        // a step of 16 keys is 16 rows of 128 bytes
+            umma_bf16_ta(d, tmem_base + TMEM_COL_P + k * 8, umma_desc_sw128(v_addr + k * 2048), idesc_pv,
+                         (j != 0 || k != 0) ? 1u : 0u);
           umma_commit(v_empty + st);
           umma_commit(o_full);
         }
@@ -364,7 +362,8 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int row = quarter * 32 + lane;               // q row of the tile = TMEM lane
     const int tok = row / p.group;
     const uint32_t t_lane = tmem_base + (uint32_t(quarter * 32) << 16);
-    const uint32_t t_o = t_lane + 128 + half * 32;     // this thread's 32 columns of the accumulator row
+    const uint32_t t_o = t_lane + TMEM_COL_O + half * 32;     // this thread's 32 columns of the accumulator row
+    const uint32_t t_p = t_lane + TMEM_COL_P + half * 32;     // and of the row of P: its 64 keys, two per column
     const float sc = 0.125f * 1.4426950408889634f;     // 1/sqrt(64) * log2(e)
     uint32_t t = 0, group_ph = 0;
     for (int r = 0; r < n_rounds; ++r) {
@@ -488,7 +487,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           pk[16 + e] = pack_bf16(a0, a1);
         }
         l = l * alpha + sum;
-        // P's buffer is read by the product of tile t - 1, which also still adds into the accumulator
+        // P's columns are read by the product of tile t - 1, which also still adds into the accumulator
         if (t > 0) {
           ok = mbar_wait(o_full, (t - 1) & 1, abort_flag, p.status, 421);
           if (!__all_sync(0xffffffffu, ok)) goto done;
@@ -505,13 +504,9 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           tmem_st_wait();
           tc_fence_before();
         }
-        // P row -> shared memory, sub-tile `half`, K-major 128B-swizzled: 16-byte chunk c of row r sits at chunk c ^ (r & 7)
-        uint8_t* prow = sP + half * P_SUB_BYTES + row * 128;
-#pragma unroll
-        for (int c = 0; c < 8; ++c)
-          *reinterpret_cast<uint4*>(prow + ((c ^ (row & 7)) << 4)) =
-              make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-        fence_proxy_async_smem();
+        // P row -> tensor memory, where the second product reads it as its A operand (no shared-memory round trip)
+        tmem_st32(t_p, pk);
+        tmem_st_wait();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(p_full);
@@ -522,14 +517,13 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (!__all_sync(0xffffffffu, ok)) goto done;
         tc_fence_after();
       }
-      // the row sum is the sum of its two threads' halves: exchanged through P's buffer, which nothing reads any more
+      // the row sum is the sum of its two threads' halves
       float l_row = l;
       if (warp_ok) {
-        float* lx = reinterpret_cast<float*>(sP);        // [2][128]
         lx[half * 128 + row] = l;
         named_bar_sync(1 + quarter, 64);                 // the two warps of this lane quarter
         l_row += lx[(half ^ 1) * 128 + row];
-        named_bar_sync(1 + quarter, 64);                 // both have read before either writes P again
+        named_bar_sync(1 + quarter, 64);                 // both have read before either writes the next item's
       }
 
       // ---- item epilogue: this thread owns dims [32 half, 32 half + 32) of its row
