@@ -73,9 +73,12 @@ extern "C" {
 #define HSD_FLAG_SIMT_DEBUG 1      /* run the plain SIMT kernels instead of the tensor-core kernels;
                                       a slow cross-check for debugging, never a fallback              */
 #define HSD_FLAG_SIMT_ATTENTION 2  /* debugging: only the attention runs through its plain kernel     */
-#define HSD_FLAG_DETERMINISTIC 4   /* no split-K in the residual-add projections: their K slices add into
+#define HSD_FLAG_DETERMINISTIC 4   /* no split-K in the residual-add projections (their K slices add into
                                       the fp32 residual in arrival order, so results can differ in the last
-                                      bit from run to run; with this flag every run is bit-identical      */
+                                      bit from run to run) and no KV slicing in the attention (where the cuts
+                                      fall depends on what else is in the batch): with this flag every run is
+                                      bit-identical and a row's result does not depend on the batch around it;
+                                      a single sequence over a long context then runs on few SMs            */
 #define HSD_FLAG_NO_PAIR 16        /* debugging: no CTA-pair (cluster of two) GEMM tiles                        */
 #define HSD_FLAG_NO_HOST_GRAPH 32  /* hsd_verify_regions_host launches its kernels one by one, never as a CUDA graph */
 #define HSD_FLAG_NO_PDL 8          /* debugging: plain stream-ordered launches (no programmatic dependent

@@ -277,7 +277,9 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
   if (!c->attn_simt) {
     Scope s(c, st, KC_SETUP);
     // items per launch: a few per CTA slot (two CTAs per SM), at least attn_min_chunk KV tiles each
-    launch_attn_plan(st, w.rm, w.plan, a.n_seqs, tokens_per_tile, max(1, c->attn_target_items / md.Hkv), c->attn_min_chunk,
+    // (a context with a fixed summation order never cuts a KV range: where the cuts fall depends on the batch)
+    launch_attn_plan(st, w.rm, w.plan, a.n_seqs, tokens_per_tile, max(1, c->attn_target_items / md.Hkv),
+                     c->max_splits == 1 ? (1 << 20) : c->attn_min_chunk,
                      w.status + 4, w.status, c->pdl);
   }
   if (!c->simt) {

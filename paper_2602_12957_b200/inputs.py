@@ -126,6 +126,29 @@ def make_weights(cfg: ModelConfig, seed: int) -> Dict[str, object]:
     return out
 
 
+def make_chain_weights(cfg: ModelConfig, seed: int, branch_scale: float = 0.004):
+    """Decoder weights whose greedy text is known in advance and decided by wide margins: (weights, order).
+
+    `order` is a random cyclic order of the vocabulary; after token order[i] the decoder emits order[i + 1].  The
+    weights are the random-init ones of `make_weights` except that the two projections that write into the residual
+    stream (w_o, w_down) are scaled by `branch_scale`, so the last token's embedding row dominates the stream, and
+    that the LM-head row of order[i + 1] is 4 x the embedding row of order[i] (the logit of the successor is the
+    squared norm of an embedding row over its RMS, about 80; every other logit is a cross product, within +-12).
+    Random-init weights have no such margins (half their rows have a top-1 / top-2 gap below 0.1), so a text decoded
+    with them changes with the summation order of a kernel; loops whose statistics depend on WHICH tokens come out
+    (accepted lengths over many steps) use these.  Every kernel runs the same dense arithmetic on them."""
+    w = make_weights(cfg, seed)
+    rng = np.random.Generator(np.random.PCG64(seed + 9_000_003))
+    order = rng.permutation(cfg.vocab).astype(np.int64)
+    for lw in w["layers"]:
+        lw["w_o"] = bf16_round(lw["w_o"] * np.float32(branch_scale))
+        lw["w_down"] = bf16_round(lw["w_down"] * np.float32(branch_scale))
+    lm = np.empty_like(w["lm_head"])
+    lm[np.roll(order, -1)] = w["embed"][order] * np.float32(4.0)       # exact in bf16
+    w["lm_head"] = lm
+    return w, order
+
+
 # --------------------------------------------------------------------------- workloads
 @dataclass
 class SeqInput:

@@ -136,3 +136,61 @@ def test_device_loop_follows_the_oracle_loop(log_tau):
     assert len(run.stage2.tokens[0]) == lengths[-1]
     print("oracle loop", log_tau, want.summary(), "device stage1 steps", run.stage1.steps.tolist(), "AAL",
           round(run.stage1.aal, 2), "checked tokens", checked)
+
+
+def _chain_page(cfg, order, seed, n_regions, p0=777):
+    """Crops and a page for the chain decoder: the last prompt token of every crop is set so that the page's text is
+    the concatenation of the regions' texts (what the method relies on)."""
+    wl = I.region_workload(seed=seed, n_regions=n_regions + 1, prefix_lo=70, prefix_hi=200, draft_mean=30, draft_lo=8,
+                           draft_hi=60, cfg=cfg)
+    rng = np.random.default_rng(seed)
+    lengths = [int(x) for x in rng.integers(20, 150, size=n_regions)]
+    offs = np.concatenate([[0], np.cumsum(lengths)]).astype(int)
+
+    def prefix(seq, pos):
+        ids = seq.prefix_ids.copy()
+        ids[-1] = order[pos % cfg.vocab]
+        return seq.prefix_embeds, ids
+    regions = [prefix(wl.seqs[i], p0 + offs[i]) for i in range(n_regions)]
+    page = prefix(wl.seqs[-1], p0)
+    walk = lambda start, n: order[(start + 1 + np.arange(n)) % cfg.vocab].astype(np.int32)
+    texts = [walk(p0 + offs[i], lengths[i]) for i in range(n_regions)]
+    return regions, page, lengths, texts, walk(p0, int(offs[-1])), rng
+
+
+@pytest.mark.parametrize("log_tau", [0.0, float(np.log(0.75))], ids=["greedy", "tau0.75"])
+def test_whole_hierarchy_on_a_decisive_decoder_equals_the_oracle_loop(log_tau):
+    """A decoder whose every decision has a wide margin (inputs.make_chain_weights): nothing is a near tie, so the device
+    loop and the oracle loop must agree on EVERYTHING — every region's text, the aggregated page draft, the page's
+    text decoded in Stage 2 against that draft (no stand-in), and per sequence the number of verification steps and
+    of accepted draft tokens.  The texts are also known in closed form (a walk along the decoder's token order)."""
+    from paper_2602_12957_b200 import driver as DR
+    from paper_2602_12957_b200 import runtime as R
+    cfg = I.small_decoder(2, 8192)
+    weights, order = I.make_chain_weights(cfg, 47)
+    regions, page, lengths, texts, page_text, rng = _chain_page(cfg, order, 47, 5)
+    drafts = [[_damaged(t, rng, max(1, len(t) // 7), cfg.vocab), _damaged(t, rng, max(1, len(t) // 5), cfg.vocab)]
+              for t in texts]
+    drafts[3] = [rng.integers(0, cfg.vocab, 40).astype(np.int32)]         # one region with a useless draft
+    model_o = O.Decoder(cfg, weights, np.float64)
+    want = T.hierarchical_decode(
+        model_o, [T.RegionInput(e, i, [d.tolist() for d in ds], n) for (e, i), ds, n in zip(regions, drafts, lengths)],
+        T.RegionInput(page[0], page[1], [], len(page_text)), n=3, max_rows=128, log_tau=log_tau)
+    # the oracle itself against the closed form
+    for tr, t in zip(want.region_traces, texts):
+        assert tr.tokens == t.tolist() and min(tr.token_gap) > 10.0
+    assert want.page_trace.tokens == page_text.tolist() and min(want.page_trace.token_gap) > 10.0
+    model = R.DeviceModel(cfg, weights, 0)
+    run = DR.run_page(model, regions, drafts, lengths, page, len(page_text), n_lanes=3, max_rows=128, log_tau=log_tau,
+                      steps_per_poll=4, seed=9, poison=True)
+    for r, tr in enumerate(want.region_traces):
+        assert run.stage1.tokens[r].tolist() == tr.tokens, f"region {r}"
+        assert run.page_draft[r].tolist() == tr.tokens
+        assert int(run.stage1.steps[r]) == tr.steps, f"region {r}: steps"
+        assert int(run.stage1.accepted[r]) == sum(tr.accepted_per_step), f"region {r}: accepted"
+    assert run.stage2.tokens[0].tolist() == want.page_trace.tokens
+    assert int(run.stage2.steps[0]) == want.page_trace.steps
+    assert int(run.stage2.accepted[0]) == sum(want.page_trace.accepted_per_step)
+    # Stage 2 really runs on the Stage-1 outputs: three plain steps after every region boundary, long runs between
+    assert want.page_trace.steps < len(page_text) / 4
+    print("decisive", log_tau, want.summary(), "device AAL", round(run.stage1.aal, 2), round(run.stage2.aal, 2))

@@ -183,3 +183,39 @@ def test_thresholded_acceptance_accepts_at_least_as_much():
     loose = O.verify_cached(seq, q[0], np.asarray(q[1:]), np.asarray(par), float(np.log(0.05)))
     assert loose.accept_len >= strict.accept_len
     assert loose.path[:strict.accept_len] == strict.path
+
+
+def test_chain_decoder_page_text_is_the_concatenation_and_stage2_step_count_is_closed_form():
+    """On the chain decoder (inputs.make_chain_weights) every text is a known walk along the token order, the page's
+    text is the concatenation of the regions' texts, and all tokens of the walk are distinct, so Stage 2's course is
+    fixed by the window rule alone.  The first token of region i's part of the page comes for free (the prefill's
+    token for i = 0, else the bonus token of the step that accepted the end of draft i - 1); two plain steps bring
+    the next two; then the window (n = 3) lies inside draft i and the remaining len_i - 3 tokens go 127 accepted + 1
+    bonus per step: ceil((len_i - 3) / 128) steps, as long as len_i >= 4 and (len_i - 3) is no multiple of 128 (then
+    the last bonus token would still belong to part i)."""
+    cfg = I.small_decoder(1, 4096)
+    weights, order = I.make_chain_weights(cfg, 11)
+    model = O.Decoder(cfg, weights, np.float64)
+    rng = np.random.default_rng(11)
+    lengths = [30, 140, 7, 300]
+    offs = np.concatenate([[0], np.cumsum(lengths)]).astype(int)
+    p0 = 50
+
+    def prefix(pos, L):
+        emb = I.bf16_round(rng.standard_normal((L, cfg.d_model)).astype(np.float32))
+        ids = np.full(L, -1, np.int32)
+        ids[-4:] = order[[5, 6, 7, pos % cfg.vocab]]
+        return emb, ids
+    walk = lambda start, n: order[(start + 1 + np.arange(n)) % cfg.vocab].tolist()
+    regions = []
+    for i, n in enumerate(lengths):
+        e, ids = prefix(p0 + offs[i], 20 + 3 * i)
+        regions.append(T.RegionInput(e, ids, [walk(p0 + offs[i], n)], n))        # exact drafts
+    e, ids = prefix(p0, 33)
+    res = T.hierarchical_decode(model, regions, T.RegionInput(e, ids, [], int(offs[-1])), n=3, max_rows=128)
+    for i, tr in enumerate(res.region_traces):
+        assert tr.tokens == walk(p0 + offs[i], lengths[i])
+    assert res.page_draft == [walk(p0 + offs[i], n) for i, n in enumerate(lengths)]
+    assert res.page_trace.tokens == walk(p0, int(offs[-1]))
+    want_steps = sum(2 + -(-(n - 3) // 128) for n in lengths)
+    assert res.page_trace.steps == want_steps, (res.page_trace.steps, want_steps, res.page_trace.accepted_per_step)
