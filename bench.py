@@ -35,10 +35,14 @@ METRIC = "draft tokens verified per second (verify step: forward over paged pref
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM traffic per launch of the dominant kernel classes of the region workload, from the ncu captures summarised
-# under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); a class is absent (-> null) when its kernel has
-# changed since its counters were taken.
-NCU_TRAFFIC_BYTES = {}
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel classes, from the ncu
+# captures summarised under profiles/, per workload; a class is absent (-> null) when its kernel has changed since
+# its counters were taken, or when no capture of that workload exists.
+NCU_TRAFFIC_BYTES = {
+    "region": {"attention": 30_961_408 + 11_008, "gemm_gate_up": 19_521_792 + 256, "gemm_qkv": 7_282_432,
+               "gemm_o": 10_249_728, "gemm_down": 24_669_184 + 768},
+    "long2048": {"attention": 43_087_104 + 4_455_424},
+}
 
 
 def load_peaks():
@@ -670,7 +674,7 @@ def run_ours(args):
     prof_steps = max(3, min(args.steps, 30))
     prof = runner.profile(prof_steps)
     roof, step_roof, kernels, ctx_lens = roofline_report(st, prof, prof_steps, ms_step, clocks, peaks, peak_src,
-                                                         NCU_TRAFFIC_BYTES if args.workload == "region" else None)
+                                                         NCU_TRAFFIC_BYTES.get(args.workload))
 
     # ---- one step of every other configuration (one GPU only; the other ranks would only repeat it)
     extra = {}
@@ -682,7 +686,7 @@ def run_ours(args):
             r2 = Runner(st2, stream, use_graph=not args.no_graph, warmup=3)
             ms2, clk2, n2 = r2.timed(20, barrier, uuid, min_seconds=1.0)
             pr2 = r2.profile(5)
-            roof2, sroof2, kern2, ctx2 = roofline_report(st2, pr2, 5, ms2, clk2, peaks, peak_src)
+            roof2, sroof2, kern2, ctx2 = roofline_report(st2, pr2, 5, ms2, clk2, peaks, peak_src, NCU_TRAFFIC_BYTES.get(name))
             tok2 = r2.draft_tokens()
             extra[name] = {"workload": WORKLOADS[name], "ms_per_step": ms2, "steps": n2, "tokens_per_s": tok2 / (ms2 * 1e-3),
                            "draft_tokens": tok2, "query_rows": st2["total_q"], "context_tokens": int(sum(ctx2)),
@@ -690,7 +694,8 @@ def run_ours(args):
                            "step_roofline_frac": sroof2["frac"], "step_roofline_frac_of_burst": sroof2["frac_of_burst"],
                            "step_roofline_frac_of_sustained": sroof2["frac_of_sustained"], "step_bound": sroof2["bound"],
                            "top_kernel": roof2["kernel"], "top_kernel_bound": roof2["bound"],
-                           "top_kernel_frac": roof2["frac"], "top_kernel_us": roof2["us_per_launch"], "clocks": clk2,
+                           "top_kernel_frac": roof2["frac"], "top_kernel_us": roof2["us_per_launch"],
+                           "top_kernel_traffic": roof2["traffic"], "clocks": clk2,
                            "kernels": {k: {"ms_per_step": round(v["ms_per_step"], 4),
                                            "roofline_frac": round(v.get("roofline_frac", 0.0), 3)} for k, v in kern2.items()}}
             if not args.no_cpu_baseline and name != "tree":      # (the oracle's tree form is not timed)
