@@ -10,6 +10,13 @@
  * KV maintenance after the step (commit of the accepted rows, rollback of the rest; counted in T_decode,
  * Sec. 4.2) is a separate call.
  *
+ * Beside the chain form there is the paper's general operator and the loop around it: hsd_dsv_build (reference
+ * window, matching, prefix tree and its packing, Eq. 5-7), hsd_verify_tree / hsd_kv_commit_tree (candidate
+ * trees under the ancestry mask, greedy traversal, compaction of the accepted path, Eq. 8-12), and
+ * hsd_stage_begin / hsd_stage_advance / hsd_stage_aggregate (outputs, retirement and lane hand-over of the two
+ * stages and the page draft, Sec. 3.1, Eq. 2-4): a whole stage runs as stream-ordered calls of fixed shape,
+ * with no host decision between steps.
+ *
  * Conventions
  *  - All functions return an int status: HSD_OK (0) or a negative HSD_ERR_* code.  Nothing throws.
  *  - "dev" pointers are CUDA device pointers on the current device; "host" pointers are ordinary memory.

@@ -33,7 +33,9 @@ Pins (tests/test_oracle_*.py): Hugging Face's Llama decoder as a library routine
 whole forward; torch's scaled_dot_product_attention / rms_norm / silu; closed forms for
 RoPE, RMSNorm and uniform-key attention; one verify call == k+1 single-token steps;
 brute-force enumeration of all drafts on a tiny vocabulary against a literal tree walk;
-the step-count identity the paper's printed numbers satisfy.  No function is unpinned.
+the step-count identity the paper's printed numbers satisfy; the input rows (token rows
+from the table, visual rows from the caller, id 0 a token) against the library decoder's
+own embedding module fed with input_ids.  No function is unpinned.
 """
 from __future__ import annotations
 
