@@ -105,28 +105,16 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 // One probe of the barrier.  The suspend-time hint lets the hardware park the warp until the phase completes
 // (or the hint expires) instead of returning at once: a parked warp takes no issue slots from the warps that
 // share its scheduler, which matters because most warps of these kernels spend most of their time waiting.
-#ifndef HSD_TRYWAIT_HINT_NS
-#define HSD_TRYWAIT_HINT_NS 20000u
-#endif
+constexpr uint32_t kTryWaitHintNs = 20000u;      // (1 us .. 100 us measured alike)
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
-#ifdef HSD_MBAR_TEST_WAIT
-  asm volatile(
-      "{\n\t.reg .pred P;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
-      "selp.b32 %0, 1, 0, P;\n\t}\n"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-#else
   asm volatile(
       "{\n\t.reg .pred P;\n\t"
       "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2, %3;\n\t"
       "selp.b32 %0, 1, 0, P;\n\t}\n"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity), "r"(HSD_TRYWAIT_HINT_NS)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(kTryWaitHintNs)
       : "memory");
-#endif
   return ok != 0;
 }
 

@@ -85,6 +85,8 @@ int make_weight_tmaps(WeightMaps* w, const void* base, uint64_t rows, uint64_t c
 }
 
 // ------------------------------------------------------------------------------------------------
+// K extent of a pipeline stage in 64-column sub-tiles.  Two (one barrier round trip per eight MMAs instead of four)
+// measured the same cycles per k-block as one: with 256-wide tiles the main loop runs at the tensor pipes' rate.
 #ifndef HSD_GEMM_KSTEPS
 #define HSD_GEMM_KSTEPS 1
 #endif
@@ -596,10 +598,11 @@ static int launch_one(cudaStream_t st, const GemmSm100Args& a, int splits) {
 }
 
 // Tile width, CTA pairing and K slices: fewest cycles by a model calibrated on B200 (cycles per k-block of one work
-// unit, measured in steady state: 128 x 256 tile ~820, 128 x 128 ~700, 128 x 64 ~600, CTA pair on 256 x 256 ~770 per
-// CTA for twice the rows).  None of them reaches the 512 clocks the MMAs of a 256-column tile take: the pipeline is
-// bound by the round trip stage-free -> TMA issue -> data -> MMA over the few stages shared memory holds.  A pair
-// costs a cluster launch; the epilogue of the last unit of a CTA is exposed.
+// unit, measured in steady state with every SM busy: 128 x 256 tile ~820, 128 x 128 ~700, 128 x 64 ~600, CTA pair on
+// 256 x 256 ~770 per CTA for twice the rows).  The 256-wide shapes run at the rate the whole chip's tensor pipes
+// sustain (the measured library peak corresponds to ~730 cycles for such a k-block; one SM alone would need 544); the
+// narrower ones are bound by L2 -> SM bytes.  A pair costs a cluster launch; the epilogue of the last unit of a CTA is
+// exposed.
 static void pick_tile(int mode, int n_cols, int M, int K, int n_sms, int max_splits, bool allow_pair, int* bn_out,
                       int* splits_out, bool* pair_out) {
   const int k_blocks = K / BK;
