@@ -39,7 +39,7 @@
  *      embed, lm_head [vocab, d_model];  *_norm [d_model] (bf16 gains)
  *  - Paged KV pool, block = kv_block (64) tokens:
  *      k_pool, v_pool bf16 [n_layers][n_blocks][n_kv_heads][64 tokens][head_dim]
- *    (one 128-byte line per token and kv head; a (block, kv head) tile is 8 KB contiguous)
+ *    (one row of head_dim bf16 per token and kv head: 128 or 256 bytes; a (block, kv head) tile is contiguous)
  *    block_table int32 [n_slots, max_blocks_per_seq]: physical block of logical block j of slot s.
  *    seq_lens int32 [n_slots]: committed K/V rows per slot.
  *  - Packed query tokens: q_tokens[cu_q[i] .. cu_q[i+1]) = [pending_i, d_i1 .. d_ik].
@@ -128,7 +128,7 @@ HSD_API const char *hsd_status_string(int status);
 
 /* Create a context for one model on the current device.  Copies the configuration and the weight POINTERS
  * (not the weights) and builds the TMA tensor maps of the weights.  Errors: INVALID_ARG, SHAPE (requires
- * head_dim == 64, kv_block == 64, n_heads a multiple of n_kv_heads with a ratio that divides 128, d_model one of
+ * head_dim 64 or 128 (128 not together with the HSD_FLAG_SIMT_* cross-check kernels), kv_block == 64, n_heads a multiple of n_kv_heads with a ratio that divides 128, d_model one of
  * 128, 256, 512, 1024, 2048, 4096, d_ffn and vocab multiples of 64),
  * NO_DEVICE, CUDA.  No stream work is issued. */
 HSD_API int hsd_create(const hsd_model_config *cfg, const hsd_weights *w, hsd_ctx **out);

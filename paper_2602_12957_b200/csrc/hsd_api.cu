@@ -290,12 +290,14 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
     if (make_tmap_2d_f32(&tm_x_add, w.x, T, md.d, 32) || make_tmap_2d(&tm_q_st, w.q, T, md.Hq * md.D, 32) ||
         make_tmap_2d(&tm_act_st, w.act, T, md.ffn, 32))
       return HSD_ERR_CUDA;
-    // q as [T][Hq][64]: one box = (128/group) tokens x group heads x 64 dims -> a 128-row MMA operand
-    if (make_tmap_3d(&tm_q, w.q, 64, md.Hq, T, 128, (uint64_t)md.Hq * 128, 64, md.group, tokens_per_tile))
+    // q as [T][Hq][D]: one box = (128/group) tokens x group heads x 64 dims -> a 128-row MMA operand (head_dim 128:
+    // two boxes, one per half of the dims)
+    if (make_tmap_3d(&tm_q, w.q, md.D, md.Hq, T, (uint64_t)md.D * 2, (uint64_t)md.Hq * md.D * 2, 64, md.group,
+                     tokens_per_tile))
       return HSD_ERR_CUDA;
-    // K / V pools as 2-D [rows, 64]: one (layer, block, kv head) tile = 64 consecutive rows
+    // K / V pools as 2-D [rows, D]: one (layer, block, kv head) tile = 64 consecutive rows, fetched 64 dims at a time
     const uint64_t pool_rows = (uint64_t)md.n_layers * kv.n_blocks * md.Hkv * 64;
-    if (make_tmap_2d(&tm_k, kv.k_pool, pool_rows, 64, 64) || make_tmap_2d(&tm_v, kv.v_pool, pool_rows, 64, 64))
+    if (make_tmap_2d(&tm_k, kv.k_pool, pool_rows, md.D, 64) || make_tmap_2d(&tm_v, kv.v_pool, pool_rows, md.D, 64))
       return HSD_ERR_CUDA;
   }
 
@@ -305,7 +307,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
       launch_rmsnorm(st, w.x, c->attn_norm[l], w.h, T, md.d, md.eps, nullptr, T, w.status, c->pdl);
     }
     if (int rc = tap(l, HSD_TAP_H_ATTN, w.h, 2 * row_d)) return rc;
-    const size_t layer_elems = (size_t)kv.n_blocks * md.Hkv * 64 * 64;
+    const size_t layer_elems = (size_t)kv.n_blocks * md.Hkv * 64 * md.D;
     if (c->simt) {
       {
         Scope s(c, st, KC_GEMM_QKV);
@@ -332,14 +334,14 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
         g.tmA = tm_h;
         g.tmB = &c->tm_qkv[l];
         g.tmC = tm_q_st;
-        g.M = T; g.n_out = md.qkv_out; g.K = md.d; g.mode = GS_QKV_ROPE;
+        g.M = T; g.n_out = md.qkv_out; g.K = md.d; g.mode = md.D == 128 ? GS_QKV_ROPE128 : GS_QKV_ROPE;
         g.qkv.row_kv = w.rm.row_kv;
         g.qkv.kv_rows = kv.n_blocks * HSD_KV_BLOCK;
         g.qkv.rope_cs = w.rm.rope_cs;
         g.qkv.q_out = w.q;
         g.qkv.k_pool_layer = kv.k_pool + (size_t)l * layer_elems;
         g.qkv.v_pool_layer = kv.v_pool + (size_t)l * layer_elems;
-        g.qkv.Hq = md.Hq; g.qkv.Hkv = md.Hkv;
+        g.qkv.Hq = md.Hq; g.qkv.Hkv = md.Hkv; g.qkv.D = md.D;
         g.qkv.q_norm = c->q_norm[l]; g.qkv.k_norm = c->k_norm[l]; g.qkv.eps = md.eps;
         g.status = w.status; g.n_sms = c->n_sms; g.device = c->device; g.max_splits = 1; g.pdl = c->pdl; g.pair = c->pair;
         g.force_bn = c->force_bn;
@@ -502,7 +504,9 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
   if (cfg->n_layers <= 0 || cfg->d_model <= 0 || cfg->n_heads <= 0 || cfg->n_kv_heads <= 0 || cfg->d_ffn <= 0 ||
       cfg->vocab <= 0)
     return HSD_ERR_INVALID_ARG;
-  if (cfg->head_dim != 64 || cfg->kv_block != HSD_KV_BLOCK) return HSD_ERR_SHAPE;
+  if ((cfg->head_dim != 64 && cfg->head_dim != 128) || cfg->kv_block != HSD_KV_BLOCK) return HSD_ERR_SHAPE;
+  // the plain cross-check kernels exist for head_dim 64 only
+  if (cfg->head_dim != 64 && (cfg->flags & (HSD_FLAG_SIMT_DEBUG | HSD_FLAG_SIMT_ATTENTION))) return HSD_ERR_SHAPE;
   if (cfg->n_heads % cfg->n_kv_heads) return HSD_ERR_SHAPE;
   const int group = cfg->n_heads / cfg->n_kv_heads;
   if (128 % group) return HSD_ERR_SHAPE;
@@ -530,8 +534,8 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
   if (!c) return HSD_ERR_INVALID_ARG;
   c->cfg = *cfg;
   ModelDims& md = c->md;
-  md.n_layers = cfg->n_layers; md.d = cfg->d_model; md.Hq = cfg->n_heads; md.Hkv = cfg->n_kv_heads; md.D = 64;
-  md.ffn = cfg->d_ffn; md.V = cfg->vocab; md.qkv_out = (md.Hq + 2 * md.Hkv) * 64; md.group = group;
+  md.n_layers = cfg->n_layers; md.d = cfg->d_model; md.Hq = cfg->n_heads; md.Hkv = cfg->n_kv_heads; md.D = cfg->head_dim;
+  md.ffn = cfg->d_ffn; md.V = cfg->vocab; md.qkv_out = (md.Hq + 2 * md.Hkv) * md.D; md.group = group;
   md.rope_base = cfg->rope_base; md.eps = cfg->rms_eps;
   c->embed = static_cast<const bf16*>(w->embed);
   c->lm_head = static_cast<const bf16*>(w->lm_head);
@@ -575,7 +579,7 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
     int bad = 0;
     for (int l = 0; l < md.n_layers; ++l) {
       bad |= make_weight_tmaps(&c->tm_qkv[l], c->w_qkv[l], md.qkv_out, md.d);
-      bad |= make_weight_tmaps(&c->tm_o[l], c->w_o[l], md.d, md.Hq * 64);
+      bad |= make_weight_tmaps(&c->tm_o[l], c->w_o[l], md.d, md.Hq * md.D);
       bad |= make_weight_tmaps(&c->tm_gate_up[l], c->w_gate_up[l], 2 * md.ffn, md.d);
       bad |= make_weight_tmaps(&c->tm_down[l], c->w_down[l], md.d, md.ffn);
     }
@@ -786,7 +790,7 @@ int hsd_kv_commit_tree(hsd_ctx* c, const hsd_kv* kv, int n_seqs, const int* seq_
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   {
     Scope s(c, st, KC_COMMIT);
-    launch_tree_compact(st, kv_view(kv), c->md.n_layers, c->md.Hkv, n_seqs, seq_slots, accept_len, accept_rows, max_q_len,
+    launch_tree_compact(st, kv_view(kv), c->md.n_layers, c->md.Hkv, c->md.D, n_seqs, seq_slots, accept_len, accept_rows, max_q_len,
                         c->pdl);
   }
   {

@@ -37,24 +37,33 @@ namespace hsd {
 constexpr int kSoftmaxWarps = 8;
 constexpr int kAttnThreads = 32 * (2 + kSoftmaxWarps);
 constexpr int KV_STAGES = 2;                       // per ring
-constexpr int Q_BYTES = 128 * 128;
-constexpr int KV_BLOCK_BYTES = 64 * 128;           // one paged block of K or of V for one kv head
-constexpr int KV_TILE_BYTES = 2 * KV_BLOCK_BYTES;  // 128 keys
+constexpr int SUB_BYTES = 128 * 128;               // one K-major operand sub-tile: 128 rows (q rows / keys) x 64 dims
+constexpr int KV_BLOCK_BYTES = 64 * 128;           // one paged block of K or of V for one kv head, 64 dims of it
 constexpr int ATTN_BAR_BYTES = 256;
 constexpr int ATTN_XCH_BYTES = 2 * 128 * 2 + 2 * 128 * 4;   // per (half, row): the tile's half-row maximum (bf16); the item's half-row sum (fp32)
-// No alignment slack: two CTAs of this size plus the per-CTA reserve just fit an SM, so the kernel relies on the
-// 1024-byte alignment it declares for its dynamic shared memory (the swizzled tiles need it) and checks it.
-constexpr int ATTN_SMEM = Q_BYTES + 2 * KV_STAGES * KV_TILE_BYTES + ATTN_XCH_BYTES + ATTN_BAR_BYTES;
-constexpr int ATTN_TMEM_COLS = 256;                // S: 128 fp32 columns, O: 64, P: 64 (128 keys, two bf16 per column)
-constexpr int TMEM_COL_O = 128, TMEM_COL_P = 192;
 constexpr float kRescaleBits = 8.f;
+// Head dimension HD = 64 or 128.  An operand tile is HD / 64 sub-tiles of 64 dims each (a 128-byte-swizzled row is 64
+// bf16): Q [sub][128 rows][64], a K or V stage [sub][block 0, block 1][64 keys][64].  The accumulator has HD columns.
+// No alignment slack: with HD = 64 two CTAs of this size plus the per-CTA reserve share an SM, so the kernel relies
+// on the 1024-byte alignment it declares for its dynamic shared memory (the swizzled tiles need it) and checks it.
+template <int HD>
+struct AttnCfg {
+  static constexpr int NSUB = HD / 64;
+  static constexpr int Q_BYTES = NSUB * SUB_BYTES;
+  static constexpr int KV_TILE_BYTES = NSUB * SUB_BYTES;           // 128 keys
+  static constexpr int SMEM = Q_BYTES + 2 * KV_STAGES * KV_TILE_BYTES + ATTN_XCH_BYTES + ATTN_BAR_BYTES;
+  static constexpr int COL_O = 128, COL_P = 128 + HD;              // S: 128 fp32 columns, O: HD, P: 64 (two keys per column)
+  static constexpr int TMEM_COLS = HD == 64 ? 256 : 512;           // allocations are powers of two
+  static constexpr int CTAS_PER_SM = HD == 64 ? 2 : 1;             // tensor memory has 512 columns
+  static constexpr int OWN = HD / 2;                               // accumulator columns of one softmax thread
+};
 
 struct AttnParams {
   AttnPlan plan;
   const int* block_table;
   int max_blocks, n_blocks, Hq, Hkv, group, layer;
-  bf16* out;            // [T, Hq*64]
-  float* split_ws;      // partials of sliced items: [q-tile][kv head][slice][2 + 64][128 rows]
+  bf16* out;            // [T, Hq*HD]
+  float* split_ws;      // partials of sliced items: [q-tile][kv head][slice][2 + HD][128 rows]
   const uint4* anc;     // [T] ancestry masks of candidate-tree rows, or nullptr: plain causal order within the call
   int* status;
 };
@@ -183,12 +192,16 @@ void launch_attn_plan(cudaStream_t st, const RowMeta& rm, const AttnPlan& pl, in
 }
 
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kAttnThreads, 2)
+template <int HD>
+__global__ void __launch_bounds__(kAttnThreads, AttnCfg<HD>::CTAS_PER_SM)
 attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, AttnParams p) {
+  using C = AttnCfg<HD>;
+  constexpr int Q_BYTES = C::Q_BYTES, KV_TILE_BYTES = C::KV_TILE_BYTES, NSUB = C::NSUB;
+  constexpr int TMEM_COL_O = C::COL_O, TMEM_COL_P = C::COL_P, OWN = C::OWN;
   extern __shared__ __align__(1024) uint8_t smem[];
   uint8_t* sQ = smem;
-  uint8_t* sK = sQ + Q_BYTES;                          // ring stage s: sK + s * KV_TILE_BYTES, block 0 then block 1
+  uint8_t* sK = sQ + Q_BYTES;                          // ring stage s: sK + s * KV_TILE_BYTES, per sub-tile block 0 then block 1
   uint8_t* sV = sK + KV_STAGES * KV_TILE_BYTES;
   __nv_bfloat16* xch = reinterpret_cast<__nv_bfloat16*>(sV + KV_STAGES * KV_TILE_BYTES);   // [half][row] maxima
   float* lx = reinterpret_cast<float*>(xch + 2 * 128);                                         // [half][row] sums
@@ -234,7 +247,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     tma_prefetch_desc(&tmV);
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, ATTN_TMEM_COLS);
+    tmem_alloc(tmem_slot, C::TMEM_COLS);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -287,7 +300,8 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (is_k) {
           if (!mbar_wait(q_empty, (n & 1) ^ 1u, abort_flag, p.status, 400)) goto done;
           mbar_expect_tx(q_full, Q_BYTES);
-          tma_load_3d(sQ, &tmQ, q_full, 0, kvh * p.group, ia.x);
+#pragma unroll
+          for (int h = 0; h < NSUB; ++h) tma_load_3d(sQ + h * SUB_BYTES, &tmQ, q_full, 64 * h, kvh * p.group, ia.x);
         }
         for (int kt = kt_lo; kt < kt_hi; kt += 2, ++t) {
           // the tile's two blocks; a slice of odd length ends with half a tile: the last block is staged twice and
@@ -299,8 +313,11 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           const int row1 = (((p.layer * p.n_blocks) + phys1) * p.Hkv + kvh) * 64;
           uint8_t* dst = ring + st * KV_TILE_BYTES;
           mbar_expect_tx(full + st, KV_TILE_BYTES);
-          tma_load_2d(dst, tm, full + st, 0, row0);
-          tma_load_2d(dst + KV_BLOCK_BYTES, tm, full + st, 0, row1);
+#pragma unroll
+          for (int h = 0; h < NSUB; ++h) {
+            tma_load_2d(dst + h * SUB_BYTES, tm, full + st, 64 * h, row0);
+            tma_load_2d(dst + h * SUB_BYTES + KV_BLOCK_BYTES, tm, full + st, 64 * h, row1);
+          }
         }
         ++n;
       }
@@ -317,7 +334,7 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (w < 0) continue;
         const int4 ib = p.plan.items[2 * (w / p.Hkv) + 1];
         const int n_it = ((ib.x >> 16) - (ib.x & 0xffff) + 1) / 2;      // 128-key tiles of the item
-        // S(ti) = Q K(ti)^T: four K = 16 steps over the 64 dims, N = 128 keys
+        // S(ti) = Q K(ti)^T: four K = 16 steps over every 64 dims, N = 128 keys
         auto issue_s = [&](uint32_t ti, bool last) -> bool {
           const int st = ti % KV_STAGES;
           if (!mbar_wait(k_full + st, (ti / KV_STAGES) & 1, abort_flag, p.status, 410)) return false;
@@ -325,8 +342,11 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           tc_fence_after();
           const uint32_t k_addr = smem_u32(sK + st * KV_TILE_BYTES);
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            umma_bf16(tmem_base, umma_desc_sw128(q_addr + k * 32), umma_desc_sw128(k_addr + k * 32), idesc_s, k != 0);
+          for (int h = 0; h < NSUB; ++h)
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              umma_bf16(tmem_base, umma_desc_sw128(q_addr + h * SUB_BYTES + k * 32),
+                        umma_desc_sw128(k_addr + h * SUB_BYTES + k * 32), idesc_s, (h | k) != 0);
           umma_commit(s_full);
           umma_commit(k_empty + st);              // K is free once S has been formed
           if (last) umma_commit(q_empty);         // last S MMA of the item: Q is free once it completes
@@ -344,10 +364,12 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           const uint32_t v_addr = smem_u32(sV + st * KV_TILE_BYTES);
           const uint32_t d = tmem_base + TMEM_COL_O;   // the item's accumulator: the first product of an item overwrites it
 #pragma unroll
-          for (int k = 0; k < 8; ++k)   // 16 keys per step: 8 columns of P in tensor memory; V [key][dim] is MN-major,
-                                        // a step of 16 keys is 16 rows of 128 bytes
-            umma_bf16_ta(d, tmem_base + TMEM_COL_P + k * 8, umma_desc_sw128(v_addr + k * 2048), idesc_pv,
-                         (j != 0 || k != 0) ? 1u : 0u);
+          for (int h = 0; h < NSUB; ++h)   // 64 output dims per product
+#pragma unroll
+            for (int k = 0; k < 8; ++k)    // 16 keys per step: 8 columns of P in tensor memory; V [key][dim] is MN-major,
+                                           // a step of 16 keys is 16 rows of 128 bytes
+              umma_bf16_ta(d + 64 * h, tmem_base + TMEM_COL_P + k * 8, umma_desc_sw128(v_addr + h * SUB_BYTES + k * 2048),
+                           idesc_pv, (j != 0 || k != 0) ? 1u : 0u);
           umma_commit(v_empty + st);
           umma_commit(o_full);
         }
@@ -362,9 +384,9 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int row = quarter * 32 + lane;               // q row of the tile = TMEM lane
     const int tok = row / p.group;
     const uint32_t t_lane = tmem_base + (uint32_t(quarter * 32) << 16);
-    const uint32_t t_o = t_lane + TMEM_COL_O + half * 32;     // this thread's 32 columns of the accumulator row
+    const uint32_t t_o = t_lane + TMEM_COL_O + half * OWN;    // this thread's OWN columns of the accumulator row
     const uint32_t t_p = t_lane + TMEM_COL_P + half * 32;     // and of the row of P: its 64 keys, two per column
-    const float sc = 0.125f * 1.4426950408889634f;     // 1/sqrt(64) * log2(e)
+    const float sc = (HD == 64 ? 0.125f : 0.08838834764831845f) * 1.4426950408889634f;     // 1/sqrt(HD) * log2(e)
     uint32_t t = 0, group_ph = 0;
     for (int r = 0; r < n_rounds; ++r) {
       const int w = item_of_round(r);
@@ -495,12 +517,15 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         }
         if (__any_sync(0xffffffffu, rescale)) {
           // rare: scale this thread's half of the accumulator row (alpha = 1 where not needed)
-          uint32_t o[32];
-          tmem_ld32(t_o, o);
-          tmem_ld_wait();
+#pragma unroll 1
+          for (int c = 0; c < OWN; c += 32) {
+            uint32_t o[32];
+            tmem_ld32(t_o + c, o);
+            tmem_ld_wait();
 #pragma unroll
-          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-          tmem_st32(t_o, o);
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st32(t_o + c, o);
+          }
           tmem_st_wait();
           tc_fence_before();
         }
@@ -526,42 +551,50 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         named_bar_sync(1 + quarter, 64);                 // both have read before either writes the next item's
       }
 
-      // ---- item epilogue: this thread owns dims [32 half, 32 half + 32) of its row
+      // ---- item epilogue: this thread owns dims [OWN half, OWN half + OWN) of its row
       const int head = kvh * p.group + row % p.group;
+      uint4* out_row = reinterpret_cast<uint4*>(p.out + (size_t)(q_row0 + tok) * p.Hq * HD + head * HD + half * OWN);
       if (n_split == 1) {
         if (warp_ok) {                                     // (a whole warp reads tensor memory together)
           const float inv = 1.f / l_row;
-          uint32_t o[32];
-          tmem_ld32(t_o, o);
-          tmem_ld_wait();
-          tc_fence_before();
-          if (row_ok) {
-            uint4* dst = reinterpret_cast<uint4*>(p.out + (size_t)(q_row0 + tok) * p.Hq * 64 + head * 64 + half * 32);
+#pragma unroll 1
+          for (int c0 = 0; c0 < OWN; c0 += 32) {
+            uint32_t o[32];
+            tmem_ld32(t_o + c0, o);
+            tmem_ld_wait();
+            if (row_ok) {
+              uint4* dst = out_row + c0 / 8;
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
-              dst[c] = make_uint4(
-                  pack_bf16(__uint_as_float(o[8 * c]) * inv, __uint_as_float(o[8 * c + 1]) * inv),
-                  pack_bf16(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv),
-                  pack_bf16(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv),
-                  pack_bf16(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv));
+              for (int c = 0; c < 4; ++c)
+                dst[c] = make_uint4(
+                    pack_bf16(__uint_as_float(o[8 * c]) * inv, __uint_as_float(o[8 * c + 1]) * inv),
+                    pack_bf16(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv),
+                    pack_bf16(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv),
+                    pack_bf16(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv));
+            }
           }
+          tc_fence_before();
         }
       } else {
-        // partials of this (q-tile, kv head): [slice][66][128 rows] floats, entry 0 the exponent reference (log2
-        // units), 1 the row sum under it, 2.. the 64 unnormalised outputs; a warp's accesses are 128-byte lines
-        float* tile_part = p.split_ws + ((size_t)(ib.z * p.Hkv + kvh) * kAttnMaxSplits) * (66 * 128) + row;
+        // partials of this (q-tile, kv head): [slice][2 + HD][128 rows] floats, entry 0 the exponent reference (log2
+        // units), 1 the row sum under it, 2.. the HD unnormalised outputs; a warp's accesses are 128-byte lines
+        constexpr int PART = (2 + HD) * 128;
+        float* tile_part = p.split_ws + ((size_t)(ib.z * p.Hkv + kvh) * kAttnMaxSplits) * PART + row;
         if (warp_ok) {
-          float* part = tile_part + (size_t)split * (66 * 128);
+          float* part = tile_part + (size_t)split * PART;
           if (half == 0) {
             part[0] = m_ref;
             part[128] = l_row;
           }
-          uint32_t o[32];
-          tmem_ld32(t_o, o);
-          tmem_ld_wait();
-          tc_fence_before();
+#pragma unroll 1
+          for (int c0 = 0; c0 < OWN; c0 += 32) {
+            uint32_t o[32];
+            tmem_ld32(t_o + c0, o);
+            tmem_ld_wait();
 #pragma unroll
-          for (int e = 0; e < 32; ++e) part[(2 + half * 32 + e) * 128] = __uint_as_float(o[e]);
+            for (int e = 0; e < 32; ++e) part[(2 + half * OWN + c0 + e) * 128] = __uint_as_float(o[e]);
+          }
+          tc_fence_before();
         }
         __threadfence();
         if (!warps_sync(group_bar, group_ph, lane, abort_flag, p.status, 427)) goto done;
@@ -575,26 +608,29 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (*s_flag && warp_ok) {
           __threadfence();
           float M = -INFINITY;
-          for (int s = 0; s < n_split; ++s) M = fmaxf(M, __ldcg(tile_part + (size_t)s * (66 * 128)));
-          float Lsum = 0.f;
-          float o[32];
+          for (int s = 0; s < n_split; ++s) M = fmaxf(M, __ldcg(tile_part + (size_t)s * PART));
+#pragma unroll 1
+          for (int c0 = 0; c0 < OWN; c0 += 32) {
+            float Lsum = 0.f;
+            float o[32];
 #pragma unroll
-          for (int e = 0; e < 32; ++e) o[e] = 0.f;
-          for (int s = 0; s < n_split; ++s) {             // fixed slice order: the result does not depend on arrival
-            const float* ps = tile_part + (size_t)s * (66 * 128);
-            const float mxs = __ldcg(ps);
-            const float wgt = (mxs == -INFINITY) ? 0.f : ex2(mxs - M);
-            Lsum += wgt * __ldcg(ps + 128);
+            for (int e = 0; e < 32; ++e) o[e] = 0.f;
+            for (int s = 0; s < n_split; ++s) {           // fixed slice order: the result does not depend on arrival
+              const float* ps = tile_part + (size_t)s * PART;
+              const float mxs = __ldcg(ps);
+              const float wgt = (mxs == -INFINITY) ? 0.f : ex2(mxs - M);
+              Lsum += wgt * __ldcg(ps + 128);
 #pragma unroll
-            for (int e = 0; e < 32; ++e) o[e] += wgt * __ldcg(ps + (2 + half * 32 + e) * 128);
-          }
-          if (row_ok) {
-            const float inv = 1.f / Lsum;
-            uint4* dst = reinterpret_cast<uint4*>(p.out + (size_t)(q_row0 + tok) * p.Hq * 64 + head * 64 + half * 32);
+              for (int e = 0; e < 32; ++e) o[e] += wgt * __ldcg(ps + (2 + half * OWN + c0 + e) * 128);
+            }
+            if (row_ok) {
+              const float inv = 1.f / Lsum;
+              uint4* dst = out_row + c0 / 8;
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
-              dst[c] = make_uint4(pack_bf16(o[8 * c] * inv, o[8 * c + 1] * inv), pack_bf16(o[8 * c + 2] * inv, o[8 * c + 3] * inv),
-                                  pack_bf16(o[8 * c + 4] * inv, o[8 * c + 5] * inv), pack_bf16(o[8 * c + 6] * inv, o[8 * c + 7] * inv));
+              for (int c = 0; c < 4; ++c)
+                dst[c] = make_uint4(pack_bf16(o[8 * c] * inv, o[8 * c + 1] * inv), pack_bf16(o[8 * c + 2] * inv, o[8 * c + 3] * inv),
+                                    pack_bf16(o[8 * c + 4] * inv, o[8 * c + 5] * inv), pack_bf16(o[8 * c + 6] * inv, o[8 * c + 7] * inv));
+            }
           }
         }
         // s_flag is rewritten by the next item only after all have read it
@@ -608,19 +644,22 @@ done:
   __syncthreads();
   if (warp == 1) {
     if (*abort_flag) __nanosleep(20000);
-    tmem_dealloc(tmem_base, ATTN_TMEM_COLS);
+    tmem_dealloc(tmem_base, C::TMEM_COLS);
   }
 }
 
 int launch_attn_sm100(cudaStream_t st, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                       const AttnPlan& plan, const KvView& kv, const ModelDims& md, int layer, bf16* out, int n_sms,
                       int device, int* status, float* split_ws, const uint4* anc, bool pdl) {
-  static bool attr_set[kMaxDevices] = {};          // the attribute is per device
-  if (device < 0 || device >= kMaxDevices) return -1;
-  if (!attr_set[device]) {
-    if (cudaFuncSetAttribute(attn_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_SMEM) != cudaSuccess)
-      return -1;
-    attr_set[device] = true;
+  static bool attr_set[2][kMaxDevices] = {};       // the attribute is per kernel and device
+  if (device < 0 || device >= kMaxDevices || (md.D != 64 && md.D != 128)) return -1;
+  const int which = md.D == 128;
+  if (!attr_set[which][device]) {
+    const cudaError_t e =
+        which ? cudaFuncSetAttribute(attn_sm100_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<128>::SMEM)
+              : cudaFuncSetAttribute(attn_sm100_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<64>::SMEM);
+    if (e != cudaSuccess) return -1;
+    attr_set[which][device] = true;
   }
   AttnParams p;
   p.plan = plan;
@@ -635,7 +674,12 @@ int launch_attn_sm100(cudaStream_t st, const CUtensorMap& tmQ, const CUtensorMap
   p.split_ws = split_ws;
   p.anc = anc;
   p.status = status;
-  return launch_kernel(attn_sm100_kernel, dim3(2 * n_sms), dim3(kAttnThreads), ATTN_SMEM, st, pdl, tmQ, tmK, tmV, p);
+  // (the grid stays two CTAs per SM for head_dim 128 as well, where one is resident at a time: the item walk and the
+  // plan's item count do not depend on the head size)
+  if (which)
+    return launch_kernel(attn_sm100_kernel<128>, dim3(2 * n_sms), dim3(kAttnThreads), AttnCfg<128>::SMEM, st, pdl, tmQ, tmK,
+                         tmV, p);
+  return launch_kernel(attn_sm100_kernel<64>, dim3(2 * n_sms), dim3(kAttnThreads), AttnCfg<64>::SMEM, st, pdl, tmQ, tmK, tmV, p);
 }
 
 }  // namespace hsd

@@ -19,7 +19,8 @@
 //   GS_SWIGLU      C bf16 = silu(gate) * up              (gate rows and up rows of W land in one tile)
 //   GS_ARGMAX      per-row running argmax over the vocabulary + the next draft token's logit; logits never
 //                  leave the SM (Eq. 10 of the paper fused into the LM head)
-//   GS_QKV_ROPE    rotary embedding on q and k heads, q -> packed bf16, k/v -> paged KV pool
+//   GS_QKV_ROPE    rotary embedding on q and k heads, q -> packed bf16, k/v -> paged KV pool (head_dim 64;
+//                  GS_QKV_ROPE128: the same for head_dim 128)
 #include "hsd_kernels.h"
 
 namespace hsd {
@@ -524,6 +525,105 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           }
         }
       }
+      else if (MODE == GS_QKV_ROPE128) {
+        // head_dim 128: a head is 128 accumulator columns and the rotation pairs dim i with dim i + 64, so a head is
+        // worked in two passes of 32 pairs (columns [32c, 32c+32) with [64+32c, 64+32c+32)); the row's (cos, sin) of
+        // those 32 frequencies come from the table per pass.  q leaves through two staging buffers (dims 0..63 and
+        // 64..127), both filled by the two passes and stored together.
+        const bool live = !(p.status && *p.status);
+        int phys = (row_ok && live) ? p.qkv.row_kv[row] : 0;
+        const bool kv_ok = live && phys >= 0 && phys < p.qkv.kv_rows;
+        if (!kv_ok) phys = 0;
+        const int blk = phys >> 6, off = phys & 63;
+#pragma unroll 1
+        for (int hh = 0; hh < BN / 128; ++hh) {
+          const int head = n0 / 128 + hh;
+          const bool is_q = head < p.qkv.Hq;
+          const bool rot = head < p.qkv.Hq + p.qkv.Hkv;           // q and k heads are normalised (if asked) and rotated
+          if (!slab_ok) break;
+          float rs = 1.f;
+          // (warp-uniform: a tensor-memory load is executed by the whole warp, rows beyond M included)
+          const bool normed = p.qkv.q_norm && rot;
+          if (normed) {                                            // per-head RMSNorm over the head's 128 dims
+            float ss = 0.f;
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+              uint32_t r[32];
+              tmem_ld32(t_acc + hh * 128 + c * 32, r);
+              tmem_ld_wait();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) ss += __uint_as_float(r[i]) * __uint_as_float(r[i]);
+            }
+            rs = rsqrtf(ss * (1.f / 128.f) + p.qkv.eps);
+          }
+          if (is_q) {
+            if (lane == 0) bulk_wait_read<0>();                    // both staging buffers are free
+            __syncwarp();
+          }
+          const bool is_k = rot && !is_q;
+          bf16* pool = is_k ? p.qkv.k_pool_layer : p.qkv.v_pool_layer;
+          const int kvh = head - p.qkv.Hq - (is_k || is_q ? 0 : p.qkv.Hkv);
+          uint4* d4 = reinterpret_cast<uint4*>(pool + (((size_t)blk * p.qkv.Hkv + (is_q ? 0 : kvh)) * 64 + off) * 128);
+#pragma unroll 1
+          for (int c = 0; c < 2; ++c) {
+            uint32_t lo[32], hi[32];
+            tmem_ld32(t_acc + hh * 128 + c * 32, lo);
+            tmem_ld32(t_acc + hh * 128 + 64 + c * 32, hi);
+            tmem_ld_wait();
+            if (normed && row_ok) {
+              const uint4* g4 = reinterpret_cast<const uint4*>(is_q ? p.qkv.q_norm : p.qkv.k_norm);
+#pragma unroll
+              for (int v = 0; v < 4; ++v) {
+                const uint4 gl = __ldg(g4 + 4 * c + v), gh = __ldg(g4 + 8 + 4 * c + v);
+                const uint32_t wl[4] = {gl.x, gl.y, gl.z, gl.w}, wh[4] = {gh.x, gh.y, gh.z, gh.w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  lo[8 * v + 2 * k] = __float_as_uint(__uint_as_float(lo[8 * v + 2 * k]) * rs * bf16_lo(wl[k]));
+                  lo[8 * v + 2 * k + 1] = __float_as_uint(__uint_as_float(lo[8 * v + 2 * k + 1]) * rs * bf16_hi(wl[k]));
+                  hi[8 * v + 2 * k] = __float_as_uint(__uint_as_float(hi[8 * v + 2 * k]) * rs * bf16_lo(wh[k]));
+                  hi[8 * v + 2 * k + 1] = __float_as_uint(__uint_as_float(hi[8 * v + 2 * k + 1]) * rs * bf16_hi(wh[k]));
+                }
+              }
+            }
+            if (rot && row_ok) {
+              const float4* src = reinterpret_cast<const float4*>(p.qkv.rope_cs + (size_t)row * 64 + c * 32);
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                const float4 c2 = __ldg(src + i);   // (cos, sin) of frequencies 32c + 2i and 32c + 2i + 1
+                const float a0 = __uint_as_float(lo[2 * i]), b0 = __uint_as_float(hi[2 * i]);
+                const float a1 = __uint_as_float(lo[2 * i + 1]), b1 = __uint_as_float(hi[2 * i + 1]);
+                lo[2 * i] = __float_as_uint(a0 * c2.x - b0 * c2.y);
+                hi[2 * i] = __float_as_uint(b0 * c2.x + a0 * c2.y);
+                lo[2 * i + 1] = __float_as_uint(a1 * c2.z - b1 * c2.w);
+                hi[2 * i + 1] = __float_as_uint(b1 * c2.z + a1 * c2.w);
+              }
+            }
+            if (is_q) {
+#pragma unroll
+              for (int v = 0; v < 4; ++v) {
+                *stg_chunk(my_stg, lane, 4 * c + v) = pack8(lo + 8 * v);
+                *stg_chunk(my_stg + STG_BYTES, lane, 4 * c + v) = pack8(hi + 8 * v);
+              }
+            } else if (row_ok && kv_ok) {
+              // K and V rows go to the paged pool: one 256-byte row per (token, kv head)
+#pragma unroll
+              for (int v = 0; v < 4; ++v) {
+                d4[4 * c + v] = pack8(lo + 8 * v);
+                d4[8 + 4 * c + v] = pack8(hi + 8 * v);
+              }
+            }
+          }
+          if (is_q) {
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0 && live) {
+              tma_store_2d(&tmC, my_stg, head * 128, wrow0);
+              tma_store_2d(&tmC, my_stg + STG_BYTES, head * 128 + 64, wrow0);
+              bulk_commit();
+            }
+          }
+        }
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) {
@@ -608,7 +708,7 @@ static void pick_tile(int mode, int n_cols, int M, int K, int n_sms, int max_spl
   const int k_blocks = K / BK;
   const int cands[4] = {256, 256, 128, 64};     // first entry: a CTA pair on a 256 x 256 tile
   double best_cost = 1e30;
-  *bn_out = (mode == GS_SWIGLU) ? 128 : 64;
+  *bn_out = (mode == GS_SWIGLU || mode == GS_QKV_ROPE128) ? 128 : 64;
   *splits_out = 1;
   *pair_out = false;
   for (int i = allow_pair ? 0 : 1; i < 4; ++i) {
@@ -616,6 +716,7 @@ static void pick_tile(int mode, int n_cols, int M, int K, int n_sms, int max_spl
     const int bn = cands[i];
     const int out_n = (mode == GS_SWIGLU) ? bn / 2 : bn;
     if (n_cols % out_n || out_n % 64) continue;
+    if (mode == GS_QKV_ROPE128 && bn < 128) continue;     // a tile holds whole 128-column heads
     const int tile_m = pair ? 2 * BM : BM;
     const int walkers = pair ? n_sms / 2 : n_sms;
     const long long tiles = (long long)((M + tile_m - 1) / tile_m) * (n_cols / out_n);
@@ -643,6 +744,7 @@ static int launch_mode(cudaStream_t st, const GemmSm100Args& a) {
     const int fbn = a.force_bn == 512 ? 256 : a.force_bn;       // 512 = a CTA pair on 256-column tiles
     const int out_n = (MODE == GS_SWIGLU) ? fbn / 2 : fbn;
     if ((fbn != 64 && fbn != 128 && fbn != 256) || out_n % 64 || n_cols % out_n) return -1;
+    if (MODE == GS_QKV_ROPE128 && fbn < 128) return -1;
     bn = fbn;
     pair = a.force_bn == 512;
   }
@@ -656,7 +758,7 @@ static int launch_mode(cudaStream_t st, const GemmSm100Args& a) {
     case 256: return launch_one<256, MODE, false>(st, a, splits);
     case 128: return launch_one<128, MODE, false>(st, a, splits);
     default:
-      if (MODE == GS_SWIGLU) return launch_one<128, MODE, false>(st, a, splits);
+      if (MODE == GS_SWIGLU || MODE == GS_QKV_ROPE128) return launch_one<128, MODE, false>(st, a, splits);
       return launch_one<64, MODE, false>(st, a, splits);
   }
 }
@@ -670,6 +772,7 @@ int launch_gemm_sm100(cudaStream_t st, const GemmSm100Args& a) {
     case GS_SWIGLU: return launch_mode<GS_SWIGLU>(st, a);
     case GS_ARGMAX: return launch_mode<GS_ARGMAX>(st, a);
     case GS_QKV_ROPE: return launch_mode<GS_QKV_ROPE>(st, a);
+    case GS_QKV_ROPE128: return launch_mode<GS_QKV_ROPE128>(st, a);
     default: return -1;
   }
 }

@@ -112,7 +112,7 @@ struct TreeAcceptArgs {
 };
 void launch_tree_accept(cudaStream_t st, const TreeAcceptArgs& a, const RowMeta& rm, const int* status, bool pdl);
 // Moves the K/V rows of an accepted tree path (cache rows L + accept_rows[d-1]) to rows L + d, every layer and head.
-void launch_tree_compact(cudaStream_t st, const KvView& kv, int n_layers, int n_kv_heads, int n_seqs, const int* seq_slots,
+void launch_tree_compact(cudaStream_t st, const KvView& kv, int n_layers, int n_kv_heads, int head_dim, int n_seqs, const int* seq_slots,
                          const int* accept_len, const int* accept_rows, int max_q_len, bool pdl);
 // Draft-target matching + prefix-tree packing on the device (Eq. 5-7)
 struct DsvArgs {
@@ -208,11 +208,11 @@ struct QkvEpilogue {      // fused RoPE + paged KV write (QKV projection)
   const int* row_kv;
   int kv_rows;            // rows of one layer of the pool (blocks x 64): a physical row outside it is never written
   const float2* rope_cs;
-  bf16* q_out;            // [T, Hq*64]
+  bf16* q_out;            // [T, Hq*D]
   bf16* k_pool_layer;     // layer base of the K pool
   bf16* v_pool_layer;
-  int Hq, Hkv;
-  const bf16* q_norm;     // per-head RMSNorm gains [64] of q and k before the rotation, or nullptr (none)
+  int Hq, Hkv, D;         // D = head_dim (64 or 128)
+  const bf16* q_norm;     // per-head RMSNorm gains [D] of q and k before the rotation, or nullptr (none)
   const bf16* k_norm;
   float eps;
 };
@@ -232,7 +232,7 @@ struct GemmSm100Args {
   int pair;                    // CTA pairs (clusters of two sharing a 256-row tile) may be used
   int force_bn, force_splits;  // tests: tile width (512 = CTA pair) / K slices instead of the model's choice (0 = choose)
 };
-enum GemmSm100Mode { GS_STORE_BF16 = 0, GS_ADD_F32 = 1, GS_SWIGLU = 2, GS_ARGMAX = 4, GS_QKV_ROPE = 5 };
+enum GemmSm100Mode { GS_STORE_BF16 = 0, GS_ADD_F32 = 1, GS_SWIGLU = 2, GS_ARGMAX = 4, GS_QKV_ROPE = 5, GS_QKV_ROPE128 = 6 };
 int launch_gemm_sm100(cudaStream_t st, const GemmSm100Args& a);
 
 }  // namespace hsd

@@ -542,8 +542,8 @@ void launch_tree_accept(cudaStream_t st, const TreeAcceptArgs& a, const RowMeta&
 // accepted path's rows move from their packed places L + r_d to the places L + d their rotary positions stand for.
 // One CTA per (sequence, layer); a path's rows increase strictly, so moving depth by depth never overwrites a row
 // that is still to be read.
-__global__ void tree_compact_kernel(KvView kv, int n_kv_heads, int n_seqs, const int* seq_slots, const int* accept_len,
-                                    const int* accept_rows, int max_q_len) {
+__global__ void tree_compact_kernel(KvView kv, int n_kv_heads, int head_dim, int n_seqs, const int* seq_slots,
+                                    const int* accept_len, const int* accept_rows, int max_q_len) {
   pdl_wait();               // everything below reads or writes what earlier kernels of the step produced
   pdl_launch_dependents();
   const int i = blockIdx.x, layer = blockIdx.y;
@@ -554,7 +554,8 @@ __global__ void tree_compact_kernel(KvView kv, int n_kv_heads, int n_seqs, const
   const int L = kv.seq_lens[slot];
   if (L < 0 || (long long)L + max_q_len > (long long)kv.max_blocks * HSD_KV_BLOCK) return;
   const int* bt = kv.block_table + (size_t)slot * kv.max_blocks;
-  const int chunks = n_kv_heads * 2 * 8;                 // 16-byte chunks of one token's K and V rows in a layer
+  const int row_chunks = head_dim / 8;                   // 16-byte chunks of one (token, kv head) row
+  const int chunks = n_kv_heads * 2 * row_chunks;        // ... of one token's K and V rows in a layer
   for (int d = 1; d <= a && d < max_q_len; ++d) {
     const int r = accept_rows[(size_t)i * max_q_len + d - 1];
     if (r != d && r > 0 && r < max_q_len) {              // a row of this call (L + r is within the table, see above)
@@ -562,10 +563,10 @@ __global__ void tree_compact_kernel(KvView kv, int n_kv_heads, int n_seqs, const
       const int bs = bt[ps / HSD_KV_BLOCK], bd = bt[pd / HSD_KV_BLOCK];
       if (bs >= 0 && bs < kv.n_blocks && bd >= 0 && bd < kv.n_blocks) {
         for (int t = threadIdx.x; t < chunks; t += blockDim.x) {
-          const int c16 = t & 7, pool = (t >> 3) & 1, h = t >> 4;
+          const int c16 = t % row_chunks, pool = (t / row_chunks) & 1, h = t / (2 * row_chunks);
           bf16* base = pool ? kv.v_pool : kv.k_pool;
-          const size_t src = ((((size_t)layer * kv.n_blocks + bs) * n_kv_heads + h) * 64 + ps % HSD_KV_BLOCK) * 64;
-          const size_t dst = ((((size_t)layer * kv.n_blocks + bd) * n_kv_heads + h) * 64 + pd % HSD_KV_BLOCK) * 64;
+          const size_t src = ((((size_t)layer * kv.n_blocks + bs) * n_kv_heads + h) * 64 + ps % HSD_KV_BLOCK) * head_dim;
+          const size_t dst = ((((size_t)layer * kv.n_blocks + bd) * n_kv_heads + h) * 64 + pd % HSD_KV_BLOCK) * head_dim;
           reinterpret_cast<uint4*>(base + dst)[c16] = reinterpret_cast<const uint4*>(base + src)[c16];
         }
       }
@@ -573,9 +574,9 @@ __global__ void tree_compact_kernel(KvView kv, int n_kv_heads, int n_seqs, const
     __syncthreads();
   }
 }
-void launch_tree_compact(cudaStream_t st, const KvView& kv, int n_layers, int n_kv_heads, int n_seqs, const int* seq_slots,
-                         const int* accept_len, const int* accept_rows, int max_q_len, bool pdl) {
-  launch_kernel(tree_compact_kernel, dim3(n_seqs, n_layers), dim3(128), 0, st, pdl, kv, n_kv_heads, n_seqs, seq_slots,
+void launch_tree_compact(cudaStream_t st, const KvView& kv, int n_layers, int n_kv_heads, int head_dim, int n_seqs,
+                         const int* seq_slots, const int* accept_len, const int* accept_rows, int max_q_len, bool pdl) {
+  launch_kernel(tree_compact_kernel, dim3(n_seqs, n_layers), dim3(128), 0, st, pdl, kv, n_kv_heads, head_dim, n_seqs, seq_slots,
                 accept_len, accept_rows, max_q_len);
 }
 

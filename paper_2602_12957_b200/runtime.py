@@ -69,7 +69,7 @@ class KvCache:
         cfg, dev = model.cfg, model.device
         table, n_blocks = I.make_block_tables(capacities, seed, cfg.kv_block)
         self.n_slots, self.n_blocks, self.max_blocks = len(capacities), n_blocks, table.shape[1]
-        shape = (cfg.n_layers, n_blocks, cfg.n_kv_heads, 64, 64)
+        shape = (cfg.n_layers, n_blocks, cfg.n_kv_heads, cfg.kv_block, cfg.head_dim)
         if poison:   # huge finite filler: an unmasked read of a row that was never written wrecks the outputs
             self.k_pool = torch.full(shape, 1e30, dtype=torch.bfloat16, device=dev)
             self.v_pool = torch.full(shape, 1e30, dtype=torch.bfloat16, device=dev)

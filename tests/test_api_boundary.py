@@ -70,8 +70,10 @@ def test_host_side_argument_checks_need_no_device(B):
     w = B.hsd_weights()                                   # all null pointers
     st, ctx = B.hsd_create(cfg, w)
     assert st == B.HSD_ERR_INVALID_ARG
-    bad = B.make_config(I.ModelConfig(1, 256, 4, 4, 128, 1024, 4096))   # head_dim 128 is not supported
+    bad = B.make_config(I.ModelConfig(1, 256, 4, 4, 96, 1024, 4096))    # head_dim is 64 or 128
     assert B.hsd_create(bad, w)[0] == B.HSD_ERR_SHAPE
+    simt128 = B.make_config(I.ModelConfig(1, 256, 2, 2, 128, 1024, 4096), B.HSD_FLAG_SIMT_ATTENTION)
+    assert B.hsd_create(simt128, w)[0] == B.HSD_ERR_SHAPE              # the plain cross-check kernels: head_dim 64 only
     bad = B.make_config(I.ModelConfig(1, 256, 4, 3, 64, 1024, 4096))     # heads not a multiple of kv heads
     assert B.hsd_create(bad, w)[0] == B.HSD_ERR_SHAPE
     # calls on a null context

@@ -112,3 +112,10 @@ def test_empty_draft_is_a_plain_decode_step():
     assert abs(float(out["row_zmax"][0]) - res.row_zmax[0]) < H.LOGIT_TOL
     if res.row_gap[0] > H.GAP_EXACT:
         assert int(out["emit_tokens"][0, 0]) == res.emitted[0]
+
+
+def test_head_dim_128_page_chunks_with_commit_and_rollback_match_oracle():
+    cfg = I.ModelConfig(n_layers=2, d_model=1024, n_heads=8, n_kv_heads=4, head_dim=128, d_ffn=4096, vocab=8192)
+    stats, n_chunks = _page_schedule(cfg, seed=34, n_visual=200, n_prompt=40, draft_len=300, chunk_len=96)
+    print("hd128 page", stats, n_chunks)
+    assert n_chunks >= 4 and stats["max_dz"] < H.LOGIT_TOL

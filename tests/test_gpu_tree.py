@@ -257,3 +257,14 @@ def test_tree_argument_and_device_checks():
     eng.verify_tree(toks, cu, eng._i32(good), 5, 10, out=out)
     eng.check_device("after the bad trees")
     assert all(0 <= a <= 4 for a in out["accept_len"].cpu().tolist())
+
+
+def test_head_dim_128_trees_match_oracle_and_compact():
+    """Head dimension 128 through the tree path: ancestry masks, traversal at tau 0.75, compaction of 256-byte KV rows,
+    then a chain step on top of the compacted cache."""
+    cfg = I.ModelConfig(n_layers=2, d_model=1024, n_heads=8, n_kv_heads=4, head_dim=128, d_ffn=4096, vocab=8192)
+    wl = I.region_workload(seed=92, n_regions=4, prefix_lo=70, prefix_hi=300, draft_mean=60, draft_lo=8, draft_hi=120,
+                           cfg=cfg, name="hd128_trees")
+    stats, _, _ = run_tree_case(wl, [127, 64, 90, 33], LOG_TAU_PAPER)
+    assert stats["exact"] + stats["tolerated"] == 4 and stats["max_dz"] < H.LOGIT_TOL
+    print("hd128 trees", stats)

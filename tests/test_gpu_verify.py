@@ -270,3 +270,38 @@ def test_wide_decoder_with_four_query_heads_per_kv_head_matches_oracle():
     stats, orc, per, _ = run_region_parity(wl, 0)
     print("wide", stats, [(len(o.draft), o.res.accept_len) for o in orc.values()])
     assert stats["max_dz"] < H.LOGIT_TOL
+
+
+def _decoder_hd128(n_layers=2, vocab=8192, qk_norm=False):
+    """d_model 1024, 8 query / 4 kv heads x 128 (the head size of the 2-9 B decoders the paper evaluates, Sec. 4.3)."""
+    return I.ModelConfig(n_layers=n_layers, d_model=1024, n_heads=8, n_kv_heads=4, head_dim=128, d_ffn=4096, vocab=vocab,
+                         qk_norm=qk_norm)
+
+
+@pytest.mark.parametrize("qk_norm", [False, True], ids=["plain", "qk_norm"])
+def test_head_dim_128_regions_match_oracle(qk_norm):
+    """Head dimension 128: two operand sub-tiles per Q / K / V tile, a 128-column accumulator, the rotation pairing
+    dim i with dim i + 64 in the QKV epilogue, 256-byte KV rows.  Several q-tiles per sequence, ragged tails,
+    prefixes that end inside a KV block, with and without the per-head RMSNorm of q and k."""
+    wl = I.region_workload(seed=83, n_regions=5, prefix_lo=70, prefix_hi=330, draft_mean=60, draft_lo=8, draft_hi=200,
+                           cfg=_decoder_hd128(qk_norm=qk_norm), name="hd128_regions")
+    stats, orc, per, _ = run_region_parity(wl, 0)
+    print("hd128", qk_norm, stats, [(len(o.draft), o.res.accept_len) for o in orc.values()])
+    assert stats["max_dz"] < H.LOGIT_TOL
+
+
+@pytest.mark.parametrize("plan", [(1 << 20, 1), (1, 1 << 20)], ids=["max_slices", "no_slices"])
+def test_head_dim_128_kv_slicing_does_not_change_the_result(plan):
+    wl = I.region_workload(seed=84, n_regions=4, prefix_lo=100, prefix_hi=520, draft_mean=50, draft_lo=8, draft_hi=150,
+                           cfg=_decoder_hd128(), name="hd128_regions_slicing")
+    stats, orc, per, _ = run_region_parity(wl, 0, attn_plan=plan)
+    print("hd128 slicing", plan, stats)
+    assert stats["max_dz"] < H.LOGIT_TOL
+
+
+def test_head_dim_128_refuses_the_plain_cross_check_kernels():
+    from paper_2602_12957_b200 import binding as B
+    from paper_2602_12957_b200 import runtime as R
+    cfg = _decoder_hd128(1, 4096)
+    with pytest.raises(Exception):
+        R.DeviceModel(cfg, I.make_weights(cfg, 1), B.HSD_FLAG_SIMT_ATTENTION)
