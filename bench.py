@@ -122,10 +122,18 @@ WORKLOADS = {
     "tree": "one step of the decoupled-verification loop on the region batch's 16 prefixes (256-1024): window matching "
             "(n = 3) against two damaged copies of each region's text and prefix-tree packing on the device (128 rows "
             "per sequence), tree verification at tau 0.75, compaction of the accepted path's K/V rows",
+    "region_hd128": "region-level stage on a wider decoder with 128-wide heads (the head size of the 2-9 B parsers of "
+                    "Sec. 4.3): 8 layers, d2048 16q/8kv x128 ffn8192 vocab32768, the same 16 regions and drafts",
     "mixed": "mixed serving batch: 64 regions (prefix 128-2048, lognormal drafts mean 96, 8-512) + 2 page chunks of 1024 "
              "over 4352-token prefixes, one varlen launch",
 }
-EXTRA_WORKLOADS = ["region_short", "page", "long1024", "long2048", "mixed", "tree"]
+EXTRA_WORKLOADS = ["region_short", "page", "long1024", "long2048", "mixed", "tree", "region_hd128"]
+# the second decoder shape (a slice of 8 layers keeps the host-side weight draw short; per-layer work is what is measured)
+DECODER_HD128 = I.ModelConfig(n_layers=8, d_model=2048, n_heads=16, n_kv_heads=8, head_dim=128, d_ffn=8192, vocab=32768)
+
+
+def workload_cfg(name):
+    return DECODER_HD128 if name == "region_hd128" else I.DECODER
 
 TREE_NODES = 127     # nodes below the root: 128 packed rows per sequence, the paper's packing limit (Sec. 4.3)
 TREE_MAIN = 64       # the planted agreement lengths of the region workload are scaled to this many tokens
@@ -137,8 +145,8 @@ PAGE_SHAPES = {"page": (7936, 512), "long1024": (17408, 1024), "long2048": (1638
 def make_workload(name, rank, world=1, sharded=False, mixed_k=0):
     """The seeded workload of this rank.  Returns (workload, plant): `plant` says whether the drafts are planted along
     the library's own greedy path (region) or random (the others: kernel time does not depend on token values)."""
-    cfg = I.DECODER
-    if name in ("region", "region_short", "tree"):
+    cfg = workload_cfg(name)
+    if name in ("region", "region_short", "tree", "region_hd128"):
         fixed = 8 if name == "region_short" else None
         if sharded and world > 1:       # ONE batch of 16 x world regions, split by the cost model
             wl = I.region_workload(seed=I.BASE_SEED + 1, n_regions=16 * world, fixed_draft_len=fixed, cfg=cfg)
@@ -151,7 +159,7 @@ def make_workload(name, rank, world=1, sharded=False, mixed_k=0):
                 s_.agree_len = int(round(TREE_MAIN * s_.agree_len / max(1, s_.draft_len)))
                 s_.draft_len = TREE_NODES
         wl.name = name
-        return wl, name != "region_short"
+        return wl, name in ("region", "tree")
     if name == "mixed":
         if mixed_k:       # the sweep over a fixed draft length: the 64 regions alone
             return I.mixed_workload(seed=I.BASE_SEED + 4 + 1000 * rank, fixed_draft_len=mixed_k, with_page_chunks=False,
@@ -174,10 +182,12 @@ def decoder_weights():
     return _WEIGHTS["w"]
 
 
-def build_model(flags=0):
+def build_model(flags=0, name="region"):
     import torch
     from paper_2602_12957_b200 import runtime as R
-    return R.DeviceModel(I.DECODER, decoder_weights(), flags, f"cuda:{torch.cuda.current_device()}")
+    cfg = workload_cfg(name)
+    weights = decoder_weights() if cfg is I.DECODER else I.make_weights(cfg, I.BASE_SEED + 6)
+    return R.DeviceModel(cfg, weights, flags, f"cuda:{torch.cuda.current_device()}")
 
 
 def plant_along_verify_rows(eng, kv, seqs, first, prefix_lens, cfg, max_rounds=600):
@@ -236,7 +246,7 @@ def plant_along_verify_rows(eng, kv, seqs, first, prefix_lens, cfg, max_rounds=6
 def build_gpu_state(name, model, rank, world=1, sharded=False, mixed_k=0, random_drafts=False):
     import torch
     from paper_2602_12957_b200 import runtime as R
-    cfg = I.DECODER
+    cfg = workload_cfg(name)
     wl, plant = make_workload(name, rank, world, sharded, mixed_k)
     plant = plant and not random_drafts
     seqs = wl.seqs
@@ -582,7 +592,7 @@ def run_ours(args):
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
-    model = build_model(args.flags)
+    model = build_model(args.flags, args.workload)
     st = build_gpu_state(args.workload, model, rank, world, args.sharded, args.mixed_k, args.random_drafts)
     eng, kv, cfg = st["eng"], st["kv"], st["cfg"]
     dev = eng.dev
@@ -682,7 +692,10 @@ def run_ours(args):
     if world == 1 and args.workload == "region" and not args.only_region:
         del runner
         for name in EXTRA_WORKLOADS:
-            st2 = build_gpu_state(name, model, 0)
+            model2 = model
+            if workload_cfg(name) is not I.DECODER:
+                model2 = build_model(0, name)
+            st2 = build_gpu_state(name, model2, 0)
             r2 = Runner(st2, stream, use_graph=not args.no_graph, warmup=3)
             ms2, clk2, n2 = r2.timed(20, barrier, uuid, min_seconds=1.0)
             pr2 = r2.profile(5)
@@ -698,9 +711,12 @@ def run_ours(args):
                            "top_kernel_traffic": roof2["traffic"], "clocks": clk2,
                            "kernels": {k: {"ms_per_step": round(v["ms_per_step"], 4),
                                            "roofline_frac": round(v.get("roofline_frac", 0.0), 3)} for k, v in kern2.items()}}
-            if not args.no_cpu_baseline and name != "tree":      # (the oracle's tree form is not timed)
+            if not args.no_cpu_baseline and name not in ("tree", "region_hd128"):   # (the oracle's tree form and the second decoder are not timed)
                 extra[name]["cpu_baseline"] = cpu_baseline_sample(st2["wl"], ctx2, budget_s=6.0, steps=1, max_rows=128)
             del r2, st2
+            if model2 is not model:
+                model2.close()
+            del model2
             torch.cuda.empty_cache()
         with torch.cuda.stream(stream):
             extra["two_stage"] = two_stage_workload(f"cuda:{torch.cuda.current_device()}")
