@@ -11,19 +11,21 @@
 // O, exponent reference, sum) partials in the workspace and the last slice to finish combines them in slice order, so
 // the result does not depend on which CTA ran what.
 //
-// A KV tile is 128 keys = two paged blocks [64 keys][64 dims] per kv head, fetched by TMA through the block table
-// into adjacent halves of a stage; K is the K-major B operand of S = Q K^T (one 128 x 128 x 64 product per tile), V
-// the MN-major B operand of O += P V (128 x 64 x 128).  Persistent CTAs, two per SM, walk the item list.  Warp roles:
+// A KV tile is 128 keys = two paged blocks [64 keys][head_dim] per kv head, fetched by TMA through the block table,
+// 64 dims at a time, into adjacent halves of a stage; K is the K-major B operand of S = Q K^T (one 128 x 128 x
+// head_dim product per tile), V the MN-major B operand of O += P V (128 x head_dim x 128).  Persistent CTAs walk the
+// item list: two per SM with head_dim 64, one with 128 (tensor-memory columns).  Warp roles:
 // warp 0 = TMA producers (lane 0: Q and the K ring, lane 1: the V ring; K is free as soon as S has been formed, V
 // only after the second product, so the two rings run at their own pace and two stages each suffice), warp 1 = MMA
 // issuer + TMEM owner, warps 2..9 = softmax: warp w works on TMEM lane quarter w mod 4 (the hardware's rule), warps
 // 2..5 on keys 0..63 of the tile and warps 6..9 on keys 64..127, one thread per (row, half).
 // Per tile: S (TMEM, 128 fp32 columns) -> softmax in registers -> P (bf16, back into TMEM: 64 columns, the A operand
-// of the second product, so P never passes through shared memory) -> O += P V accumulated IN TENSOR MEMORY.  What the measurements behind this shape said (per 64-key tile
-// and CTA, before): the softmax warps' own instruction stream ~1,950 cycles, half of it the 64 exponentials of a row
-// queueing with the other CTA's on the SM's 16 exp lanes per clock; the issuing thread ~1,300 (140-220 cycles for
-// every probe of an already completed barrier, 70-90 per MMA or commit).  Twice the keys per barrier round and MMA
-// group, and twice the warps on the exponentials, attack both.
+// of the second product, so P never passes through shared memory) -> O += P V accumulated in tensor memory.
+// What the measurements behind this shape said (64-key tiles, four softmax warps, P through shared memory, per tile
+// and CTA): the softmax warps' own instruction stream ~1,950 cycles, half of it the 64 exponentials of a row queueing
+// with the other CTA's on the SM's 16 exp lanes per clock; the issuing thread ~1,300 (140-220 cycles for every probe
+// of an already completed barrier, 70-90 per MMA or commit).  Twice the keys per barrier round and MMA group, twice
+// the warps on the exponentials, and no shared-memory round trip for P attack both.
 // The exponent reference of a row is not its running maximum but a value that is raised only when the maximum has
 // grown by more than kRescaleBits binary orders since it was set (P stays below 2^kRescaleBits, far inside bf16 and
 // fp32 range): then, and only then, the row's accumulator is read, scaled and written back; after the first tiles of
