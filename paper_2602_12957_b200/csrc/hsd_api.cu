@@ -144,8 +144,10 @@ Ws carve(const hsd_ctx* c, void* base, int T, int S) {
     w.plan.tile_seq = static_cast<int*>(take(sizeof(int) * mt));
     w.plan.tile_nkv = static_cast<int*>(take(sizeof(int) * mt));
     w.plan.counters = static_cast<int*>(take(sizeof(int) * (size_t)mt * md.Hkv));
+    w.plan.first = static_cast<int4*>(take(sizeof(int4) * 3 * 2 * (size_t)c->n_sms));
     w.plan.n_items = w.status ? w.status + 5 : nullptr;
     w.plan.n_kv_heads = md.Hkv;
+    w.plan.grid = 2 * c->n_sms;
   }
   w.bytes = off;
   return w;
@@ -278,7 +280,7 @@ int run_layers(hsd_ctx* c, const hsd_kv* kvp, const StepArgs& a, const Ws& w, cu
     Scope s(c, st, KC_SETUP);
     // items per launch: a few per CTA slot (two CTAs per SM), at least attn_min_chunk KV tiles each
     // (a context with a fixed summation order never cuts a KV range: where the cuts fall depends on the batch)
-    launch_attn_plan(st, w.rm, w.plan, a.n_seqs, tokens_per_tile, max(1, c->attn_target_items / md.Hkv),
+    launch_attn_plan(st, w.rm, w.plan, kv, a.n_seqs, tokens_per_tile, max(1, c->attn_target_items / md.Hkv),
                      c->max_splits == 1 ? (1 << 20) : c->attn_min_chunk,
                      w.status + 4, w.status, c->pdl);
   }

@@ -94,10 +94,28 @@ __device__ __forceinline__ bool warps_sync(uint64_t* bar, uint32_t& phase, int l
   return __all_sync(0xffffffffu, ok);
 }
 
+// The item x kv-head index that CTA `bx` of a grid of `G` takes in round r of its walk (-1: none).  Round r: CTA i
+// takes index r G + i in even rounds and r G + (G - 1 - i) in odd ones (the list is sorted longest first, so the CTA
+// that drew a long item in one round draws a short one in the next).  A launch with fewer items than CTAs leaves
+// some SMs with one busy CTA (the grid is two CTAs per SM, and CTA b shares its SM with CTA b + G/2 under the usual
+// placement); a CTA that has its SM alone walks its tiles faster, so the longest items go to those SMs and the
+// others pair a long item with a short one.
+__device__ __forceinline__ int attn_item_at(int r, int total, int bx, int G) {
+  const int n_rounds = (total + G - 1) / G, half_grid = G / 2;
+  if (n_rounds == 1 && total > half_grid) {
+    const int n_second = total - half_grid;            // busy CTAs in the second half of the grid
+    if (bx < half_grid) return bx >= n_second ? bx - n_second : (half_grid - n_second) + bx;
+    return bx - half_grid < n_second ? total - 1 - (bx - half_grid) : -1;
+  }
+  const int i = (r & 1) ? G - 1 - bx : bx;
+  const int w = r * G + i;
+  return w < total ? w : -1;
+}
+
 // ------------------------------------------------------------------------------------------------
 // Plan: one CTA.  For every q-tile the KV tiles it can see and into how many slices that range is cut, then
 // the flat list of (q-tile, slice) items with everything a CTA needs to run one.
-__global__ void attn_plan_kernel(RowMeta rm, AttnPlan pl, int n_seqs, int tokens_per_tile, int target_items,
+__global__ void attn_plan_kernel(RowMeta rm, AttnPlan pl, KvView kv, int n_seqs, int tokens_per_tile, int target_items,
                                  int min_chunk, const int* tile_count, const int* status) {
   pdl_wait();
   pdl_launch_dependents();
@@ -106,6 +124,7 @@ __global__ void attn_plan_kernel(RowMeta rm, AttnPlan pl, int n_seqs, int tokens
   __syncthreads();
   if (*status) {
     if (threadIdx.x == 0) *pl.n_items = 0;
+    for (int b = threadIdx.x; b < pl.grid; b += blockDim.x) pl.first[3 * b + 2] = make_int4(-1, 0, 0, 0);
     return;
   }
   const int n_tiles = *tile_count;
@@ -185,12 +204,35 @@ __global__ void attn_plan_kernel(RowMeta rm, AttnPlan pl, int n_seqs, int tokens
   }
   // slice-arrival counters of every (q-tile, kv head): zero at the start of a step, reset by the combiner
   for (int i = threadIdx.x; i < n_tiles * pl.n_kv_heads; i += blockDim.x) pl.counters[i] = 0;
+  // what every CTA of the attention grid starts with, in one record: its first item and the physical blocks of that
+  // item's first KV tile, so that a CTA's first loads do not wait for a chain of dependent reads (item -> block table)
+  __syncthreads();
+  const int total = n * pl.n_kv_heads;
+  for (int b = threadIdx.x; b < pl.grid; b += blockDim.x) {
+    const int w = attn_item_at(0, total, b, pl.grid);
+    if (w < 0) {
+      pl.first[3 * b + 2] = make_int4(-1, 0, 0, 0);
+      continue;
+    }
+    const int4 ia = pl.items[2 * (w / pl.n_kv_heads)], ib = pl.items[2 * (w / pl.n_kv_heads) + 1];
+    const int kt_lo = ib.x & 0xffff, kt_hi = ib.x >> 16;
+    int phys0 = 0, phys1 = 0;
+    if (kt_hi > kt_lo && ia.w >= 0 && ia.w < kv.n_slots && kt_hi <= kv.max_blocks) {
+      const int* bt = kv.block_table + (size_t)ia.w * kv.max_blocks;
+      phys0 = bt[kt_lo];
+      phys1 = bt[kt_lo + 1 < kt_hi ? kt_lo + 1 : kt_lo];
+    }
+    pl.first[3 * b] = ia;
+    pl.first[3 * b + 1] = ib;
+    pl.first[3 * b + 2] = make_int4(w, w % pl.n_kv_heads, phys0, phys1);
+  }
 }
 
-void launch_attn_plan(cudaStream_t st, const RowMeta& rm, const AttnPlan& pl, int n_seqs, int tokens_per_tile,
-                      int target_items, int min_chunk, const int* tile_count, const int* status, bool pdl) {
-  launch_kernel(attn_plan_kernel, dim3(1), dim3(256), 0, st, pdl, rm, pl, n_seqs, tokens_per_tile, target_items, min_chunk,
-                tile_count, status);
+void launch_attn_plan(cudaStream_t st, const RowMeta& rm, const AttnPlan& pl, const KvView& kv, int n_seqs,
+                      int tokens_per_tile, int target_items, int min_chunk, const int* tile_count, const int* status,
+                      bool pdl) {
+  launch_kernel(attn_plan_kernel, dim3(1), dim3(256), 0, st, pdl, rm, pl, kv, n_seqs, tokens_per_tile, target_items,
+                min_chunk, tile_count, status);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -260,25 +302,20 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   pdl_wait();               // q, the K/V rows of this step, the row metadata and the plan come from earlier kernels
   pdl_launch_dependents();
 
-  const int total = (*p.status) ? 0 : *p.plan.n_items * p.Hkv;
-  // Round r of the walk: CTA i takes item r G + i in even rounds and r G + (G - 1 - i) in odd ones (the list is
-  // sorted longest first, so the CTA that drew a long item in one round draws a short one in the next).
+  // The plan's record of this CTA's first item (the item and the physical blocks of its first KV tile) for the two
+  // warps that start the pipeline: read together with the status word and the item count, before any of them is
+  // used, so that the first TMA loads are one round trip away instead of four (status -> count -> item -> block table).
+  int4 rec_a = make_int4(0, 0, 0, 0), rec_b = rec_a, rec_c = rec_a;
+  if (warp < 2) {
+    const int4* rec = p.plan.first + 3 * (size_t)blockIdx.x;
+    rec_a = rec[0];
+    rec_b = rec[1];
+    rec_c = rec[2];
+  }
+  const int status_now = *p.status, n_items_now = *p.plan.n_items;
+  const int total = status_now ? 0 : n_items_now * p.Hkv;
   const int n_rounds = (total + (int)gridDim.x - 1) / (int)gridDim.x;
-  // A launch with fewer items than CTAs leaves some SMs with one busy CTA (the grid is two CTAs per SM, and CTA b
-  // shares its SM with CTA b + G/2 under the usual placement); a CTA that has its SM alone walks its tiles faster,
-  // so the longest items go to those SMs and the others pair a long item with a short one.
-  const int half_grid = (int)gridDim.x / 2;
-  auto item_of_round = [&](int r) -> int {
-    if (n_rounds == 1 && total > half_grid) {
-      const int n_second = total - half_grid;          // busy CTAs in the second half of the grid
-      const int bx = (int)blockIdx.x;
-      if (bx < half_grid) return bx >= n_second ? bx - n_second : (half_grid - n_second) + bx;
-      return bx - half_grid < n_second ? total - 1 - (bx - half_grid) : -1;
-    }
-    const int i = (r & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x;
-    const int w = r * (int)gridDim.x + i;
-    return w < total ? w : -1;
-  };
+  auto item_of_round = [&](int r) -> int { return attn_item_at(r, total, (int)blockIdx.x, (int)gridDim.x); };
 
   // Tile counter t (all 128-key tiles of all items of this CTA): ring stage = t % KV_STAGES, and every barrier's
   // parity follows from how often t has used it; n counts items (Q hand-over barriers).
@@ -293,10 +330,15 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       uint32_t t = 0;
       int n = 0;
       for (int r = 0; r < n_rounds; ++r) {
-        const int w = item_of_round(r);
+        const int w = r == 0 ? (total > 0 ? rec_c.x : -1) : item_of_round(r);
         if (w < 0) continue;
-        const int4 ia = p.plan.items[2 * (w / p.Hkv)], ib = p.plan.items[2 * (w / p.Hkv) + 1];
-        const int kvh = w % p.Hkv;
+        int4 ia = rec_a, ib = rec_b;
+        int kvh = rec_c.y;
+        if (r != 0) {
+          ia = p.plan.items[2 * (w / p.Hkv)];
+          ib = p.plan.items[2 * (w / p.Hkv) + 1];
+          kvh = w % p.Hkv;
+        }
         const int kt_lo = ib.x & 0xffff, kt_hi = ib.x >> 16;
         const int* bt = p.block_table + (size_t)ia.w * p.max_blocks;
         if (is_k) {
@@ -308,7 +350,11 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         for (int kt = kt_lo; kt < kt_hi; kt += 2, ++t) {
           // the tile's two blocks; a slice of odd length ends with half a tile: the last block is staged twice and
           // the softmax warps mask its second copy
-          const int phys0 = bt[kt], phys1 = bt[kt + 1 < kt_hi ? kt + 1 : kt];
+          int phys0 = rec_c.z, phys1 = rec_c.w;
+          if (r != 0 || kt != kt_lo) {
+            phys0 = bt[kt];
+            phys1 = bt[kt + 1 < kt_hi ? kt + 1 : kt];
+          }
           const int st = t % KV_STAGES;
           if (!mbar_wait(empty + st, ((t / KV_STAGES) & 1) ^ 1u, abort_flag, p.status, 401)) goto done;
           const int row0 = (((p.layer * p.n_blocks) + phys0) * p.Hkv + kvh) * 64;
@@ -332,9 +378,9 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       uint32_t t = 0;
       int n = 0;
       for (int r = 0; r < n_rounds; ++r) {
-        const int w = item_of_round(r);
+        const int w = r == 0 ? (total > 0 ? rec_c.x : -1) : item_of_round(r);
         if (w < 0) continue;
-        const int4 ib = p.plan.items[2 * (w / p.Hkv) + 1];
+        const int4 ib = r == 0 ? rec_b : p.plan.items[2 * (w / p.Hkv) + 1];
         const int n_it = ((ib.x >> 16) - (ib.x & 0xffff) + 1) / 2;      // 128-key tiles of the item
         // S(ti) = Q K(ti)^T: four K = 16 steps over every 64 dims, N = 128 keys
         auto issue_s = [&](uint32_t ti, bool last) -> bool {
@@ -679,9 +725,9 @@ int launch_attn_sm100(cudaStream_t st, const CUtensorMap& tmQ, const CUtensorMap
   // (the grid stays two CTAs per SM for head_dim 128 as well, where one is resident at a time: the item walk and the
   // plan's item count do not depend on the head size)
   if (which)
-    return launch_kernel(attn_sm100_kernel<128>, dim3(2 * n_sms), dim3(kAttnThreads), AttnCfg<128>::SMEM, st, pdl, tmQ, tmK,
+    return launch_kernel(attn_sm100_kernel<128>, dim3(plan.grid), dim3(kAttnThreads), AttnCfg<128>::SMEM, st, pdl, tmQ, tmK,
                          tmV, p);
-  return launch_kernel(attn_sm100_kernel<64>, dim3(2 * n_sms), dim3(kAttnThreads), AttnCfg<64>::SMEM, st, pdl, tmQ, tmK, tmV, p);
+  return launch_kernel(attn_sm100_kernel<64>, dim3(plan.grid), dim3(kAttnThreads), AttnCfg<64>::SMEM, st, pdl, tmQ, tmK, tmV, p);
 }
 
 }  // namespace hsd

@@ -170,10 +170,14 @@ struct AttnPlan {
   int* tile_seq;    // [max_tiles] sequence of a q-tile
   int* tile_nkv;    // [max_tiles] KV tiles it can see
   int* counters;    // [max_tiles, n_kv_heads] slices that have delivered their partial
+  int4* first;      // [grid CTAs][3]: the item a CTA of the attention grid starts with, ready to use: the item's two
+                    // words, then {item x kv head index (-1: none), kv head, first two physical KV blocks}
   int n_kv_heads;
+  int grid;         // CTAs of the attention launches this plan is made for
 };
-void launch_attn_plan(cudaStream_t st, const RowMeta& rm, const AttnPlan& pl, int n_seqs, int tokens_per_tile,
-                      int target_items, int min_chunk, const int* tile_count, const int* status, bool pdl);
+void launch_attn_plan(cudaStream_t st, const RowMeta& rm, const AttnPlan& pl, const KvView& kv, int n_seqs,
+                      int tokens_per_tile, int target_items, int min_chunk, const int* tile_count, const int* status,
+                      bool pdl);
 int launch_attn_sm100(cudaStream_t st, const CUtensorMap& tmQ, const CUtensorMap& tmK, const CUtensorMap& tmV,
                       const AttnPlan& plan, const KvView& kv, const ModelDims& md, int layer, bf16* out, int n_sms,
                       int device, int* status, float* split_ws, const uint4* anc, bool pdl);
