@@ -89,6 +89,9 @@ struct Ws {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// CTAs of an attention launch: as many as are resident at once (two per SM with head_dim 64, one with 128)
+inline int attn_grid(const hsd_ctx* c) { return (c->md.D == 128 ? 1 : 2) * c->n_sms; }
+
 inline int attn_max_tiles(const ModelDims& md, int T, int S) { return T / (128 / md.group) + S; }
 // Split-KV partial results: per (q-tile, kv head, slice) 128 rows of an fp32 accumulator row plus (max, sum).
 inline size_t split_ws_floats(const ModelDims& md, int T, int S) {
@@ -147,7 +150,7 @@ Ws carve(const hsd_ctx* c, void* base, int T, int S) {
     w.plan.first = static_cast<int4*>(take(sizeof(int4) * 3 * 2 * (size_t)c->n_sms));
     w.plan.n_items = w.status ? w.status + 5 : nullptr;
     w.plan.n_kv_heads = md.Hkv;
-    w.plan.grid = 2 * c->n_sms;
+    w.plan.grid = attn_grid(c);
   }
   w.bytes = off;
   return w;
@@ -566,7 +569,7 @@ int hsd_create(const hsd_model_config* cfg, const hsd_weights* w, hsd_ctx** out)
   c->hg_seen_valid = false;
   c->hg_exec = nullptr;
   c->hg_launches = 0;
-  c->attn_target_items = 2 * c->n_sms;   // one item per CTA slot: slicing costs a partial hand-over per slice
+  c->attn_target_items = attn_grid(c);   // one item per CTA slot: slicing costs a partial hand-over per slice
   c->attn_min_chunk = 4;
   c->tap_layer = -1; c->tap_which = 0; c->tap_dst = nullptr; c->tap_bytes = 0;
   c->last_cuda_error = 0;
@@ -1130,7 +1133,7 @@ int hsd_debug_set_gemm_tile(hsd_ctx* c, int tile_n, int k_slices) {
 
 int hsd_debug_set_attn_plan(hsd_ctx* c, int target_items, int min_kv_tiles) {
   if (!c || target_items < 0 || min_kv_tiles < 0) return HSD_ERR_INVALID_ARG;
-  c->attn_target_items = target_items ? target_items : 2 * c->n_sms;
+  c->attn_target_items = target_items ? target_items : attn_grid(c);
   c->attn_min_chunk = min_kv_tiles ? min_kv_tiles : 4;
   return HSD_OK;
 }

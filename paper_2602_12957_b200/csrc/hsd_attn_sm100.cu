@@ -722,8 +722,6 @@ int launch_attn_sm100(cudaStream_t st, const CUtensorMap& tmQ, const CUtensorMap
   p.split_ws = split_ws;
   p.anc = anc;
   p.status = status;
-  // (the grid stays two CTAs per SM for head_dim 128 as well, where one is resident at a time: the item walk and the
-  // plan's item count do not depend on the head size)
   if (which)
     return launch_kernel(attn_sm100_kernel<128>, dim3(plan.grid), dim3(kAttnThreads), AttnCfg<128>::SMEM, st, pdl, tmQ, tmK,
                          tmV, p);
