@@ -139,11 +139,12 @@ __device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, const 
                : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void bulk_wait_read() {
   asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
 }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 
 // 16-byte chunk `c` of this lane's 128-byte staging row, at its 128-byte-swizzle position.
 __device__ __forceinline__ uint4* stg_chunk(uint8_t* buf, int lane, int c) {
@@ -341,6 +342,17 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
         for (int i = 0; i < 16; ++i) cs[i] = __ldg(src + i);
       }
+      // likewise the two words the K/V stores depend on (read here, used after the accumulator is ready).  row_kv
+      // comes from the step's set-up kernel: after a failed device-side check it was not written, so nothing is
+      // stored through it (q included: the step is a no-op), nor through a row outside the pool
+      bool live = true;
+      int phys = 0;
+      if (MODE == GS_QKV_ROPE || MODE == GS_QKV_ROPE128) {
+        const int st_word = p.status ? *p.status : 0;
+        const int kv_row = row_ok ? p.qkv.row_kv[row] : 0;
+        live = st_word == 0;
+        phys = live ? kv_row : 0;
+      }
       bool ok = mbar_wait(tfull + b, aph, abort_flag, p.status, 300);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) goto done;
@@ -444,10 +456,6 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           if (nxt >= n0 && nxt < n0 + BN) p.out.zdraft[row] = zd;
         }
       } else if (MODE == GS_QKV_ROPE) {
-        // row_kv comes from the step's set-up kernel: after a failed device-side check it was not written, so
-        // nothing is stored through it (q included: the step is a no-op), nor through a row outside the pool
-        const bool live = !(p.status && *p.status);
-        int phys = (row_ok && live) ? p.qkv.row_kv[row] : 0;
         const bool kv_ok = live && phys >= 0 && phys < p.qkv.kv_rows;
         if (!kv_ok) phys = 0;
         const int blk = phys >> 6, off = phys & 63;
@@ -530,8 +538,6 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         // worked in two passes of 32 pairs (columns [32c, 32c+32) with [64+32c, 64+32c+32)); the row's (cos, sin) of
         // those 32 frequencies come from the table per pass.  q leaves through two staging buffers (dims 0..63 and
         // 64..127), both filled by the two passes and stored together.
-        const bool live = !(p.status && *p.status);
-        int phys = (row_ok && live) ? p.qkv.row_kv[row] : 0;
         const bool kv_ok = live && phys >= 0 && phys < p.qkv.kv_rows;
         if (!kv_ok) phys = 0;
         const int blk = phys >> 6, off = phys & 63;
@@ -630,7 +636,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         if (PAIR) mbar_arrive_even_cta(tempty + b); else mbar_arrive(tempty + b);
       }
     }
-    if (lane == 0) bulk_wait_all();               // staged rows have reached global memory
+    if (lane == 0) bulk_wait_all();               // staged rows have reached global memory (waiting only for the
+                                                  // staging reads measured no shorter)
   }
 
 done:
