@@ -192,20 +192,22 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const bf16* __restri
   const int src = sel_rows ? sel_rows[r] : r;
   if (src < 0 || src >= src_rows) return;
   const float4* xp = reinterpret_cast<const float4*>(x + (size_t)src * d);
+  const uint2* gp = reinterpret_cast<const uint2*>(gain);
   float4 v[VEC];
+  uint2 gv[VEC];
+#pragma unroll
+  for (int i = 0; i < VEC; ++i) v[i] = xp[lane + 32 * i];
+#pragma unroll
+  for (int i = 0; i < VEC; ++i) gv[i] = __ldg(gp + lane + 32 * i);      // in flight together with the row
   float ss = 0.f;
 #pragma unroll
-  for (int i = 0; i < VEC; ++i) {
-    v[i] = xp[lane + 32 * i];
-    ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
-  }
+  for (int i = 0; i < VEC; ++i) ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
   for (int o = 16; o; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
   const float rs = rsqrtf(ss / (float)d + eps);
-  const uint2* gp = reinterpret_cast<const uint2*>(gain);
   uint2* hp = reinterpret_cast<uint2*>(h + (size_t)r * d);
 #pragma unroll
   for (int i = 0; i < VEC; ++i) {
-    uint2 g = gp[lane + 32 * i];
+    const uint2 g = gv[i];
     uint2 o;
     o.x = pack_bf16(v[i].x * rs * bf16_lo(g.x), v[i].y * rs * bf16_hi(g.x));
     o.y = pack_bf16(v[i].z * rs * bf16_lo(g.y), v[i].w * rs * bf16_hi(g.y));
