@@ -39,9 +39,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # captures summarised under profiles/, per workload; a class is absent (-> null) when its kernel has changed since
 # its counters were taken, or when no capture of that workload exists.
 NCU_TRAFFIC_BYTES = {
-    "region": {"attention": 30_961_408 + 11_008, "gemm_gate_up": 19_521_792 + 256, "gemm_qkv": 7_282_432,
-               "gemm_o": 10_249_728, "gemm_down": 24_669_184 + 768},
-    "long2048": {"attention": 43_087_104 + 4_455_424},
+    "region": {"attention": 30_975_744 + 4_352, "gemm_gate_up": 19_522_048, "gemm_qkv": 7_284_992 + 1_280,
+               "gemm_o": 10_249_984, "gemm_down": 24_669_696},
+    "long2048": {"attention": 42_460_928 + 4_530_176},
 }
 
 
