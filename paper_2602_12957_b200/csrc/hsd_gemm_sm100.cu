@@ -347,6 +347,8 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       // stored through it (q included: the step is a no-op), nor through a row outside the pool
       bool live = true;
       int phys = 0;
+      int nxt = -1;                                 // LM head: the row's next draft token (its logit is captured)
+      if (MODE == GS_ARGMAX) nxt = (row_ok && p.out.row_next) ? p.out.row_next[row] : -1;
       if (MODE == GS_QKV_ROPE || MODE == GS_QKV_ROPE128) {
         const int st_word = p.status ? *p.status : 0;
         const int kv_row = row_ok ? p.qkv.row_kv[row] : 0;
@@ -435,7 +437,6 @@ gemm_sm100_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           ++n_stores;
         }
       } else if (MODE == GS_ARGMAX) {
-        const int nxt = (row_ok && p.out.row_next) ? p.out.row_next[row] : -1;
         float best_v = -INFINITY, zd = 0.f;
         int best_c = n0;
 #pragma unroll 1

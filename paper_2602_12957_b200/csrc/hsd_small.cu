@@ -394,11 +394,13 @@ __global__ void accept_kernel(AcceptArgs a, RowMeta rm, const int* status) {
   const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (i >= a.n_seqs) return;
   const int lane = threadIdx.x & 31;
-  if (*status) {            // a failed step decides nothing: -1 makes the commit that follows leave the lengths alone
+  // (three independent reads in flight together; after a failed check the two row words are unwritten and unused)
+  const int failed = *status;
+  const int q0 = rm.seq_q0[i], n = rm.seq_n[i];
+  if (failed) {             // a failed step decides nothing: -1 makes the commit that follows leave the lengths alone
     if (lane == 0) { a.accept_len[i] = -1; a.n_emit[i] = 0; }
     return;
   }
-  const int q0 = rm.seq_q0[i], n = rm.seq_n[i];
   if (n <= 0) {
     if (lane == 0) { a.accept_len[i] = 0; a.n_emit[i] = 0; }
     return;
