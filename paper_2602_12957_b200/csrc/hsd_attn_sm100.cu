@@ -511,9 +511,13 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             if (!((v1 >> e) & 1u)) s1[e] = 0xff800000u;
           }
         }
-        float mx = -INFINITY;
+        float mx = -INFINITY, mx_b = -INFINITY;              // two chains
 #pragma unroll
-        for (int e = 0; e < 32; ++e) mx = max3(mx, __uint_as_float(s0[e]), __uint_as_float(s1[e]));
+        for (int e = 0; e < 32; e += 2) {
+          mx = max3(mx, __uint_as_float(s0[e]), __uint_as_float(s1[e]));
+          mx_b = max3(mx_b, __uint_as_float(s0[e + 1]), __uint_as_float(s1[e + 1]));
+        }
+        mx = fmaxf(mx, mx_b);
         // The row's maximum over all 128 keys: the two threads of a row swap their halves' maxima through shared memory.
         // Both use the bf16-rounded values of BOTH halves, so they arrive at the same number (the reference only has to
         // be near the maximum, and identical for the row's two threads).
@@ -540,23 +544,23 @@ attn_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           }
         }
         const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-        float sum = 0.f;
+        float sum = 0.f, sum_b = 0.f, sum_c = 0.f, sum_d = 0.f;   // four chains
         uint32_t pk[32];
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
           const float a0 = ex2(fmaf(__uint_as_float(s0[2 * e]), sc, -m_use));
           const float a1 = ex2(fmaf(__uint_as_float(s0[2 * e + 1]), sc, -m_use));
-          sum += a0 + a1;
+          if (e & 1) sum_b += a0 + a1; else sum += a0 + a1;
           pk[e] = pack_bf16(a0, a1);
         }
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
           const float a0 = ex2(fmaf(__uint_as_float(s1[2 * e]), sc, -m_use));
           const float a1 = ex2(fmaf(__uint_as_float(s1[2 * e + 1]), sc, -m_use));
-          sum += a0 + a1;
+          if (e & 1) sum_d += a0 + a1; else sum_c += a0 + a1;
           pk[16 + e] = pack_bf16(a0, a1);
         }
-        l = l * alpha + sum;
+        l = l * alpha + ((sum + sum_b) + (sum_c + sum_d));
         // P's columns are read by the product of tile t - 1, which also still adds into the accumulator
         if (t > 0) {
           ok = mbar_wait(o_full, (t - 1) & 1, abort_flag, p.status, 421);
