@@ -424,6 +424,21 @@ class Runner:
         clocks["sampled"] = "timed region"
         return ms, clocks, steps
 
+    def per_step_stats(self, n=50):
+        """Median and minimum over `n` replays timed one by one (an event pair around each), in a pass of its own."""
+        torch = self.torch
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+        with torch.cuda.stream(self.stream):
+            for _ in range(3):
+                self.run()
+            evs[0].record(self.stream)
+            for i in range(n):
+                self.run()
+                evs[i + 1].record(self.stream)
+            self.stream.synchronize()
+        t = sorted(evs[i].elapsed_time(evs[i + 1]) for i in range(n))
+        return {"median": t[n // 2], "min": t[0], "replays": n}
+
     def draft_tokens(self):
         if self.tree:          # the nodes the device actually packed
             return int(self.bout["n_rows"].sum().item()) - self.st["S"]
@@ -610,6 +625,7 @@ def run_ours(args):
     uuid = str(torch.cuda.get_device_properties(dev).uuid)
     uuid = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
     ms_step, clocks, _ = runner.timed(args.steps, barrier, uuid)
+    one_by_one = runner.per_step_stats(100)
     if clocks["samples"] < 3:        # a short timed region leaves nvidia-smi nothing to sample: replay longer
         sampler = ClockSampler(uuid)
         with torch.cuda.stream(stream):
@@ -703,6 +719,7 @@ def run_ours(args):
             roof2, sroof2, kern2, ctx2 = roofline_report(st2, pr2, 5, ms2, clk2, peaks, peak_src, NCU_TRAFFIC_BYTES.get(name))
             tok2 = r2.draft_tokens()
             extra[name] = {"workload": WORKLOADS[name], "ms_per_step": ms2, "steps": n2, "tokens_per_s": tok2 / (ms2 * 1e-3),
+                           "ms_per_step_one_by_one": r2.per_step_stats(),
                            "draft_tokens": tok2, "query_rows": st2["total_q"], "context_tokens": int(sum(ctx2)),
                            "launches_per_step": int(r2.launches_per_step),
                            "step_roofline_frac": sroof2["frac"], "step_roofline_frac_of_burst": sroof2["frac_of_burst"],
@@ -731,7 +748,8 @@ def run_ours(args):
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+                "warmup": max(3, args.warmup), "ms_per_step": ms_step, "ms_per_step_one_by_one": one_by_one,
+                "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                 "config": {"workload": WORKLOADS[args.workload] + (f" [64 regions only, every draft {args.mixed_k} tokens]"
                                                                    if args.workload == "mixed" and args.mixed_k else ""),
